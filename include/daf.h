@@ -1,0 +1,172 @@
+/*
+ * daf.h - C ABI of the B200 (sm_100a) library for the prefill-attention path of
+ * Decoupled Attention Fusion (DAF).
+ *
+ * The path, per layer (paper, section "Methods", items 1-3):
+ *   daf_select          important-token selection, gather into the condensed
+ *                       sequence, hybrid KV-cache update              (items 1, 2)
+ *   daf_important_attn  self-attention among the condensed tokens     (item 1)
+ *   daf_qd_attn         question rows over the hybrid cache           (item 2)
+ *   daf_fuse            state fusion into the final hidden-state rows (item 3)
+ *   daf_full_causal_attn  full recomputation, the comparison path (section
+ *                       "Preliminary Results", the full-recompute baseline)
+ *
+ * Conventions, unless an argument says otherwise
+ *   - Every data pointer is a DEVICE pointer owned by the caller, 16-byte
+ *     aligned.  The library allocates no device memory; scratch comes from the
+ *     caller's `workspace` (size from daf_workspace_bytes), which must not be
+ *     shared by calls that may overlap on the GPU.
+ *   - Tensors are token-major [tokens, heads, head_dim], bf16, contiguous,
+ *     head_dim = 128.  N = L_d + L_q.
+ *   - Calls enqueue work on `stream` (a cudaStream_t passed as void*, NULL = the
+ *     default stream) and return without synchronising.
+ *   - Return value: DAF_OK or a negative daf_status.  Arguments are validated on
+ *     the host before anything is launched; a call that fails validation
+ *     launches nothing.  Device-side problems (a bounded wait that ran out)
+ *     are recorded in the workspace status word and read by daf_poll_status.
+ *     Nothing aborts, traps or throws.
+ */
+#ifndef DAF_H_
+#define DAF_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum daf_status {
+    DAF_OK = 0,
+    DAF_ERR_INVALID_ARG = -1, /* NULL where a buffer is required, negative size, r out of range, ... */
+    DAF_ERR_UNSUPPORTED = -2, /* head_dim != 128, n_q_heads % n_kv_heads != 0, sizes beyond the limits  */
+    DAF_ERR_ALIGNMENT = -3,   /* a pointer or a row stride is not a multiple of 16 bytes              */
+    DAF_ERR_WORKSPACE = -4,   /* workspace missing or smaller than daf_workspace_bytes                */
+    DAF_ERR_CUDA = -5,        /* a CUDA runtime/driver call failed; see daf_last_cuda_error           */
+    DAF_ERR_TIMEOUT = -6,     /* device: a bounded barrier wait ran out (from daf_poll_status)        */
+    DAF_ERR_BOUNDS = -7       /* device: an index outside its tensor was skipped (from daf_poll_status) */
+} daf_status;
+
+/* Problem statement of one layer (paper, "Methods", notation paragraph: L_d, L_q, r). */
+typedef struct daf_params {
+    int32_t L_d;              /* total document tokens                                   */
+    int32_t L_q;              /* question tokens (may be 0)                              */
+    double  r;                /* fraction of document tokens recomputed, 0 <= r <= 1     */
+    int32_t n_q_heads;        /* query heads                                              */
+    int32_t n_kv_heads;       /* key/value heads; must divide n_q_heads                   */
+    int32_t head_dim;         /* must be 128                                              */
+    float   softmax_scale;    /* <= 0 selects 1/sqrt(head_dim)                            */
+    int32_t fuse_mode;        /* 0: compact rows [important ; question]  1: scatter to original positions */
+    int32_t overwrite_doc_kv; /* 1 (the paper's hybrid cache): important rows of the document cache are
+                                 replaced by fresh K/V.  0: document rows stay offline (ablation).       */
+} daf_params;
+
+/* Number of important tokens k = ceil(r * L_d), clamped to [0, L_d].  r*L_d is
+ * shrunk by a relative 1e-6 first so that an r rounded to single precision gives
+ * the intended count.  (Notation paragraph: "r is the fraction of important tokens".) */
+int32_t daf_num_important(int32_t L_d, double r);
+
+/* Bytes of device scratch every call below may need for this problem (selection
+ * keys and histograms, split-KV partial results, the status word). */
+size_t daf_workspace_bytes(const daf_params* p);
+
+/* Clears the status word at the head of a freshly allocated workspace.  Call once
+ * per workspace before its first use (a workspace that is all zero bytes needs no call). */
+int daf_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
+
+/* Step 1 (Methods item 1 "selection", "gather"; item 2 "hybrid KV cache").
+ *   scores   fp32 [n_sig, L_d] per-layer importance signals, summed over n_sig in
+ *            ascending row order in fp32; the k highest sums are selected (ties:
+ *            lower position first; NaN ranks lowest).  NULL: use idx_in instead.
+ *   idx_in   int32 [k] strictly increasing positions in [0, L_d); read iff scores == NULL.
+ *   q_fresh  [N, n_q_heads, 128]; k_fresh, v_fresh [N, n_kv_heads, 128]   (read only)
+ *   kv_k, kv_v  [N, n_kv_heads, 128] IN/OUT: rows < L_d hold the offline document
+ *            cache on entry.  On exit rows idx hold fresh K/V (if overwrite_doc_kv)
+ *            and rows L_d..N-1 hold the fresh question K/V.  Must not alias k_fresh/v_fresh.
+ *   idx_out  int32 [k] selected positions, ascending (also written when idx_in is given)
+ *   q_pack   [k, n_q_heads, 128]; k_pack, v_pack [k, n_kv_heads, 128]: rows idx of the fresh tensors
+ */
+int daf_select(const daf_params* p, const float* scores, int32_t n_sig, const int32_t* idx_in,
+               const void* q_fresh, const void* k_fresh, const void* v_fresh,
+               void* kv_k, void* kv_v,
+               int32_t* idx_out, void* q_pack, void* k_pack, void* v_pack,
+               void* workspace, size_t workspace_bytes, void* stream);
+
+/* Step 2 (Methods item 1; the r^2 L_d^2 term of the complexity analysis): causal
+ * softmax attention among the k packed rows, query head h reading KV head
+ * h / (n_q_heads / n_kv_heads).  bf16 operands, fp32 accumulation and softmax.
+ *   out      bf16; packed row j, head h goes to
+ *            out + dst_rows[j] * out_row_stride_bytes + h * 256   (dst_rows == NULL: row j)
+ *   lse      optional fp32 [n_q_heads, k]: natural-log sum of exponentials of each row
+ */
+int daf_important_attn(const daf_params* p, int32_t k,
+                       const void* q_pack, const void* k_pack, const void* v_pack,
+                       void* out, int64_t out_row_stride_bytes, const int32_t* dst_rows, float* lse,
+                       void* workspace, size_t workspace_bytes, void* stream);
+
+/* Step 3 (Methods item 2): the L_q question rows attend over the L_d + L_q rows of
+ * the hybrid cache; question row i sits at position L_d + i and sees keys <= L_d + i.
+ *   q_question  [L_q, n_q_heads, 128]  (= q_fresh + L_d rows)
+ *   kv_k, kv_v  [N, n_kv_heads, 128]   the hybrid cache left by daf_select
+ *   out, out_row_stride_bytes, dst_rows, lse: as in daf_important_attn, with L_q rows
+ */
+int daf_qd_attn(const daf_params* p, const void* q_question, const void* kv_k, const void* kv_v,
+                void* out, int64_t out_row_stride_bytes, const int32_t* dst_rows, float* lse,
+                void* workspace, size_t workspace_bytes, void* stream);
+
+/* Step 4 (Methods item 3), stand-alone form: copy o_imp [k, n_q_heads*128] and
+ * o_q [L_q, n_q_heads*128] into `hidden`: compact mode -> rows 0..k+L_q-1 of a
+ * [k+L_q, n_q_heads*128] buffer; scatter mode -> rows idx and L_d..N-1 of an
+ * [N, n_q_heads*128] buffer (other rows untouched).  row_pos_out (optional, int32
+ * [k+L_q]) receives the original position of each compact row.  The two attention
+ * calls can write these rows themselves through out/dst_rows; this call exists for
+ * callers that keep the stage outputs separate. */
+int daf_fuse(const daf_params* p, int32_t k, const int32_t* idx, const void* o_imp, const void* o_q,
+             void* hidden, int32_t* row_pos_out, void* stream);
+
+/* Comparison path: causal attention over n_tokens fresh rows (full recomputation). */
+int daf_full_causal_attn(const daf_params* p, int32_t n_tokens, const void* q, const void* k, const void* v,
+                         void* out, float* lse, void* workspace, size_t workspace_bytes, void* stream);
+
+/* One whole layer, steps 1-4 in order with the fusion done by the attention
+ * epilogues (device pointers; arguments as in daf_select, plus)
+ *   hidden       compact: [k+L_q, n_q_heads*128]; scatter: [N, n_q_heads*128]
+ *   row_pos_out  optional int32 [k+L_q]
+ */
+int daf_layer(const daf_params* p, const float* scores, int32_t n_sig, const int32_t* idx_in,
+              const void* q_fresh, const void* k_fresh, const void* v_fresh, void* kv_k, void* kv_v,
+              int32_t* idx_out, void* q_pack, void* k_pack, void* v_pack,
+              void* hidden, int32_t* row_pos_out,
+              void* workspace, size_t workspace_bytes, void* stream);
+
+/* The same layer for callers whose tensors live in HOST memory (pinned memory
+ * makes the copies asynchronous).  h_* are host pointers; every copy to and from
+ * the device is part of the call.  `arena` is caller-owned device memory of at
+ * least daf_layer_host_arena_bytes(p) bytes.
+ *   h_kv_k, h_kv_v  [N, n_kv_heads, 128] host IN/OUT like kv_k/kv_v above
+ *                   (copied back only if copy_back_kv != 0)
+ *   h_hidden        host output, layout by fuse_mode (compact mode recommended)
+ *   h_idx_out       host int32 [k] (optional)
+ * The call synchronises `stream` before returning. */
+size_t daf_layer_host_arena_bytes(const daf_params* p);
+int daf_layer_host(const daf_params* p, const float* h_scores, int32_t n_sig, const int32_t* h_idx_in,
+                   const void* h_q_fresh, const void* h_k_fresh, const void* h_v_fresh,
+                   void* h_kv_k, void* h_kv_v, int32_t copy_back_kv,
+                   void* h_hidden, int32_t* h_idx_out,
+                   void* arena, size_t arena_bytes, void* stream);
+
+/* Reads the device status word kept in `workspace` (synchronises `stream`):
+ * DAF_OK, DAF_ERR_TIMEOUT or DAF_ERR_BOUNDS; the word is cleared. */
+int daf_poll_status(void* workspace, void* stream);
+
+/* Text for a daf_status; the numeric cudaError_t behind the last DAF_ERR_CUDA of this thread. */
+const char* daf_strerror(int status);
+int daf_last_cuda_error(void);
+
+/* Number of kernels this library has launched in this process (for accounting). */
+int64_t daf_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DAF_H_ */

@@ -1,0 +1,355 @@
+// C ABI of the DAF library (see include/daf.h): argument validation, workspace
+// carving and the order of launches.  No arithmetic of the method lives here.
+#include <atomic>
+#include <math.h>
+#include <string.h>
+
+#include "daf_common.cuh"
+
+namespace daf {
+
+static thread_local int g_last_cuda_error = 0;
+static std::atomic<long long> g_launches{0};
+
+void set_cuda_error(cudaError_t e) { g_last_cuda_error = (int)e; }
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+int check_launch() {
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { set_cuda_error(e); return DAF_ERR_CUDA; }
+    return DAF_OK;
+}
+
+static int num_important(int L_d, double r) {
+    if (L_d <= 0 || !(r > 0.0)) return 0;
+    double x = ceil(r * (double)L_d * (1.0 - 1e-6));
+    if (x < 0.0) x = 0.0;
+    if (x > (double)L_d) x = (double)L_d;
+    return (int)x;
+}
+
+constexpr int kMaxTokens = 1 << 22;   // 4M rows: keeps every 32-bit index product in range
+constexpr int kMaxHeads = 256;
+
+int resolve_params(const daf_params* p, ResolvedParams* out) {
+    if (p == nullptr) return DAF_ERR_INVALID_ARG;
+    if (p->L_d < 0 || p->L_q < 0) return DAF_ERR_INVALID_ARG;
+    if (!(p->r >= 0.0) || p->r > 1.0) return DAF_ERR_INVALID_ARG;
+    if (p->n_q_heads <= 0 || p->n_kv_heads <= 0) return DAF_ERR_INVALID_ARG;
+    if (p->fuse_mode != 0 && p->fuse_mode != 1) return DAF_ERR_INVALID_ARG;
+    if (p->head_dim != 128) return DAF_ERR_UNSUPPORTED;
+    if (p->n_q_heads % p->n_kv_heads != 0) return DAF_ERR_UNSUPPORTED;
+    if (p->n_q_heads > kMaxHeads) return DAF_ERR_UNSUPPORTED;
+    if ((long long)p->L_d + p->L_q > kMaxTokens) return DAF_ERR_UNSUPPORTED;
+    out->L_d = p->L_d; out->L_q = p->L_q; out->N = p->L_d + p->L_q;
+    out->Hq = p->n_q_heads; out->Hkv = p->n_kv_heads; out->G = out->Hq / out->Hkv;
+    out->k = num_important(p->L_d, p->r);
+    out->scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf((float)p->head_dim);
+    out->fuse_mode = p->fuse_mode;
+    out->overwrite = p->overwrite_doc_kv != 0;
+    return DAF_OK;
+}
+
+struct Workspace {
+    DeviceStatus* status;
+    void* select_scratch;
+    void* attn_scratch;
+    size_t attn_bytes;
+};
+
+static size_t qd_partial_bytes(const ResolvedParams& rp) {
+    if (rp.L_q == 0) return 0;
+    AttnPlan pl = plan_attention(rp.L_q, rp.N, rp.Hq, rp.G, rp.L_d, true, true);
+    return attn_partial_bytes(rp.L_q, rp.Hq, pl.n_splits);
+}
+
+static size_t workspace_bytes(const ResolvedParams& rp) {
+    return kStatusBytes + select_scratch_bytes(rp.L_d) + qd_partial_bytes(rp);
+}
+
+static int carve_workspace(const ResolvedParams& rp, void* workspace, size_t bytes, Workspace* ws) {
+    if (workspace == nullptr || bytes < workspace_bytes(rp)) return DAF_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return DAF_ERR_ALIGNMENT;
+    char* base = reinterpret_cast<char*>(workspace);
+    ws->status = reinterpret_cast<DeviceStatus*>(base);
+    ws->select_scratch = base + kStatusBytes;
+    ws->attn_scratch = base + kStatusBytes + select_scratch_bytes(rp.L_d);
+    ws->attn_bytes = bytes - kStatusBytes - select_scratch_bytes(rp.L_d);
+    return DAF_OK;
+}
+
+static int do_select(const ResolvedParams& rp, const float* scores, int32_t n_sig, const int32_t* idx_in,
+                     const void* q_fresh, const void* k_fresh, const void* v_fresh, void* kv_k, void* kv_v,
+                     int32_t* idx_out, void* q_pack, void* k_pack, void* v_pack, const Workspace& ws, cudaStream_t st) {
+    if (scores != nullptr && n_sig < 1) return DAF_ERR_INVALID_ARG;
+    if (rp.k > 0) {
+        if (scores == nullptr && idx_in == nullptr) return DAF_ERR_INVALID_ARG;
+        if (scores != nullptr && idx_out == nullptr) return DAF_ERR_INVALID_ARG;
+        if (!q_fresh || !k_fresh || !v_fresh || !q_pack || !k_pack || !v_pack) return DAF_ERR_INVALID_ARG;
+        if (rp.overwrite && (!kv_k || !kv_v)) return DAF_ERR_INVALID_ARG;
+    }
+    if (rp.L_q > 0 && (!k_fresh || !v_fresh || !kv_k || !kv_v)) return DAF_ERR_INVALID_ARG;
+    if (kv_k != nullptr && (kv_k == k_fresh || kv_v == v_fresh)) return DAF_ERR_INVALID_ARG;
+    const void* ptrs[] = {scores, idx_in, q_fresh, k_fresh, v_fresh, kv_k, kv_v, idx_out, q_pack, k_pack, v_pack};
+    for (const void* ptr : ptrs)
+        if (ptr != nullptr && !aligned16(ptr)) return DAF_ERR_ALIGNMENT;
+    return launch_select(rp, scores, n_sig, idx_in, q_fresh, k_fresh, v_fresh, kv_k, kv_v, idx_out, q_pack, k_pack,
+                         v_pack, ws.status, ws.select_scratch, st);
+}
+
+static int check_out(const void* out, int64_t stride_bytes, int Hq) {
+    if (out == nullptr) return DAF_ERR_INVALID_ARG;
+    if (!aligned16(out) || stride_bytes % 16 != 0) return DAF_ERR_ALIGNMENT;
+    if (stride_bytes < (int64_t)Hq * 256) return DAF_ERR_INVALID_ARG;
+    return DAF_OK;
+}
+
+}  // namespace daf
+
+using namespace daf;
+
+extern "C" {
+
+int32_t daf_num_important(int32_t L_d, double r) { return num_important(L_d, r); }
+
+size_t daf_workspace_bytes(const daf_params* p) {
+    ResolvedParams rp;
+    if (resolve_params(p, &rp) != DAF_OK) return 0;
+    return workspace_bytes(rp);
+}
+
+int daf_select(const daf_params* p, const float* scores, int32_t n_sig, const int32_t* idx_in,
+               const void* q_fresh, const void* k_fresh, const void* v_fresh, void* kv_k, void* kv_v,
+               int32_t* idx_out, void* q_pack, void* k_pack, void* v_pack,
+               void* workspace, size_t workspace_bytes_, void* stream) {
+    ResolvedParams rp;
+    if (int rc = resolve_params(p, &rp)) return rc;
+    Workspace ws;
+    if (int rc = carve_workspace(rp, workspace, workspace_bytes_, &ws)) return rc;
+    return do_select(rp, scores, n_sig, idx_in, q_fresh, k_fresh, v_fresh, kv_k, kv_v, idx_out, q_pack, k_pack, v_pack,
+                     ws, (cudaStream_t)stream);
+}
+
+int daf_important_attn(const daf_params* p, int32_t k, const void* q_pack, const void* k_pack, const void* v_pack,
+                       void* out, int64_t out_row_stride_bytes, const int32_t* dst_rows, float* lse,
+                       void* workspace, size_t workspace_bytes_, void* stream) {
+    ResolvedParams rp;
+    if (int rc = resolve_params(p, &rp)) return rc;
+    if (k < 0 || k > rp.L_d) return DAF_ERR_INVALID_ARG;
+    Workspace ws;
+    if (int rc = carve_workspace(rp, workspace, workspace_bytes_, &ws)) return rc;
+    if (k == 0) return DAF_OK;
+    if (!q_pack || !k_pack || !v_pack) return DAF_ERR_INVALID_ARG;
+    if (!aligned16(q_pack) || !aligned16(k_pack) || !aligned16(v_pack)) return DAF_ERR_ALIGNMENT;
+    if (int rc = check_out(out, out_row_stride_bytes, rp.Hq)) return rc;
+    return launch_attention(q_pack, k_pack, v_pack, k, k, rp.Hq, rp.Hkv, 0, rp.scale, false, false, out,
+                            out_row_stride_bytes, dst_rows, lse, ws.status, ws.attn_scratch, ws.attn_bytes,
+                            (cudaStream_t)stream);
+}
+
+int daf_qd_attn(const daf_params* p, const void* q_question, const void* kv_k, const void* kv_v,
+                void* out, int64_t out_row_stride_bytes, const int32_t* dst_rows, float* lse,
+                void* workspace, size_t workspace_bytes_, void* stream) {
+    ResolvedParams rp;
+    if (int rc = resolve_params(p, &rp)) return rc;
+    Workspace ws;
+    if (int rc = carve_workspace(rp, workspace, workspace_bytes_, &ws)) return rc;
+    if (rp.L_q == 0) return DAF_OK;
+    if (!q_question || !kv_k || !kv_v) return DAF_ERR_INVALID_ARG;
+    if (!aligned16(q_question) || !aligned16(kv_k) || !aligned16(kv_v)) return DAF_ERR_ALIGNMENT;
+    if (int rc = check_out(out, out_row_stride_bytes, rp.Hq)) return rc;
+    return launch_attention(q_question, kv_k, kv_v, rp.L_q, rp.N, rp.Hq, rp.Hkv, rp.L_d, rp.scale, true, true, out,
+                            out_row_stride_bytes, dst_rows, lse, ws.status, ws.attn_scratch, ws.attn_bytes,
+                            (cudaStream_t)stream);
+}
+
+int daf_fuse(const daf_params* p, int32_t k, const int32_t* idx, const void* o_imp, const void* o_q,
+             void* hidden, int32_t* row_pos_out, void* stream) {
+    ResolvedParams rp;
+    if (int rc = resolve_params(p, &rp)) return rc;
+    if (k < 0 || k > rp.L_d) return DAF_ERR_INVALID_ARG;
+    rp.k = k;
+    if (hidden == nullptr && row_pos_out == nullptr) return DAF_ERR_INVALID_ARG;
+    if (k > 0 && (idx == nullptr || (hidden != nullptr && o_imp == nullptr))) return DAF_ERR_INVALID_ARG;
+    if (rp.L_q > 0 && hidden != nullptr && o_q == nullptr) return DAF_ERR_INVALID_ARG;
+    if ((o_imp && !aligned16(o_imp)) || (o_q && !aligned16(o_q)) || (hidden && !aligned16(hidden))) return DAF_ERR_ALIGNMENT;
+    return launch_fuse(rp, idx, o_imp, o_q, hidden, row_pos_out, (cudaStream_t)stream);
+}
+
+int daf_full_causal_attn(const daf_params* p, int32_t n_tokens, const void* q, const void* k, const void* v,
+                         void* out, float* lse, void* workspace, size_t workspace_bytes_, void* stream) {
+    ResolvedParams rp;
+    if (int rc = resolve_params(p, &rp)) return rc;
+    if (n_tokens < 0 || n_tokens > kMaxTokens) return DAF_ERR_INVALID_ARG;
+    Workspace ws;
+    if (int rc = carve_workspace(rp, workspace, workspace_bytes_, &ws)) return rc;
+    if (n_tokens == 0) return DAF_OK;
+    if (!q || !k || !v) return DAF_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v)) return DAF_ERR_ALIGNMENT;
+    if (int rc = check_out(out, (int64_t)rp.Hq * 256, rp.Hq)) return rc;
+    return launch_attention(q, k, v, n_tokens, n_tokens, rp.Hq, rp.Hkv, 0, rp.scale, false, false, out,
+                            (long long)rp.Hq * 256, nullptr, lse, ws.status, ws.attn_scratch, ws.attn_bytes,
+                            (cudaStream_t)stream);
+}
+
+int daf_layer(const daf_params* p, const float* scores, int32_t n_sig, const int32_t* idx_in,
+              const void* q_fresh, const void* k_fresh, const void* v_fresh, void* kv_k, void* kv_v,
+              int32_t* idx_out, void* q_pack, void* k_pack, void* v_pack,
+              void* hidden, int32_t* row_pos_out,
+              void* workspace, size_t workspace_bytes_, void* stream) {
+    ResolvedParams rp;
+    if (int rc = resolve_params(p, &rp)) return rc;
+    Workspace ws;
+    if (int rc = carve_workspace(rp, workspace, workspace_bytes_, &ws)) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (rp.k + rp.L_q == 0) return DAF_OK;
+    if (rp.k > 0 && idx_out == nullptr) return DAF_ERR_INVALID_ARG;
+    const int64_t row_bytes = (int64_t)rp.Hq * 256;
+    if (int rc = check_out(hidden, row_bytes, rp.Hq)) return rc;
+    if (int rc = do_select(rp, scores, n_sig, idx_in, q_fresh, k_fresh, v_fresh, kv_k, kv_v, idx_out, q_pack, k_pack,
+                           v_pack, ws, st)) return rc;
+    char* h = reinterpret_cast<char*>(hidden);
+    // state fusion is done by the attention epilogues: each stage writes its final rows
+    if (rp.k > 0) {
+        const int32_t* dst = rp.fuse_mode == 1 ? idx_out : nullptr;
+        if (int rc = launch_attention(q_pack, k_pack, v_pack, rp.k, rp.k, rp.Hq, rp.Hkv, 0, rp.scale, false, false, h,
+                                      row_bytes, dst, nullptr, ws.status, ws.attn_scratch, ws.attn_bytes, st)) return rc;
+    }
+    if (rp.L_q > 0) {
+        const int64_t first_row = rp.fuse_mode == 1 ? rp.L_d : rp.k;
+        const char* qq = reinterpret_cast<const char*>(q_fresh) + (int64_t)rp.L_d * row_bytes;
+        if (int rc = launch_attention(qq, kv_k, kv_v, rp.L_q, rp.N, rp.Hq, rp.Hkv, rp.L_d, rp.scale, true, true,
+                                      h + first_row * row_bytes, row_bytes, nullptr, nullptr, ws.status,
+                                      ws.attn_scratch, ws.attn_bytes, st)) return rc;
+    }
+    if (row_pos_out != nullptr) {
+        if (int rc = launch_fuse(rp, idx_out, nullptr, nullptr, nullptr, row_pos_out, st)) return rc;
+    }
+    return DAF_OK;
+}
+
+// ---- host-buffer form
+namespace {
+struct Arena {
+    char* ws; size_t ws_bytes;
+    float* scores; int32_t* idx_in; int32_t* idx_out;
+    char *q_fresh, *k_fresh, *v_fresh, *kv_k, *kv_v, *q_pack, *k_pack, *v_pack, *hidden;
+    size_t total;
+};
+size_t up256(size_t x) { return (x + 255) / 256 * 256; }
+void carve_arena(const ResolvedParams& rp, int n_sig, char* base, Arena* a) {
+    size_t off = 0;
+    auto take = [&](size_t bytes) { char* ptr = base ? base + off : nullptr; off += up256(bytes); return ptr; };
+    const size_t qrow = (size_t)rp.Hq * 256, kvrow = (size_t)rp.Hkv * 256;
+    a->ws_bytes = workspace_bytes(rp);
+    a->ws = take(a->ws_bytes);
+    a->scores = reinterpret_cast<float*>(take((size_t)(n_sig > 0 ? n_sig : 1) * rp.L_d * 4));
+    a->idx_in = reinterpret_cast<int32_t*>(take((size_t)rp.L_d * 4));
+    a->idx_out = reinterpret_cast<int32_t*>(take((size_t)rp.L_d * 4));
+    a->q_fresh = take(qrow * rp.N);
+    a->k_fresh = take(kvrow * rp.N);
+    a->v_fresh = take(kvrow * rp.N);
+    a->kv_k = take(kvrow * rp.N);
+    a->kv_v = take(kvrow * rp.N);
+    a->q_pack = take(qrow * rp.k);
+    a->k_pack = take(kvrow * rp.k);
+    a->v_pack = take(kvrow * rp.k);
+    a->hidden = take(qrow * (rp.fuse_mode == 1 ? rp.N : rp.k + rp.L_q));
+    a->total = off;
+}
+constexpr int kArenaSignalRows = 8;   // arena is sized for up to this many signal rows
+}  // namespace
+
+size_t daf_layer_host_arena_bytes(const daf_params* p) {
+    ResolvedParams rp;
+    if (resolve_params(p, &rp) != DAF_OK) return 0;
+    Arena a;
+    carve_arena(rp, kArenaSignalRows, nullptr, &a);
+    return a.total;
+}
+
+#define DAF_CUDA_TRY(expr)                                                \
+    do {                                                                  \
+        cudaError_t e_ = (expr);                                          \
+        if (e_ != cudaSuccess) { set_cuda_error(e_); return DAF_ERR_CUDA; } \
+    } while (0)
+
+int daf_layer_host(const daf_params* p, const float* h_scores, int32_t n_sig, const int32_t* h_idx_in,
+                   const void* h_q_fresh, const void* h_k_fresh, const void* h_v_fresh,
+                   void* h_kv_k, void* h_kv_v, int32_t copy_back_kv,
+                   void* h_hidden, int32_t* h_idx_out,
+                   void* arena, size_t arena_bytes, void* stream) {
+    ResolvedParams rp;
+    if (int rc = resolve_params(p, &rp)) return rc;
+    if (h_scores != nullptr && (n_sig < 1 || n_sig > kArenaSignalRows)) return DAF_ERR_INVALID_ARG;
+    if (arena == nullptr || !aligned16(arena)) return DAF_ERR_WORKSPACE;
+    Arena a;
+    carve_arena(rp, kArenaSignalRows, reinterpret_cast<char*>(arena), &a);
+    if (arena_bytes < a.total) return DAF_ERR_WORKSPACE;
+    if (rp.k + rp.L_q == 0) return DAF_OK;
+    if (!h_q_fresh || !h_k_fresh || !h_v_fresh || !h_kv_k || !h_kv_v || !h_hidden) return DAF_ERR_INVALID_ARG;
+    if (rp.k > 0 && !h_scores && !h_idx_in) return DAF_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t qrow = (size_t)rp.Hq * 256, kvrow = (size_t)rp.Hkv * 256;
+    DAF_CUDA_TRY(cudaMemsetAsync(a.ws, 0, kStatusBytes, st));
+    if (h_scores) DAF_CUDA_TRY(cudaMemcpyAsync(a.scores, h_scores, (size_t)n_sig * rp.L_d * 4, cudaMemcpyHostToDevice, st));
+    else if (rp.k > 0) DAF_CUDA_TRY(cudaMemcpyAsync(a.idx_in, h_idx_in, (size_t)rp.k * 4, cudaMemcpyHostToDevice, st));
+    DAF_CUDA_TRY(cudaMemcpyAsync(a.q_fresh, h_q_fresh, qrow * rp.N, cudaMemcpyHostToDevice, st));
+    DAF_CUDA_TRY(cudaMemcpyAsync(a.k_fresh, h_k_fresh, kvrow * rp.N, cudaMemcpyHostToDevice, st));
+    DAF_CUDA_TRY(cudaMemcpyAsync(a.v_fresh, h_v_fresh, kvrow * rp.N, cudaMemcpyHostToDevice, st));
+    // only the document rows of the cache carry information on entry
+    DAF_CUDA_TRY(cudaMemcpyAsync(a.kv_k, h_kv_k, kvrow * rp.L_d, cudaMemcpyHostToDevice, st));
+    DAF_CUDA_TRY(cudaMemcpyAsync(a.kv_v, h_kv_v, kvrow * rp.L_d, cudaMemcpyHostToDevice, st));
+    if (int rc = daf_layer(p, h_scores ? a.scores : nullptr, n_sig, h_scores ? nullptr : a.idx_in, a.q_fresh, a.k_fresh,
+                           a.v_fresh, a.kv_k, a.kv_v, a.idx_out, a.q_pack, a.k_pack, a.v_pack, a.hidden, nullptr, a.ws,
+                           a.ws_bytes, stream)) return rc;
+    const size_t hidden_rows = rp.fuse_mode == 1 ? rp.N : rp.k + rp.L_q;
+    DAF_CUDA_TRY(cudaMemcpyAsync(h_hidden, a.hidden, qrow * hidden_rows, cudaMemcpyDeviceToHost, st));
+    if (h_idx_out && rp.k > 0) DAF_CUDA_TRY(cudaMemcpyAsync(h_idx_out, a.idx_out, (size_t)rp.k * 4, cudaMemcpyDeviceToHost, st));
+    if (copy_back_kv) {
+        DAF_CUDA_TRY(cudaMemcpyAsync(h_kv_k, a.kv_k, kvrow * rp.N, cudaMemcpyDeviceToHost, st));
+        DAF_CUDA_TRY(cudaMemcpyAsync(h_kv_v, a.kv_v, kvrow * rp.N, cudaMemcpyDeviceToHost, st));
+    }
+    DAF_CUDA_TRY(cudaStreamSynchronize(st));
+    DeviceStatus hs;
+    DAF_CUDA_TRY(cudaMemcpy(&hs, a.ws, sizeof(hs), cudaMemcpyDeviceToHost));
+    return hs.code;
+}
+
+int daf_workspace_init(void* workspace, size_t workspace_bytes_, void* stream) {
+    if (workspace == nullptr || workspace_bytes_ < kStatusBytes) return DAF_ERR_WORKSPACE;
+    DAF_CUDA_TRY(cudaMemsetAsync(workspace, 0, kStatusBytes, (cudaStream_t)stream));
+    return DAF_OK;
+}
+
+int daf_poll_status(void* workspace, void* stream) {
+    if (workspace == nullptr) return DAF_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    DeviceStatus hs;
+    DAF_CUDA_TRY(cudaMemcpyAsync(&hs, workspace, sizeof(hs), cudaMemcpyDeviceToHost, st));
+    DAF_CUDA_TRY(cudaStreamSynchronize(st));
+    if (hs.code != 0) {
+        DAF_CUDA_TRY(cudaMemsetAsync(workspace, 0, sizeof(hs), st));
+        DAF_CUDA_TRY(cudaStreamSynchronize(st));
+    }
+    return hs.code;
+}
+
+const char* daf_strerror(int status) {
+    switch (status) {
+        case DAF_OK: return "ok";
+        case DAF_ERR_INVALID_ARG: return "invalid argument";
+        case DAF_ERR_UNSUPPORTED: return "unsupported shape (head_dim must be 128, n_q_heads a multiple of n_kv_heads)";
+        case DAF_ERR_ALIGNMENT: return "pointer or stride not 16-byte aligned";
+        case DAF_ERR_WORKSPACE: return "workspace missing or too small";
+        case DAF_ERR_CUDA: return "CUDA call failed (see daf_last_cuda_error)";
+        case DAF_ERR_TIMEOUT: return "device-side bounded wait ran out";
+        case DAF_ERR_BOUNDS: return "device-side index out of range";
+        default: return "unknown status";
+    }
+}
+
+int daf_last_cuda_error(void) { return g_last_cuda_error; }
+
+int64_t daf_launch_count(void) { return (int64_t)g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

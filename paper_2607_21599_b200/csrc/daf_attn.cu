@@ -1,0 +1,535 @@
+// Steps 2 and 3 of the DAF layer and the full-recompute comparison path: dense
+// softmax attention with a causal limit (Methods, items 1 and 2; complexity
+// analysis: the r^2 L_d^2 and L_q (L_d + L_q) terms).
+//
+// One kernel serves all three.  A CTA owns up to two 128-row query tiles that
+// share one KV head and walks the key/value tiles they can see:
+//   - one thread issues TMA loads of K and V tiles into a shared-memory ring,
+//   - one thread issues tcgen05 MMAs: S = Q K^T into tensor memory, then
+//     O += P V with P read back from tensor memory,
+//   - one warpgroup per query tile runs the online softmax, one thread per row,
+//     straight out of tensor memory, and writes the final rows.
+// The two query tiles alternate on the tensor pipe so that the softmax of one
+// overlaps the MMAs of the other.
+//
+// A query tile's 128 rows are (token, head) pairs: `Gp` query heads of one KV
+// group times 128/Gp consecutive tokens.  Gp = 1 for the packed causal
+// attention; Gp = group size for the question rows, so that one pass over the
+// KV cache serves every query head of the group.
+#include <math.h>
+
+#include "daf_common.cuh"
+
+namespace daf {
+
+constexpr int kNQ = 2;                  // query tiles per CTA
+constexpr int kBlockM = 128;            // rows per query tile
+constexpr int kBlockN = 128;            // keys per KV tile
+constexpr int kD = 128;                 // head_dim
+constexpr int kStages = 4;              // KV ring slots (K and V tiles alternate through it)
+constexpr int kTileBytes = kBlockN * kD * 2;      // 32 KB: one Q, K or V tile
+constexpr int kHalfBytes = kTileBytes / 2;        // one 64-column half (128-byte rows)
+constexpr int kSoftmaxWarps = 4 * kNQ;
+constexpr int kTmaWarp = kSoftmaxWarps;
+constexpr int kMmaWarp = kSoftmaxWarps + 1;
+constexpr int kAttnThreads = 32 * (kSoftmaxWarps + 2);
+constexpr int kTmemCols = 512;          // S0 S1 O0 O1, 128 fp32 columns each
+constexpr int kMaxSplits = 32;
+constexpr float kRescaleThreshold = 8.0f;   // in log2 units: keep a stale row maximum up to 2^8
+
+struct AttnSmem {
+    uint64_t q_full[kNQ];
+    uint64_t kv_full[kStages];
+    uint64_t kv_empty[kStages];
+    uint64_t s_full[kNQ];
+    uint64_t p_full[kNQ];
+    uint64_t o_done[kNQ];
+    uint32_t tmem_base;
+    int abort_flag;
+};
+constexpr size_t kAttnSmemBytes = 1024 /*alignment slack*/ + (size_t)(kNQ + kStages) * kTileBytes + sizeof(AttnSmem);
+
+struct AttnArgs {
+    int n_q;            // query tokens
+    int n_kv;           // key rows
+    int Hq, G;          // query heads; group size Hq / Hkv
+    int Gp;             // query heads per tile (1 or G)
+    int Tt;             // tokens per tile = 128 / Gp
+    int n_tb;           // token blocks = ceil(n_q / Tt)
+    int causal_off;     // token t sees keys <= t + causal_off
+    int n_splits;       // KV splits (1: write final rows; >1: write partials)
+    int tiles_per_split;
+    float scale;        // softmax scale
+    float scale_log2;   // scale * log2(e)
+    __nv_bfloat16* out; long long out_row_stride;  // elements
+    const int32_t* dst_rows;
+    float* lse;         // [Hq, n_q] or null
+    float* part_o;      // [n_splits, n_q, Hq, 128] fp32, normalised per split
+    float* part_lse;    // [n_splits, n_q, Hq]
+    DeviceStatus* status;
+};
+
+__global__ void __launch_bounds__(kAttnThreads, 1)
+attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
+                const __grid_constant__ CUtensorMap tmap_v, const AttnArgs a) {
+    extern __shared__ unsigned char attn_smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(attn_smem_raw) + 1023) & ~(uintptr_t)1023);
+    unsigned char* q_smem = smem;                                   // kNQ tiles
+    unsigned char* kv_smem = smem + (size_t)kNQ * kTileBytes;       // kStages tiles
+    AttnSmem* sm = reinterpret_cast<AttnSmem*>(kv_smem + (size_t)kStages * kTileBytes);
+
+    // a CTA of this grid (or an earlier kernel sharing the workspace) has already given up: do nothing
+    __shared__ int skip_cta;
+    if (threadIdx.x == 0) skip_cta = (a.status != nullptr && *reinterpret_cast<volatile int*>(&a.status->code) != 0) ? 1 : 0;
+    __syncthreads();
+    if (skip_cta) return;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int pair = (int)gridDim.x - 1 - (int)blockIdx.x;          // heaviest causal work first
+    const int hb = blockIdx.y, split = blockIdx.z;
+    const int h0 = hb * a.Gp;
+    const int g_kv = h0 / a.G;
+
+    // per-tile geometry (uniform across the CTA)
+    int t0[kNQ], n_j[kNQ];
+    const int j_begin = split * a.tiles_per_split;
+    int n_j_max = 0;
+#pragma unroll
+    for (int q = 0; q < kNQ; ++q) {
+        const int tb = pair * kNQ + q;
+        t0[q] = tb * a.Tt;
+        int nj = 0;
+        if (tb < a.n_tb) {
+            const int max_tok = min(a.n_q, t0[q] + a.Tt) - 1;
+            const long long kv_hi = min((long long)a.n_kv, (long long)max_tok + a.causal_off + 1);
+            const int tiles_total = kv_hi > 0 ? (int)((kv_hi + kBlockN - 1) / kBlockN) : 0;
+            nj = max(0, min(tiles_total, j_begin + a.tiles_per_split) - j_begin);
+        }
+        n_j[q] = nj;
+        n_j_max = max(n_j_max, nj);
+    }
+
+    if (threadIdx.x == 0) {
+        for (int q = 0; q < kNQ; ++q) {
+            mbar_init(&sm->q_full[q], 1);
+            mbar_init(&sm->s_full[q], 1);
+            mbar_init(&sm->p_full[q], 128);
+            mbar_init(&sm->o_done[q], 1);
+        }
+        for (int s = 0; s < kStages; ++s) { mbar_init(&sm->kv_full[s], 1); mbar_init(&sm->kv_empty[s], 1); }
+        sm->abort_flag = 0;
+        mbar_fence_init();
+    }
+    if (warp == kMmaWarp) {
+        tmem_alloc(&sm->tmem_base, kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = sm->tmem_base;
+    volatile int* abort_flag = &sm->abort_flag;
+
+    if (warp == kTmaWarp) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            tma_prefetch_desc(&tmap_q);
+            tma_prefetch_desc(&tmap_k);
+            tma_prefetch_desc(&tmap_v);
+            const uint32_t q_tx = 2u * 128u * (uint32_t)(a.Gp * a.Tt);
+            for (int q = 0; q < kNQ; ++q) {
+                if (n_j[q] > 0) {
+                    unsigned char* dst = q_smem + (size_t)q * kTileBytes;
+                    mbar_arrive_expect_tx(&sm->q_full[q], q_tx);
+                    tma_load_3d(dst, &tmap_q, &sm->q_full[q], 0, h0, t0[q]);
+                    tma_load_3d(dst + kHalfBytes, &tmap_q, &sm->q_full[q], 64, h0, t0[q]);
+                }
+            }
+            bool ok = true;
+            int seq = 0;
+            for (int j = 0; j < n_j_max && ok; ++j) {
+                const int key0 = (j_begin + j) * kBlockN;
+                for (int kv = 0; kv < 2 && ok; ++kv, ++seq) {
+                    const int slot = seq % kStages;
+                    const uint32_t round = (uint32_t)(seq / kStages);
+                    if (round > 0) ok = mbar_wait(&sm->kv_empty[slot], (round - 1) & 1u, abort_flag, a.status, 10 + slot);
+                    if (!ok) break;
+                    unsigned char* dst = kv_smem + (size_t)slot * kTileBytes;
+                    const CUtensorMap* tm = kv == 0 ? &tmap_k : &tmap_v;
+                    mbar_arrive_expect_tx(&sm->kv_full[slot], (uint32_t)kTileBytes);
+                    tma_load_3d(dst, tm, &sm->kv_full[slot], 0, g_kv, key0);
+                    tma_load_3d(dst + kHalfBytes, tm, &sm->kv_full[slot], 64, g_kv, key0);
+                }
+            }
+            if (!ok) {
+                // give loads already in flight a bounded chance to land before the CTA retires
+                for (int s = 0; s < kStages; ++s)
+                    for (int it = 0; it < 4096 && !mbar_try_wait(&sm->kv_full[s], 0) && !mbar_try_wait(&sm->kv_full[s], 1); ++it) {}
+            }
+        }
+    } else if (warp == kMmaWarp) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0 && n_j_max > 0) {
+            constexpr uint32_t idesc_qk = make_idesc_bf16(kBlockM, kBlockN, 0);
+            constexpr uint32_t idesc_pv = make_idesc_bf16(kBlockM, kD, 1);
+            bool ok = true;
+            for (int q = 0; q < kNQ && ok; ++q)
+                if (n_j[q] > 0) ok = mbar_wait(&sm->q_full[q], 0, abort_flag, a.status, 20 + q);
+            auto slot_of = [](int seq) { return seq % kStages; };
+            auto parity_of = [](int seq) { return (uint32_t)((seq / kStages) & 1); };
+            auto issue_qk = [&](int q, int slot) {
+                const uint32_t qa = smem_u32(q_smem + (size_t)q * kTileBytes);
+                const uint32_t ka = smem_u32(kv_smem + (size_t)slot * kTileBytes);
+#pragma unroll
+                for (int kk = 0; kk < kD / 16; ++kk) {
+                    const uint32_t off = (uint32_t)((kk & 3) * 32 + (kk >> 2) * kHalfBytes);
+                    tc_mma_ss(tmem + (uint32_t)(q * kBlockN), make_smem_desc(qa + off, 16, 1024),
+                              make_smem_desc(ka + off, 16, 1024), idesc_qk, kk > 0 ? 1u : 0u);
+                }
+            };
+            auto issue_pv = [&](int q, int slot, bool first) {
+                const uint32_t va = smem_u32(kv_smem + (size_t)slot * kTileBytes);
+#pragma unroll
+                for (int kk = 0; kk < kBlockN / 16; ++kk) {
+                    // 16 keys per MMA: two 8-key groups of 1024 bytes; the two 64-column halves are kHalfBytes apart
+                    tc_mma_ts(tmem + (uint32_t)(kNQ * kBlockN + q * kD), tmem + (uint32_t)(q * kBlockN + kk * 8),
+                              make_smem_desc(va + (uint32_t)kk * 2048u, kHalfBytes, 1024), idesc_pv,
+                              (first && kk == 0) ? 0u : 1u);
+                }
+            };
+            if (ok) ok = mbar_wait(&sm->kv_full[slot_of(0)], parity_of(0), abort_flag, a.status, 30);
+            if (ok) {
+                tc_fence_after();
+                for (int q = 0; q < kNQ; ++q)
+                    if (n_j[q] > 0) { issue_qk(q, slot_of(0)); tc_commit(&sm->s_full[q]); }
+                tc_commit(&sm->kv_empty[slot_of(0)]);
+            }
+            for (int j = 0; j < n_j_max && ok; ++j) {
+                const int seq_v = 2 * j + 1, seq_k = 2 * j + 2;
+                const bool more = j + 1 < n_j_max;
+                ok = mbar_wait(&sm->kv_full[slot_of(seq_v)], parity_of(seq_v), abort_flag, a.status, 31);
+                if (ok && more) ok = mbar_wait(&sm->kv_full[slot_of(seq_k)], parity_of(seq_k), abort_flag, a.status, 32);
+                if (!ok) break;
+                tc_fence_after();
+                bool last_tile[kNQ];
+                for (int q = 0; q < kNQ && ok; ++q) {
+                    last_tile[q] = false;
+                    if (j >= n_j[q]) continue;
+                    ok = mbar_wait(&sm->p_full[q], (uint32_t)(j & 1), abort_flag, a.status, 40 + q);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_pv(q, slot_of(seq_v), j == 0);
+                    if (j + 1 < n_j[q]) { issue_qk(q, slot_of(seq_k)); tc_commit(&sm->s_full[q]); }
+                    else last_tile[q] = true;
+                }
+                if (!ok) break;
+                tc_commit(&sm->kv_empty[slot_of(seq_v)]);
+                if (more) tc_commit(&sm->kv_empty[slot_of(seq_k)]);
+                // the "output ready" arrival goes last, so that no arrival of this CTA is still
+                // outstanding once its softmax warps have seen it
+                for (int q = 0; q < kNQ; ++q)
+                    if (last_tile[q]) tc_commit(&sm->o_done[q]);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ softmax + epilogue, one row per thread
+        const int q = warp >> 2;
+        const int quad = warp & 3;
+        const int r = quad * 32 + lane;
+        const int tok = t0[q] + r / a.Gp;
+        const int head = h0 + r % a.Gp;
+        const bool row_valid = (r < a.Gp * a.Tt) && (tok < a.n_q) && (n_j[q] > 0 || a.n_splits > 1) &&
+                               (pair * kNQ + q < a.n_tb);
+        const long long lim_ll = (long long)tok + a.causal_off;
+        const int limit = row_valid ? (int)min(lim_ll, (long long)a.n_kv - 1) : -1;   // last visible key
+        const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+        const uint32_t s_addr = tmem + lane_addr + (uint32_t)(q * kBlockN);
+        const uint32_t o_addr = tmem + lane_addr + (uint32_t)(kNQ * kBlockN + q * kD);
+        const float c = a.scale_log2;
+
+        float m = -INFINITY, l = 0.f;
+        bool ok = true;
+        for (int j = 0; j < n_j[q]; ++j) {
+            ok = mbar_wait(&sm->s_full[q], (uint32_t)(j & 1), abort_flag, a.status, 50 + q);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            uint32_t sr[4][32];
+#pragma unroll
+            for (int cchunk = 0; cchunk < 4; ++cchunk) tmem_ld32(s_addr + (uint32_t)(cchunk * 32), sr[cchunk]);
+            tc_wait_ld();
+            const int key0 = (j_begin + j) * kBlockN;
+            if (key0 + kBlockN - 1 > limit) {
+#pragma unroll
+                for (int cchunk = 0; cchunk < 4; ++cchunk)
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        if (key0 + cchunk * 32 + i > limit) sr[cchunk][i] = 0xFF800000u;  // -inf
+            }
+            float tmax = -INFINITY;
+#pragma unroll
+            for (int cchunk = 0; cchunk < 4; ++cchunk)
+#pragma unroll
+                for (int i = 0; i < 32; ++i) tmax = fmaxf(tmax, __uint_as_float(sr[cchunk][i]));
+            float m_new = fmaxf(m, tmax);
+            // keep a slightly stale maximum: rescaling O is skipped while the growth stays below 2^8
+            if (m != -INFINITY && (m_new - m) * c <= kRescaleThreshold) m_new = m;
+            const float m_used = (m_new == -INFINITY) ? 0.f : m_new;
+            const float alpha = (m == -INFINITY) ? 1.f : fast_exp2((m - m_new) * c);
+            const float mc = m_used * c;
+            float rowsum = 0.f;
+            uint32_t pr[2][32];
+#pragma unroll
+            for (int cchunk = 0; cchunk < 4; ++cchunk)
+#pragma unroll
+                for (int i = 0; i < 32; i += 2) {
+                    const float p0 = fast_exp2(fmaf(__uint_as_float(sr[cchunk][i]), c, -mc));
+                    const float p1 = fast_exp2(fmaf(__uint_as_float(sr[cchunk][i + 1]), c, -mc));
+                    rowsum += p0 + p1;
+                    pr[cchunk >> 1][(cchunk & 1) * 16 + (i >> 1)] = pack_bf16(p0, p1);
+                }
+            l = l * alpha + rowsum;
+            m = m_new;
+            // P (bf16, two keys per 32-bit column) overlays the first 64 columns of S
+            tmem_st32(s_addr, pr[0]);
+            tmem_st32(s_addr + 32u, pr[1]);
+            if (j > 0 && __any_sync(0xFFFFFFFFu, alpha != 1.f)) {
+                // the commit that released S_j also covers the previous P V product, so O is quiescent here
+#pragma unroll
+                for (int cchunk = 0; cchunk < 4; ++cchunk) {
+                    uint32_t orr[32];
+                    tmem_ld32(o_addr + (uint32_t)(cchunk * 32), orr);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * alpha);
+                    tmem_st32(o_addr + (uint32_t)(cchunk * 32), orr);
+                }
+            }
+            tc_wait_st();
+            tc_fence_before();
+            mbar_arrive(&sm->p_full[q]);
+        }
+        // ---- epilogue
+        if (ok && n_j[q] > 0) {
+            ok = mbar_wait(&sm->o_done[q], 0, abort_flag, a.status, 60 + q);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+        }
+        if (ok) {
+            tc_fence_after();
+            const float inv_l = l > 0.f ? 1.f / l : 0.f;
+            const float lse_val = l > 0.f ? m * a.scale + logf(l) : -INFINITY;
+            if (a.n_splits == 1) {
+                __nv_bfloat16* dst = nullptr;
+                if (row_valid) {
+                    const long long drow = a.dst_rows ? (long long)a.dst_rows[tok] : (long long)tok;
+                    dst = a.out + drow * a.out_row_stride + (long long)head * kD;
+                    if (a.lse != nullptr) a.lse[(size_t)head * a.n_q + tok] = lse_val;
+                }
+                if (n_j[q] > 0) {
+#pragma unroll
+                    for (int cchunk = 0; cchunk < 4; ++cchunk) {
+                        uint32_t orr[32];
+                        tmem_ld32(o_addr + (uint32_t)(cchunk * 32), orr);
+                        tc_wait_ld();
+                        if (row_valid) {
+                            uint4* d4 = reinterpret_cast<uint4*>(dst + cchunk * 32);
+#pragma unroll
+                            for (int v = 0; v < 4; ++v) {
+                                uint4 w;
+                                w.x = pack_bf16(__uint_as_float(orr[v * 8 + 0]) * inv_l, __uint_as_float(orr[v * 8 + 1]) * inv_l);
+                                w.y = pack_bf16(__uint_as_float(orr[v * 8 + 2]) * inv_l, __uint_as_float(orr[v * 8 + 3]) * inv_l);
+                                w.z = pack_bf16(__uint_as_float(orr[v * 8 + 4]) * inv_l, __uint_as_float(orr[v * 8 + 5]) * inv_l);
+                                w.w = pack_bf16(__uint_as_float(orr[v * 8 + 6]) * inv_l, __uint_as_float(orr[v * 8 + 7]) * inv_l);
+                                d4[v] = w;
+                            }
+                        }
+                    }
+                }
+            } else {
+                const size_t prow = ((size_t)split * a.n_q + (size_t)max(tok, 0)) * a.Hq + head;
+                if (row_valid) a.part_lse[prow] = lse_val;
+                float4* d4 = reinterpret_cast<float4*>(a.part_o + prow * kD);
+                if (n_j[q] > 0) {
+#pragma unroll
+                    for (int cchunk = 0; cchunk < 4; ++cchunk) {
+                        uint32_t orr[32];
+                        tmem_ld32(o_addr + (uint32_t)(cchunk * 32), orr);
+                        tc_wait_ld();
+                        if (row_valid) {
+#pragma unroll
+                            for (int v = 0; v < 8; ++v)
+                                d4[cchunk * 8 + v] = make_float4(__uint_as_float(orr[v * 4 + 0]) * inv_l, __uint_as_float(orr[v * 4 + 1]) * inv_l,
+                                                                 __uint_as_float(orr[v * 4 + 2]) * inv_l, __uint_as_float(orr[v * 4 + 3]) * inv_l);
+                        }
+                    }
+                } else if (row_valid) {
+                    for (int v = 0; v < 32; ++v) d4[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == kMmaWarp) {
+        tc_fence_after();
+        tmem_dealloc(tmem, kTmemCols);
+    }
+}
+
+// Merge of split-KV partials: one warp per (token, head) row.
+__global__ void __launch_bounds__(256)
+attn_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_lse, int n_splits, int n_q, int Hq,
+                    __nv_bfloat16* __restrict__ out, long long out_row_stride, const int32_t* __restrict__ dst_rows,
+                    float* __restrict__ lse) {
+    const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (row >= n_q * Hq) return;
+    const int tok = row / Hq, head = row % Hq;
+    float mx = -INFINITY;
+    for (int s = 0; s < n_splits; ++s) mx = fmaxf(mx, part_lse[(size_t)s * n_q * Hq + row]);
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float wsum = 0.f;
+    for (int s = 0; s < n_splits; ++s) {
+        const float ls = part_lse[(size_t)s * n_q * Hq + row];
+        const float w = (ls == -INFINITY) ? 0.f : __expf(ls - mx);
+        if (w != 0.f) {
+            const float4 v = reinterpret_cast<const float4*>(part_o + ((size_t)s * n_q * Hq + row) * kD)[lane];
+            acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
+            wsum += w;
+        }
+    }
+    const float inv = wsum > 0.f ? 1.f / wsum : 0.f;
+    const long long drow = dst_rows ? (long long)dst_rows[tok] : (long long)tok;
+    uint2 w2;
+    w2.x = pack_bf16(acc.x * inv, acc.y * inv);
+    w2.y = pack_bf16(acc.z * inv, acc.w * inv);
+    reinterpret_cast<uint2*>(out + drow * out_row_stride + (long long)head * kD)[lane] = w2;
+    if (lse != nullptr && lane == 0) lse[(size_t)head * n_q + tok] = wsum > 0.f ? mx + logf(wsum) : -INFINITY;
+}
+
+// ----------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn get_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (fn == nullptr) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres);
+        if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || p == nullptr) {
+            set_cuda_error(e != cudaSuccess ? e : cudaErrorUnknown);
+            return nullptr;
+        }
+        fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// [tokens, heads, 128] bf16 viewed as (d, head, token); a box is 64 columns x box_heads x box_tokens,
+// written to shared memory as 128-byte rows with the 128-byte swizzle.
+static int make_tmap(CUtensorMap* m, const void* base, int tokens, int heads, int box_heads, int box_tokens) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (fn == nullptr) return DAF_ERR_CUDA;
+    cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)heads, (cuuint64_t)tokens};
+    cuuint64_t strides[2] = {(cuuint64_t)kD * 2, (cuuint64_t)heads * kD * 2};
+    cuuint32_t box[3] = {64u, (cuuint32_t)box_heads, (cuuint32_t)box_tokens};
+    cuuint32_t estr[3] = {1u, 1u, 1u};
+    CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { set_cuda_error(cudaErrorInvalidValue); return DAF_ERR_CUDA; }
+    return DAF_OK;
+}
+
+// How a problem is cut into CTAs.  Splitting the KV axis is only used for the
+// question rows, where there are few query tiles and a long KV axis.
+AttnPlan plan_attention(int n_q, int n_kv, int Hq, int G, int causal_off, bool pack_group, bool allow_split) {
+    AttnPlan pl;
+    pl.Gp = pack_group ? G : 1;
+    if (pl.Gp > 128) pl.Gp = 1;
+    pl.Tt = kBlockM / pl.Gp;
+    pl.n_tb = (n_q + pl.Tt - 1) / pl.Tt;
+    pl.pairs = (pl.n_tb + kNQ - 1) / kNQ;
+    pl.head_blocks = Hq / pl.Gp;
+    long long kv_hi = (long long)n_q - 1 + causal_off + 1;
+    if (kv_hi > n_kv) kv_hi = n_kv;
+    const int total_tiles = kv_hi > 0 ? (int)((kv_hi + kBlockN - 1) / kBlockN) : 0;
+    pl.n_splits = 1;
+    pl.tiles_per_split = total_tiles > 0 ? total_tiles : 1;
+    if (allow_split && total_tiles > 1) {
+        const int ctas = pl.pairs * pl.head_blocks;
+        int want = ctas > 0 ? 148 / ctas : 1;
+        if (want > kMaxSplits) want = kMaxSplits;
+        if (want > total_tiles) want = total_tiles;
+        if (want > 1) {
+            pl.tiles_per_split = (total_tiles + want - 1) / want;
+            pl.n_splits = (total_tiles + pl.tiles_per_split - 1) / pl.tiles_per_split;
+        }
+    }
+    return pl;
+}
+
+size_t attn_partial_bytes(int n_q, int Hq, int n_splits) {
+    if (n_splits <= 1) return 0;
+    size_t o = (size_t)n_splits * n_q * Hq * kD * sizeof(float);
+    size_t l = ((size_t)n_splits * n_q * Hq * sizeof(float) + 255) / 256 * 256;
+    return o + l;
+}
+
+int launch_attention(const void* q, const void* k, const void* v, int n_q, int n_kv, int Hq, int Hkv, int causal_off,
+                     float scale, bool pack_group, bool allow_split, void* out, long long out_row_stride_bytes,
+                     const int32_t* dst_rows, float* lse, DeviceStatus* status, void* scratch, size_t scratch_bytes,
+                     cudaStream_t stream) {
+    if (n_q <= 0) return DAF_OK;
+    const int G = Hq / Hkv;
+    AttnPlan pl = plan_attention(n_q, n_kv, Hq, G, causal_off, pack_group, allow_split);
+    const size_t need = attn_partial_bytes(n_q, Hq, pl.n_splits);
+    if (need > scratch_bytes) return DAF_ERR_WORKSPACE;
+
+    CUtensorMap tq, tk, tv;
+    if (int rc = make_tmap(&tq, q, n_q, Hq, pl.Gp, pl.Tt)) return rc;
+    if (int rc = make_tmap(&tk, k, n_kv, Hkv, 1, kBlockN)) return rc;
+    if (int rc = make_tmap(&tv, v, n_kv, Hkv, 1, kBlockN)) return rc;
+
+    static bool attr_done[64] = {false};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !attr_done[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(attn_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttnSmemBytes);
+        if (e != cudaSuccess) { set_cuda_error(e); return DAF_ERR_CUDA; }
+        attr_done[dev] = true;
+    }
+
+    AttnArgs a;
+    a.n_q = n_q; a.n_kv = n_kv; a.Hq = Hq; a.G = G;
+    a.Gp = pl.Gp; a.Tt = pl.Tt; a.n_tb = pl.n_tb;
+    a.causal_off = causal_off;
+    a.n_splits = pl.n_splits; a.tiles_per_split = pl.tiles_per_split;
+    a.scale = scale; a.scale_log2 = scale * 1.4426950408889634f;
+    a.out = reinterpret_cast<__nv_bfloat16*>(out);
+    a.out_row_stride = out_row_stride_bytes / 2;
+    a.dst_rows = dst_rows;
+    a.lse = lse;
+    a.part_o = reinterpret_cast<float*>(scratch);
+    a.part_lse = pl.n_splits > 1 ? reinterpret_cast<float*>(reinterpret_cast<char*>(scratch) +
+                                                            (size_t)pl.n_splits * n_q * Hq * kD * sizeof(float))
+                                 : nullptr;
+    a.status = status;
+    dim3 grid((unsigned)pl.pairs, (unsigned)pl.head_blocks, (unsigned)pl.n_splits);
+    attn_fwd_kernel<<<grid, kAttnThreads, kAttnSmemBytes, stream>>>(tq, tk, tv, a);
+    count_launch();
+    if (int rc = check_launch()) return rc;
+    if (pl.n_splits > 1) {
+        const int rows = n_q * Hq;
+        attn_combine_kernel<<<(rows + 7) / 8, 256, 0, stream>>>(a.part_o, a.part_lse, pl.n_splits, n_q, Hq, a.out,
+                                                                a.out_row_stride, dst_rows, lse);
+        count_launch();
+        if (int rc = check_launch()) return rc;
+    }
+    return DAF_OK;
+}
+
+}  // namespace daf

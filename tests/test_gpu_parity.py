@@ -1,0 +1,356 @@
+"""Parity of the CUDA path (through the C ABI) against the CPU oracle, element by
+element on the same seeded inputs.  Integer and byte results must be identical;
+attention outputs must be within max-abs 2e-2 and mean-abs 2e-3 of the oracle
+(bf16 operands and output, fp32 accumulation), plus a relative Frobenius bound
+that stays meaningful where outputs are small."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2607_21599_b200 import api, build
+from paper_2607_21599_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+MAX_ABS, MEAN_ABS, REL_FRO = 2e-2, 2e-3, 1e-2
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    assert torch.cuda.is_available(), "these tests need a CUDA device"
+    build.build()
+    api.lib()
+    yield
+    torch.cuda.synchronize()
+
+
+def _f(t):
+    return t.float().cpu().numpy()
+
+
+def _assert_close(got_bf16, ref_f64, what):
+    got = got_bf16.float().cpu().numpy().astype(np.float64)
+    assert got.shape == ref_f64.shape, (what, got.shape, ref_f64.shape)
+    assert np.isfinite(got).all(), f"{what}: non-finite output"
+    err = np.abs(got - ref_f64)
+    fro = np.linalg.norm(got - ref_f64) / max(np.linalg.norm(ref_f64), 1e-30)
+    assert err.max() <= MAX_ABS, f"{what}: max-abs {err.max():.3e}"
+    assert err.mean() <= MEAN_ABS, f"{what}: mean-abs {err.mean():.3e}"
+    assert fro <= REL_FRO, f"{what}: relative Frobenius {fro:.3e}"
+
+
+def _ok(status, workspace, what):
+    api.check(status, what)
+    torch.cuda.synchronize()
+    api.check(api.daf_poll_status(workspace), what + " (device status)")
+
+
+def _normal(shape, seed, scale=1.0):
+    return (W.normal_bf16(shape, seed).float() * scale).to(torch.bfloat16)
+
+
+# --------------------------------------------------------------------------- selection
+@pytest.mark.parametrize("L_d,r,n_sig,kind", [
+    (1024, 0.15, 1, "lognormal"), (6144, 0.15, 1, "lognormal"), (16384, 0.10, 3, "lognormal"),
+    (32768, 0.20, 1, "pareto"), (1000, 0.1, 2, "ties"), (777, 1.0, 1, "lognormal"), (130, 0.5, 1, "special"),
+    (50000, 0.07, 1, "lognormal"), (33, 0.03, 1, "ties"), (4096, 0.25, 1, "constant"),
+])
+def test_select_indices_bit_exact(L_d, r, n_sig, kind):
+    if kind == "pareto":
+        w = W.Workload("t", 3, 4, 2, 128, 1, L_d, 512, 0, r, "pareto_clustered", n_sig)
+        S = W.importance_scores(w, 1)
+    else:
+        w = W.Workload("t", 7, 4, 2, 128, 1, L_d, L_d, 0, r, "lognormal", n_sig)
+        S = W.importance_scores(w, 2)
+        if kind == "ties":
+            S = torch.round(S * 2) / 2
+        if kind == "constant":
+            S = torch.full_like(S, 1.5)
+        if kind == "special":
+            S[0, 3] = float("nan"); S[0, 4] = float("inf"); S[0, 5] = -float("inf")
+            S[0, 6] = 0.0; S[0, 7] = -0.0; S[0, 8] = float("nan"); S[0, 9:40] = -S[0, 9:40]
+    p = api.make_params(L_d, 0, r, 4, 2)
+    k = api.daf_num_important(L_d, r)
+    assert k == oracle.num_important(L_d, r)
+    ws = api.alloc_workspace(p)
+    dev = "cuda"
+    H = 4
+    qf = torch.zeros(L_d, H, 128, dtype=torch.bfloat16, device=dev)
+    kf = torch.zeros(L_d, 2, 128, dtype=torch.bfloat16, device=dev)
+    kvk, kvv = torch.zeros_like(kf), torch.zeros_like(kf)
+    idx_out = torch.full((max(k, 1),), -1, dtype=torch.int32, device=dev)
+    qp = torch.zeros(max(k, 1), H, 128, dtype=torch.bfloat16, device=dev)
+    kp = torch.zeros(max(k, 1), 2, 128, dtype=torch.bfloat16, device=dev)
+    vp = torch.zeros_like(kp)
+    _ok(api.daf_select(p, S.to(dev), n_sig, None, qf, kf, kf.clone(), kvk, kvv, idx_out, qp, kp, vp, ws), ws, "daf_select")
+    ref = oracle.select(S.numpy(), k)
+    assert np.array_equal(idx_out[:k].cpu().numpy(), ref)
+
+
+# --------------------------------------------------------------------------- gather / hybrid cache / fusion
+@pytest.mark.parametrize("name,Hq,Hkv,L_d,L_q,r", [("c0", 28, 4, 1024, 32, 0.15), ("x", 8, 8, 300, 7, 0.4),
+                                                  ("y", 40, 8, 513, 0, 0.2), ("z", 4, 1, 64, 5, 0.0)])
+def test_gather_hybrid_cache_and_fuse_bit_exact(name, Hq, Hkv, L_d, L_q, r):
+    w = W.Workload(name, 11, Hq, Hkv, 128, 1, L_d, L_d, L_q, r, "lognormal")
+    L = W.make_layer(w, 0)
+    dev = "cuda"
+    p = api.make_params(L_d, L_q, r, Hq, Hkv)
+    k = api.daf_num_important(L_d, r)
+    ws = api.alloc_workspace(p)
+    N = L_d + L_q
+    g = {n: L[n].to(dev) for n in ("q_fresh", "k_fresh", "v_fresh")}
+    kvk = torch.zeros(N, Hkv, 128, dtype=torch.bfloat16, device=dev)
+    kvv = torch.zeros_like(kvk)
+    kvk[:L_d], kvv[:L_d] = L["k_cached"].to(dev), L["v_cached"].to(dev)
+    kvk[L_d:], kvv[L_d:] = 7.0, 7.0  # stale question rows must be replaced
+    idx_out = torch.full((max(k, 1),), -1, dtype=torch.int32, device=dev)
+    qp = torch.full((max(k, 1), Hq, 128), 3.0, dtype=torch.bfloat16, device=dev)
+    kp = torch.full((max(k, 1), Hkv, 128), 3.0, dtype=torch.bfloat16, device=dev)
+    vp = torch.full_like(kp, 3.0)
+    _ok(api.daf_select(p, L["scores"].to(dev), 1, None, g["q_fresh"], g["k_fresh"], g["v_fresh"], kvk, kvv, idx_out,
+                       qp, kp, vp, ws), ws, "daf_select")
+    idx = oracle.select(L["scores"].numpy(), k)
+    assert np.array_equal(idx_out[:k].cpu().numpy(), idx)
+    assert np.array_equal(_f(qp[:k]), oracle.gather_rows(_f(L["q_fresh"]), idx))
+    assert np.array_equal(_f(kp[:k]), oracle.gather_rows(_f(L["k_fresh"]), idx))
+    assert np.array_equal(_f(vp[:k]), oracle.gather_rows(_f(L["v_fresh"]), idx))
+    assert np.array_equal(_f(kvk), oracle.hybrid_kv(_f(L["k_cached"]), _f(L["k_fresh"]), idx, L_d, L_q))
+    assert np.array_equal(_f(kvv), oracle.hybrid_kv(_f(L["v_cached"]), _f(L["v_fresh"]), idx, L_d, L_q))
+    # the same call with given indices and without overwriting the document rows
+    p0 = api.make_params(L_d, L_q, r, Hq, Hkv, overwrite_doc_kv=0)
+    kvk0 = torch.zeros_like(kvk)
+    kvk0[:L_d] = L["k_cached"].to(dev)
+    kvv0 = kvk0.clone()
+    idx_in = torch.from_numpy(idx).to(dev) if k else None
+    idx_out2 = torch.full((max(k, 1),), -1, dtype=torch.int32, device=dev)
+    _ok(api.daf_select(p0, None, 0, idx_in, g["q_fresh"], g["k_fresh"], g["v_fresh"], kvk0, kvv0, idx_out2, qp, kp,
+                       vp, ws), ws, "daf_select(idx_in)")
+    assert np.array_equal(idx_out2[:k].cpu().numpy(), idx)
+    assert np.array_equal(_f(kvk0), oracle.hybrid_kv(_f(L["k_cached"]), _f(L["k_fresh"]), idx, L_d, L_q, overwrite=False))
+    # stand-alone fusion: compact and scatter placement, canary rows untouched
+    o_imp = _normal((max(k, 1), Hq, 128), 5).to(dev)
+    o_q = _normal((max(L_q, 1), Hq, 128), 6).to(dev)
+    for mode in (0, 1):
+        pm = api.make_params(L_d, L_q, r, Hq, Hkv, fuse_mode=mode)
+        rows = k + L_q if mode == 0 else N
+        hidden = torch.full((rows + 2, Hq, 128), -9.0, dtype=torch.bfloat16, device=dev)  # 2 canary rows
+        row_pos = torch.full((max(k + L_q, 1),), -1, dtype=torch.int32, device=dev)
+        api.check(api.daf_fuse(pm, k, idx_in, o_imp, o_q, hidden, row_pos), "daf_fuse")
+        torch.cuda.synchronize()
+        base = np.full((rows, Hq, 128), -9.0)
+        ref, ref_pos = oracle.fuse(_f(o_imp[:k]).astype(np.float64), _f(o_q[:L_q]).astype(np.float64), idx, L_d,
+                                   mode, hidden=base if mode == 1 else None)
+        assert np.array_equal(_f(hidden[:rows]).astype(np.float64), ref)
+        assert np.all(_f(hidden[rows:]) == -9.0)
+        assert np.array_equal(row_pos[: k + L_q].cpu().numpy(), ref_pos)
+
+
+# --------------------------------------------------------------------------- attention stages
+@pytest.mark.parametrize("n,Hq,Hkv,qscale", [(154, 28, 4, 1.0), (1, 4, 2, 1.0), (128, 4, 4, 1.0), (129, 8, 2, 1.0),
+                                             (300, 40, 8, 1.0), (257, 4, 1, 4.0), (922, 28, 4, 1.0)])
+def test_important_attention_matches_oracle(n, Hq, Hkv, qscale):
+    q, k, v = _normal((n, Hq, 128), 21, qscale), _normal((n, Hkv, 128), 22), _normal((n, Hkv, 128), 23)
+    p = api.make_params(max(n, 1), 0, 1.0, Hq, Hkv)
+    ws = api.alloc_workspace(p)
+    out = torch.full((n + 1, Hq, 128), 5.0, dtype=torch.bfloat16, device="cuda")
+    lse = torch.zeros(Hq, n, dtype=torch.float32, device="cuda")
+    _ok(api.daf_important_attn(p, n, q.cuda(), k.cuda(), v.cuda(), out, Hq * 256, None, lse, ws), ws, "daf_important_attn")
+    scale = 1.0 / math.sqrt(128)
+    ref, ref_lse = oracle.important_attn(_f(q), _f(k), _f(v), scale, return_lse=True)
+    _assert_close(out[:n], ref, f"important attention n={n}")
+    assert torch.all(out[n] == 5.0), "row past the end was written"
+    np.testing.assert_allclose(lse.cpu().numpy().T, ref_lse, atol=2e-3, rtol=0)
+    # first packed row sees one key: its output is that value row exactly
+    assert np.array_equal(_f(out[0]), np.repeat(_f(v[0]), Hq // Hkv, axis=0))
+
+
+def test_important_attention_scatters_rows_through_dst_rows():
+    n, Hq, Hkv = 200, 4, 2
+    q, k, v = _normal((n, Hq, 128), 31), _normal((n, Hkv, 128), 32), _normal((n, Hkv, 128), 33)
+    dst = torch.randperm(400, generator=torch.Generator().manual_seed(1))[:n].sort().values.to(torch.int32)
+    p = api.make_params(n, 0, 1.0, Hq, Hkv)
+    ws = api.alloc_workspace(p)
+    out = torch.full((400, Hq, 128), 5.0, dtype=torch.bfloat16, device="cuda")
+    _ok(api.daf_important_attn(p, n, q.cuda(), k.cuda(), v.cuda(), out, Hq * 256, dst.cuda(), None, ws), ws, "imp")
+    ref = oracle.important_attn(_f(q), _f(k), _f(v), 1.0 / math.sqrt(128))
+    _assert_close(out[dst.long().cuda()], ref, "scattered rows")
+    others = np.setdiff1d(np.arange(400), dst.numpy())
+    assert torch.all(out[torch.from_numpy(others).cuda()] == 5.0)
+
+
+@pytest.mark.parametrize("L_d,L_q,Hq,Hkv,qscale", [(1024, 32, 28, 4, 1.0), (1000, 1, 4, 4, 1.0), (333, 17, 8, 2, 1.0),
+                                                   (2048, 128, 40, 8, 1.0), (640, 64, 32, 8, 4.0), (100, 130, 4, 1, 1.0),
+                                                   (6144, 64, 28, 4, 1.0)])
+def test_question_attention_matches_oracle(L_d, L_q, Hq, Hkv, qscale):
+    N = L_d + L_q
+    q, k, v = _normal((L_q, Hq, 128), 41, qscale), _normal((N, Hkv, 128), 42), _normal((N, Hkv, 128), 43)
+    p = api.make_params(L_d, L_q, 0.1, Hq, Hkv)
+    ws = api.alloc_workspace(p)
+    out = torch.full((L_q + 1, Hq, 128), 5.0, dtype=torch.bfloat16, device="cuda")
+    lse = torch.zeros(Hq, L_q, dtype=torch.float32, device="cuda")
+    _ok(api.daf_qd_attn(p, q.cuda(), k.cuda(), v.cuda(), out, Hq * 256, None, lse, ws), ws, "daf_qd_attn")
+    ref, ref_lse = oracle.qd_attn(_f(q), _f(k), _f(v), L_d, 1.0 / math.sqrt(128), return_lse=True)
+    _assert_close(out[:L_q], ref, f"question attention L_d={L_d} L_q={L_q}")
+    assert torch.all(out[L_q] == 5.0)
+    np.testing.assert_allclose(lse.cpu().numpy().T, ref_lse, atol=2e-3, rtol=0)
+
+
+@pytest.mark.parametrize("n,Hq,Hkv", [(1056, 28, 4), (513, 8, 8)])
+def test_full_causal_attention_matches_oracle(n, Hq, Hkv):
+    q, k, v = _normal((n, Hq, 128), 51), _normal((n, Hkv, 128), 52), _normal((n, Hkv, 128), 53)
+    p = api.make_params(n, 0, 1.0, Hq, Hkv)
+    ws = api.alloc_workspace(p)
+    out = torch.zeros(n, Hq, 128, dtype=torch.bfloat16, device="cuda")
+    _ok(api.daf_full_causal_attn(p, n, q.cuda(), k.cuda(), v.cuda(), out, None, ws), ws, "daf_full_causal_attn")
+    ref = oracle.full_causal_attn(_f(q), _f(k), _f(v), 1.0 / math.sqrt(128))
+    _assert_close(out, ref, f"full causal n={n}")
+
+
+def test_closed_forms_on_the_gpu():
+    """Zero keys give the running mean of the values; constant values come back unchanged."""
+    n, Hq, Hkv = 260, 4, 2
+    q, v = _normal((n, Hq, 128), 61), _normal((n, Hkv, 128), 62)
+    k = torch.zeros(n, Hkv, 128, dtype=torch.bfloat16)
+    p = api.make_params(n, 0, 1.0, Hq, Hkv)
+    ws = api.alloc_workspace(p)
+    out = torch.zeros(n, Hq, 128, dtype=torch.bfloat16, device="cuda")
+    _ok(api.daf_important_attn(p, n, q.cuda(), k.cuda(), v.cuda(), out, Hq * 256, None, None, ws), ws, "imp")
+    mean = np.cumsum(_f(v).astype(np.float64), axis=0) / np.arange(1, n + 1)[:, None, None]
+    _assert_close(out, np.repeat(mean, 2, axis=1), "running mean")
+    vc = torch.full((n, Hkv, 128), 1.75, dtype=torch.bfloat16)
+    _ok(api.daf_important_attn(p, n, q.cuda(), _normal((n, Hkv, 128), 63).cuda(), vc.cuda(), out, Hq * 256, None, None, ws), ws, "imp")
+    assert torch.all((out.float() - 1.75).abs() <= 1.75 * 2 ** -7)
+
+
+# --------------------------------------------------------------------------- whole layer
+def _run_layer(w, layer, fuse_mode, host=False):
+    L = W.make_layer(w, layer)
+    dev = "cuda"
+    p = api.make_params(w.L_d, w.L_q, w.r, w.n_q_heads, w.n_kv_heads, fuse_mode=fuse_mode)
+    k = api.daf_num_important(w.L_d, w.r)
+    N, Hq, Hkv = w.N, w.n_q_heads, w.n_kv_heads
+    rows = k + w.L_q if fuse_mode == 0 else N
+    kv_k = torch.zeros(N, Hkv, 128, dtype=torch.bfloat16)
+    kv_v = torch.zeros_like(kv_k)
+    kv_k[: w.L_d], kv_v[: w.L_d] = L["k_cached"], L["v_cached"]
+    n_sig = 0 if L["scores"] is None else L["scores"].shape[0]
+    if host:
+        arena = torch.zeros(api.daf_layer_host_arena_bytes(p), dtype=torch.uint8, device=dev)
+        hidden = torch.full((rows, Hq, 128), -9.0, dtype=torch.bfloat16).pin_memory()
+        idx_out = torch.full((max(k, 1),), -1, dtype=torch.int32)
+        pin = lambda t: None if t is None else t.pin_memory()  # noqa: E731
+        st = api.daf_layer_host(p, pin(L["scores"]), n_sig, pin(L["idx_in"]), pin(L["q_fresh"]), pin(L["k_fresh"]),
+                                pin(L["v_fresh"]), kv_k, kv_v, 1, hidden, idx_out, arena)
+        api.check(st, "daf_layer_host")
+        return L, hidden, idx_out[:k].numpy(), None, kv_k, kv_v
+    g = {n: (None if t is None else t.to(dev)) for n, t in L.items()}
+    kv_k, kv_v = kv_k.to(dev), kv_v.to(dev)
+    ws = api.alloc_workspace(p)
+    idx_out = torch.full((max(k, 1),), -1, dtype=torch.int32, device=dev)
+    qp = torch.zeros(max(k, 1), Hq, 128, dtype=torch.bfloat16, device=dev)
+    kp = torch.zeros(max(k, 1), Hkv, 128, dtype=torch.bfloat16, device=dev)
+    vp = torch.zeros_like(kp)
+    hidden = torch.full((rows, Hq, 128), -9.0, dtype=torch.bfloat16, device=dev)
+    row_pos = torch.full((max(k + w.L_q, 1),), -1, dtype=torch.int32, device=dev)
+    _ok(api.daf_layer(p, g["scores"], n_sig, g["idx_in"], g["q_fresh"], g["k_fresh"], g["v_fresh"], kv_k, kv_v,
+                      idx_out, qp, kp, vp, hidden, row_pos, ws), ws, "daf_layer")
+    return L, hidden.cpu(), idx_out[:k].cpu().numpy(), row_pos[: k + w.L_q].cpu().numpy(), kv_k.cpu(), kv_v.cpu()
+
+
+def _oracle_layer(w, L, fuse_mode):
+    base = np.full((w.N, w.n_q_heads, 128), -9.0) if fuse_mode == 1 else None
+    return oracle.daf_layer(_f(L["q_fresh"]), _f(L["k_fresh"]), _f(L["v_fresh"]), _f(L["k_cached"]), _f(L["v_cached"]),
+                            w.L_d, w.L_q, w.softmax_scale,
+                            scores=None if L["scores"] is None else L["scores"].numpy(),
+                            idx=None if L["idx_in"] is None else L["idx_in"].numpy(), r=w.r, fuse_mode=fuse_mode,
+                            hidden=base)
+
+
+@pytest.mark.parametrize("fuse_mode", [0, 1])
+def test_layer_smallest_configuration(fuse_mode):
+    w = W.CONFIGS["c0"]
+    L, hidden, idx, row_pos, kv_k, kv_v = _run_layer(w, 0, fuse_mode)
+    ref = _oracle_layer(w, L, fuse_mode)
+    assert np.array_equal(idx, ref["idx"])
+    assert np.array_equal(row_pos, ref["row_pos"])
+    assert np.array_equal(_f(kv_k), ref["kv_k"]) and np.array_equal(_f(kv_v), ref["kv_v"])
+    if fuse_mode == 0:
+        _assert_close(hidden, ref["hidden"], "fused hidden rows (compact)")
+    else:
+        rows = ref["row_pos"]
+        _assert_close(hidden[rows], ref["hidden"][rows], "fused hidden rows (scatter)")
+        others = np.setdiff1d(np.arange(w.N), rows)
+        assert torch.all(hidden[others] == -9.0), "a row that is neither important nor a question row was written"
+    # fused epilogues and the stand-alone fusion pass agree bit for bit
+    p = api.make_params(w.L_d, w.L_q, w.r, w.n_q_heads, w.n_kv_heads, fuse_mode=fuse_mode)
+    ws = api.alloc_workspace(p)
+    k = len(idx)
+    dev = "cuda"
+    idx_d = torch.from_numpy(idx).to(dev)
+    Hq = w.n_q_heads
+    o_imp = torch.zeros(k, Hq, 128, dtype=torch.bfloat16, device=dev)
+    o_q = torch.zeros(w.L_q, Hq, 128, dtype=torch.bfloat16, device=dev)
+    qp = L["q_fresh"][idx].to(dev); kp = L["k_fresh"][idx].to(dev); vp = L["v_fresh"][idx].to(dev)
+    _ok(api.daf_important_attn(p, k, qp, kp, vp, o_imp, Hq * 256, None, None, ws), ws, "imp")
+    _ok(api.daf_qd_attn(p, L["q_fresh"][w.L_d:].to(dev), kv_k.to(dev), kv_v.to(dev), o_q, Hq * 256, None, None, ws), ws, "qd")
+    h2 = torch.full(hidden.shape, -9.0, dtype=torch.bfloat16, device=dev)
+    api.check(api.daf_fuse(p, k, idx_d, o_imp, o_q, h2, None), "daf_fuse")
+    torch.cuda.synchronize()
+    assert torch.equal(h2.cpu(), hidden)
+
+
+def test_layer_with_selection_and_three_signal_rows():
+    w = W.Workload("m", 21, 8, 2, 128, 1, 2000, 500, 48, 0.13, "lognormal", 3)
+    L, hidden, idx, row_pos, kv_k, kv_v = _run_layer(w, 0, 0)
+    ref = _oracle_layer(w, L, 0)
+    assert np.array_equal(idx, ref["idx"]) and np.array_equal(row_pos, ref["row_pos"])
+    assert np.array_equal(_f(kv_k), ref["kv_k"])
+    _assert_close(hidden, ref["hidden"], "layer m")
+
+
+def test_layer_host_buffers():
+    w = W.Workload("h", 22, 8, 2, 128, 1, 1500, 500, 40, 0.2, "pareto_clustered", 1)
+    L, hidden, idx, _, kv_k, kv_v = _run_layer(w, 0, 0, host=True)
+    ref = _oracle_layer(w, L, 0)
+    assert np.array_equal(idx, ref["idx"])
+    assert np.array_equal(_f(kv_k), ref["kv_k"]) and np.array_equal(_f(kv_v), ref["kv_v"])
+    _assert_close(hidden, ref["hidden"], "layer through host buffers")
+
+
+def test_degenerate_sizes():
+    # r = 1 and no question: the layer is full causal attention
+    w = W.Workload("d1", 23, 4, 2, 128, 1, 200, 100, 0, 1.0, "lognormal", 1)
+    L, hidden, idx, _, _, _ = _run_layer(w, 0, 0)
+    assert np.array_equal(idx, np.arange(200))
+    ref_full = oracle.full_causal_attn(_f(L["q_fresh"]), _f(L["k_fresh"]), _f(L["v_fresh"]), w.softmax_scale)
+    _assert_close(hidden, ref_full, "r=1, L_q=0")
+    # r = 0: only the question stage runs
+    w0 = W.Workload("d0", 24, 4, 2, 128, 1, 200, 100, 9, 0.0, "lognormal", 1)
+    L0, hidden0, idx0, row_pos0, kv_k0, _ = _run_layer(w0, 0, 0)
+    ref0 = _oracle_layer(w0, L0, 0)
+    assert len(idx0) == 0 and np.array_equal(row_pos0, ref0["row_pos"])
+    _assert_close(hidden0, ref0["hidden"], "r=0")
+
+
+def test_fresh_change_at_non_important_row_is_invisible():
+    """The hybrid-cache reading: only important rows of the document cache are replaced."""
+    w = W.CONFIGS["c0"]
+    L, hidden, idx, _, _, _ = _run_layer(w, 0, 0)
+    non_imp = int(np.setdiff1d(np.arange(w.L_d), idx)[0])
+    orig = W.make_layer
+
+    def patched(wl, layer, device="cpu"):
+        out = orig(wl, layer, device)
+        out["k_fresh"][non_imp] += 3.0
+        out["v_fresh"][non_imp] -= 2.0
+        return out
+
+    W.make_layer = patched
+    try:
+        _, hidden2, idx2, _, _, _ = _run_layer(w, 0, 0)
+    finally:
+        W.make_layer = orig
+    assert np.array_equal(idx, idx2) and torch.equal(hidden, hidden2)
