@@ -1,0 +1,430 @@
+#!/usr/bin/env python
+"""Benchmark of the DAF prefill-attention path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config c1] [--impl ours|reference]
+
+One step = one pass of the whole path (select + gather + hybrid-cache update,
+important-token attention, question-document attention with the fusion done by
+the epilogues) over every layer of the workload, each layer with its own seeded
+synthetic tensors already resident in HBM.  Prints ONE JSON line.
+
+metric: microseconds per layer (lower is better); the same run also reports the
+algorithmic TFLOP/s, the roofline of the dominant kernel, the full-recompute
+comparison, an end-to-end figure through the host-buffer entry point, and the
+CPU oracle timed on this machine's cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2607_21599_b200 import workloads as W  # noqa: E402
+
+METRIC = "daf_prefill_attention_us_per_layer"
+UNIT = "us/layer"
+
+# DRAM bytes per launch of the dominant kernel from the ncu capture summarised under profiles/
+# (dram__bytes_read.sum + dram__bytes_write.sum); None where no capture exists for the workload.
+NCU_TRAFFIC_BYTES = {}
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"bf16_tflops": float(d["bf16_tflops"]), "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", 0)),
+                "hbm_gbs": float(d["hbm_gbs"]), "source": "measured"}
+    return {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML (read only) while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._nv = None
+
+    def _run(self):
+        nv = self._nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4),
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                try:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
+                except Exception:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+                for n, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(n)
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def __enter__(self):
+        if self._nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        return {"sm_mhz": int(statistics.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def _dist_env():
+    return int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+
+
+def _config_dict(w: W.Workload, n_gpus: int):
+    return {"workload": f"{w.name}: {w.layers} layers, Hq={w.n_q_heads} Hkv={w.n_kv_heads} D={w.head_dim}, "
+                        f"L_d={w.L_d} ({w.n_docs} docs of {w.doc_len}), L_q={w.L_q}, r={w.r} (k={w.k}), "
+                        f"{w.selection} importance scores",
+            "layers": w.layers, "L_d": w.L_d, "L_q": w.L_q, "r": w.r, "k": w.k,
+            "n_q_heads": w.n_q_heads, "n_kv_heads": w.n_kv_heads, "head_dim": w.head_dim,
+            "parallelism": f"replicas x{n_gpus} (no data-path collective)",
+            "l2_policy": "inputs larger than L2: every layer has its own tensors, a step touches far more than 126 MB"}
+
+
+# ----------------------------------------------------------------------------- reference arm (the CPU oracle)
+def run_reference(args, w: W.Workload):
+    rank, _, world = _dist_env()
+    if rank != 0:
+        return
+    import oracle
+    cores = oracle.num_threads()
+    f = lambda t: t.float().numpy()  # noqa: E731
+    layers = [W.make_layer(w, i % w.layers) for i in range(min(w.layers, max(1, args.steps + args.warmup)))]
+    arrs = [{n: (None if t is None else (f(t) if t.dtype == torch.bfloat16 else t.numpy())) for n, t in L.items()}
+            for L in layers]
+
+    def one(i):
+        A = arrs[i % len(arrs)]
+        oracle.daf_layer(A["q_fresh"], A["k_fresh"], A["v_fresh"], A["k_cached"], A["v_cached"], w.L_d, w.L_q,
+                         w.softmax_scale, scores=A["scores"], idx=A["idx_in"], r=w.r)
+
+    for i in range(args.warmup):
+        one(i)
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        one(args.warmup + i)
+    dt = time.perf_counter() - t0
+    us_per_layer = dt / args.steps * 1e6
+    sample = f"each step = one layer of {w.name} through the fp64 CPU oracle (all {cores} OpenMP threads)"
+    line = {"impl": "reference", "metric": METRIC, "value": us_per_layer, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+            "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": _config_dict(w, args.gpus),
+            "cpu_baseline": {"value": us_per_layer, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": us_per_layer, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------- our arm
+class LayerBuffers:
+    """Device tensors of one layer plus the outputs the library writes."""
+
+    def __init__(self, w: W.Workload, layer: int, api, dev):
+        L = W.make_layer(w, layer, dev)
+        self.L = L
+        N, Hq, Hkv = w.N, w.n_q_heads, w.n_kv_heads
+        k = api.daf_num_important(w.L_d, w.r)
+        self.k = k
+        bf = torch.bfloat16
+        self.kv_k = torch.empty(N, Hkv, 128, dtype=bf, device=dev)
+        self.kv_v = torch.empty(N, Hkv, 128, dtype=bf, device=dev)
+        self.kv_k[: w.L_d] = L["k_cached"]
+        self.kv_v[: w.L_d] = L["v_cached"]
+        self.kv_k[w.L_d:] = 0
+        self.kv_v[w.L_d:] = 0
+        self.idx_out = torch.zeros(max(k, 1), dtype=torch.int32, device=dev)
+        self.q_pack = torch.empty(max(k, 1), Hq, 128, dtype=bf, device=dev)
+        self.k_pack = torch.empty(max(k, 1), Hkv, 128, dtype=bf, device=dev)
+        self.v_pack = torch.empty(max(k, 1), Hkv, 128, dtype=bf, device=dev)
+        self.hidden = torch.empty(k + w.L_q, Hq, 128, dtype=bf, device=dev)
+        self.full_out = None
+        self.n_sig = 0 if L["scores"] is None else L["scores"].shape[0]
+
+
+def run_ours(args, w: W.Workload):
+    rank, local_rank, world = _dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the DAF library has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=dev)
+    from paper_2607_21599_b200 import api, build
+    if rank == 0 or world == 1:
+        build.build()
+    if dist is not None:
+        dist.barrier()
+    api.lib()
+    peaks = _peaks()
+
+    p = api.make_params(w.L_d, w.L_q, w.r, w.n_q_heads, w.n_kv_heads)
+    ws = api.alloc_workspace(p, dev)
+    # every rank owns its own replica of the workload (distinct seeds per rank): weak scaling, no exchange
+    bufs = [LayerBuffers(w, rank * w.layers + i, api, dev) for i in range(w.layers)]
+    torch.cuda.synchronize()
+    stream = torch.cuda.current_stream()
+
+    def layer_call(b: LayerBuffers):
+        L = b.L
+        st = api.daf_layer(p, L["scores"], b.n_sig, L["idx_in"], L["q_fresh"], L["k_fresh"], L["v_fresh"], b.kv_k,
+                           b.kv_v, b.idx_out, b.q_pack, b.k_pack, b.v_pack, b.hidden, None, ws, stream)
+        if st != 0:
+            api.check(st, "daf_layer")
+
+    def step():
+        for b in bufs:
+            layer_call(b)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    api.check(api.daf_poll_status(ws), "warm-up (device status)")
+
+    launches0 = api.daf_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local_rank) as clocks:
+        barrier()
+        e0.record(stream)
+        for _ in range(args.steps):
+            step()
+        e1.record(stream)
+        barrier()
+    ms_total = e0.elapsed_time(e1)
+    launches = api.daf_launch_count() - launches0
+    api.check(api.daf_poll_status(ws), "timed region (device status)")
+    if dist is not None:
+        t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_per_step = ms_total / args.steps
+    us_per_layer = ms_per_step * 1e3 / (w.layers * world)
+
+    flops = W.attention_flops(w)
+    daf_flops = flops["important"] + flops["question"]
+    tflops = daf_flops * w.layers * world / (ms_per_step * 1e-3) / 1e12
+
+    # ---- per-stage timings (one launch group at a time, events on the launching stream)
+    def time_stage(fn, reps=3):
+        times = []
+        for _ in range(reps):
+            for b in bufs:
+                a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                fn(b)
+                z.record(stream)
+                times.append((a, z))
+        torch.cuda.synchronize()
+        return statistics.mean(x.elapsed_time(y) for x, y in times) * 1e3  # us
+
+    Hq = w.n_q_heads
+    row_bytes = Hq * 256
+
+    def st_select(b):
+        L = b.L
+        api.check(api.daf_select(p, L["scores"], b.n_sig, L["idx_in"], L["q_fresh"], L["k_fresh"], L["v_fresh"],
+                                 b.kv_k, b.kv_v, b.idx_out, b.q_pack, b.k_pack, b.v_pack, ws, stream), "daf_select")
+
+    def st_imp(b):
+        api.check(api.daf_important_attn(p, b.k, b.q_pack, b.k_pack, b.v_pack, b.hidden, row_bytes, None, None, ws,
+                                         stream), "daf_important_attn")
+
+    def st_qd(b):
+        api.check(api.daf_qd_attn(p, b.L["q_fresh"][w.L_d:], b.kv_k, b.kv_v, b.hidden, row_bytes, None, None, ws,
+                                  stream, out_offset_bytes=b.k * row_bytes), "daf_qd_attn")
+
+    us_select = time_stage(st_select)
+    us_imp = time_stage(st_imp) if w.k > 0 else 0.0
+    us_qd = time_stage(st_qd) if w.L_q > 0 else 0.0
+
+    # ---- full recompute on the same kernels (comparison path), bounded number of layers
+    n_full = min(len(bufs), 4)
+    pf = api.make_params(w.N, 0, 1.0, w.n_q_heads, w.n_kv_heads)
+    wsf = api.alloc_workspace(pf, dev)
+    full_out = torch.empty(w.N, Hq, 128, dtype=torch.bfloat16, device=dev)
+
+    def st_full(b):
+        api.check(api.daf_full_causal_attn(pf, w.N, b.L["q_fresh"], b.L["k_fresh"], b.L["v_fresh"], full_out, None,
+                                           wsf, stream), "daf_full_causal_attn")
+
+    saved = bufs
+    bufs = bufs[:n_full]
+    time_stage(st_full, reps=1)
+    us_full = time_stage(st_full, reps=3)
+    bufs = saved
+    api.check(api.daf_poll_status(wsf), "full recompute (device status)")
+
+    imp_tflops = flops["important"] / (us_imp * 1e-6) / 1e12 if us_imp else 0.0
+    qd_tflops = flops["question"] / (us_qd * 1e-6) / 1e12 if us_qd else 0.0
+    full_tflops = flops["full"] / (us_full * 1e-6) / 1e12
+    gather_bytes = 2 * w.k * (w.n_q_heads + 2 * w.n_kv_heads) * 256 + (w.k + 2 * w.L_q) * 2 * w.n_kv_heads * 256
+
+    dominant_is_imp = flops["important"] >= flops["question"]
+    roofline = {
+        "kernel": "attn_fwd_kernel (" + ("important-token stage" if dominant_is_imp else "question-document stage") + ")",
+        "bound": "tensor",
+        "achieved": imp_tflops if dominant_is_imp else qd_tflops,
+        "peak": peaks["bf16_tflops"],
+        "unit": "TFLOP/s",
+        "frac": (imp_tflops if dominant_is_imp else qd_tflops) / peaks["bf16_tflops"],
+        "peak_source": f"{peaks['source']} bf16 burst (kernel timed alone)",
+        "traffic": NCU_TRAFFIC_BYTES.get(w.name),
+    }
+
+    # ---- end to end through the host-buffer entry point (pinned host tensors, copies inside the timed region)
+    e2e = None
+    if rank == 0 or world > 1:
+        per_layer_in = (w.N * (w.n_q_heads + 2 * w.n_kv_heads) + 2 * w.L_d * w.n_kv_heads) * 256 + \
+                       (w.L_d * 4 * max(bufs[0].n_sig, 1))
+        n_e2e = max(1, min(w.layers, int(4e9 // per_layer_in)))
+        arena = torch.zeros(api.daf_layer_host_arena_bytes(p), dtype=torch.uint8, device=dev)
+        host = []
+        for b in bufs[:n_e2e]:
+            h = {n: (None if t is None else t.cpu().pin_memory()) for n, t in b.L.items()}
+            h["kv_k"] = torch.zeros(w.N, w.n_kv_heads, 128, dtype=torch.bfloat16).pin_memory()
+            h["kv_v"] = torch.zeros(w.N, w.n_kv_heads, 128, dtype=torch.bfloat16).pin_memory()
+            h["kv_k"][: w.L_d] = h["k_cached"]
+            h["kv_v"][: w.L_d] = h["v_cached"]
+            h["hidden"] = torch.empty(b.k + w.L_q, Hq, 128, dtype=torch.bfloat16).pin_memory()
+            h["n_sig"] = b.n_sig
+            host.append(h)
+
+        def e2e_step():
+            for h in host:
+                api.check(api.daf_layer_host(p, h["scores"], h["n_sig"], h["idx_in"], h["q_fresh"], h["k_fresh"],
+                                             h["v_fresh"], h["kv_k"], h["kv_v"], 0, h["hidden"], None, arena, stream),
+                          "daf_layer_host")
+
+        e2e_steps = max(1, min(args.steps, 5))
+        e2e_step()
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            e2e_step()
+        torch.cuda.synchronize()
+        dt = time.perf_counter() - t0
+        if dist is not None:
+            t = torch.tensor([dt], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            dt = float(t.item())
+        e2e = {"value": dt / e2e_steps / (n_e2e * world) * 1e6, "unit": UNIT,
+               "h2d_bytes_per_step": int(per_layer_in * n_e2e), "d2h_bytes_per_step": int((w.k + w.L_q) * row_bytes * n_e2e),
+               "layers_per_step": n_e2e, "steps": e2e_steps,
+               "api": "daf_layer_host (pinned host tensors in, hidden rows out, synchronises)"}
+        del arena, host
+
+    # ---- CPU oracle on this machine's cores, bounded sample (rank 0, N = 1 only)
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        f = lambda t: t.float().cpu().numpy()  # noqa: E731
+        t_cpu, n_cpu = 0.0, 0
+        while t_cpu < 10.0 and n_cpu < w.layers:
+            L = bufs[n_cpu].L
+            A = {n: (None if t is None else (f(t) if t.dtype == torch.bfloat16 else t.cpu().numpy())) for n, t in L.items()}
+            t0 = time.perf_counter()
+            oracle.daf_layer(A["q_fresh"], A["k_fresh"], A["v_fresh"], A["k_cached"], A["v_cached"], w.L_d, w.L_q,
+                             w.softmax_scale, scores=A["scores"], idx=A["idx_in"], r=w.r)
+            t_cpu += time.perf_counter() - t0
+            n_cpu += 1
+        cpu_baseline = {"value": t_cpu / n_cpu * 1e6, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                        "sample": f"first {n_cpu} of {w.layers} layers of {w.name}, whole DAF path per layer, fp64 oracle"}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": us_per_layer, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": _config_dict(w, world),
+            "tflops": tflops, "frac_of_bf16_peak": tflops / (peaks["bf16_tflops"] * world),
+            "roofline": roofline,
+            "stages_us": {"select_gather_update": us_select, "important_attn": us_imp, "question_attn": us_qd},
+            "stages": {
+                "important_attn": {"bound": "tensor", "tflops": imp_tflops, "frac": imp_tflops / peaks["bf16_tflops"]},
+                "question_attn": {"bound": "tensor", "tflops": qd_tflops, "frac": qd_tflops / peaks["bf16_tflops"],
+                                  "kv_gbs": 2 * w.N * w.n_kv_heads * 256 / (us_qd * 1e-6) / 1e9 if us_qd else None},
+                "select_gather_update": {"bound": "hbm", "gbs": gather_bytes / (us_select * 1e-6) / 1e9,
+                                         "frac": gather_bytes / (us_select * 1e-6) / 1e9 / peaks["hbm_gbs"],
+                                         "note": "includes the latency-bound top-k kernel"},
+            },
+            "full_recompute": {"us_per_layer": us_full, "tflops": full_tflops, "frac": full_tflops / peaks["bf16_tflops"],
+                               "speedup_daf_vs_full": us_full / us_per_layer / world if world == 1 else None,
+                               "flop_ratio": flops["full"] / daf_flops, "layers_timed": n_full},
+            "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks.summary(),
+            "peaks": peaks, "cpu_baseline": cpu_baseline,
+        }
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--config", default="c1", help="c0..c3 or a sweep point name (c4_L<L_d>_r<r>)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.config in W.CONFIGS:
+        w = W.CONFIGS[args.config]
+    else:
+        pts = {x.name: x for x in W.sweep_points()}
+        if args.config not in pts:
+            raise SystemExit(f"unknown config {args.config}; choose from {list(W.CONFIGS) + list(pts)}")
+        w = pts[args.config]
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()
