@@ -114,6 +114,33 @@ int daf_qd_attn(const daf_params* p, const void* q_question, const void* kv_k, c
                 void* out, int64_t out_row_stride_bytes, const int32_t* dst_rows, float* lse,
                 void* workspace, size_t workspace_bytes, void* stream);
 
+/* daf_qd_attn for callers that cannot provide a workspace.  (The paper has no
+ * counterpart of this entry point; it exists for integration only.)
+ *
+ * Who needs it: code that runs where device memory can no longer be obtained,
+ * e.g. inside a serving process whose memory pool already owns the whole GPU,
+ * or inside another framework's allocator scope where a driver allocation would
+ * stall every stream.  Such a caller passes inputs and outputs only; the status
+ * word and the split-KV partial results of the question-document stage live in
+ * a fixed 16 MiB array that is part of this library's device image (each GPU
+ * that loads the library holds it until the process exits).  The call makes no
+ * cudaMalloc/cudaFree and calls no allocating routine.
+ *
+ *   - Arguments as in daf_qd_attn, without workspace.
+ *   - Problems whose scratch need exceeds daf_qd_attn_static_max_bytes() are
+ *     rejected with DAF_ERR_WORKSPACE before anything is launched.
+ *   - The first call on each device looks up the array's device address (with
+ *     that device current); make that first call outside any stream capture.
+ *   - All calls on one device share the array, and it keeps the previous call's
+ *     contents; the call clears the part that must start at zero.  Two calls that
+ *     may overlap on the GPU (different streams) race on it: serialise them.
+ *   - Device-side status is not reported through daf_poll_status here; results
+ *     are exactly those of daf_qd_attn. */
+int daf_qd_attn_static(const daf_params* p, const void* q_question, const void* kv_k, const void* kv_v,
+                       void* out, int64_t out_row_stride_bytes, const int32_t* dst_rows, float* lse,
+                       void* stream);
+size_t daf_qd_attn_static_max_bytes(void);
+
 /* Step 4 (Methods item 3), stand-alone form: copy o_imp [k, n_q_heads*128] and
  * o_q [L_q, n_q_heads*128] into `hidden`: compact mode -> rows 0..k+L_q-1 of a
  * [k+L_q, n_q_heads*128] buffer; scatter mode -> rows idx and L_d..N-1 of an

@@ -30,6 +30,7 @@ EXPORTS = [
     "daf_num_important", "daf_workspace_bytes", "daf_workspace_init", "daf_select", "daf_important_attn",
     "daf_qd_attn", "daf_fuse", "daf_full_causal_attn", "daf_layer", "daf_layer_host_arena_bytes",
     "daf_layer_host", "daf_poll_status", "daf_strerror", "daf_last_cuda_error", "daf_launch_count",
+    "daf_qd_attn_static", "daf_qd_attn_static_max_bytes",
 ]
 
 
@@ -84,6 +85,10 @@ def lib() -> ctypes.CDLL:
         L.daf_important_attn.argtypes = [pp, i32, vp, vp, vp, vp, i64, vp, vp, vp, sz, vp]
         L.daf_qd_attn.restype = ctypes.c_int
         L.daf_qd_attn.argtypes = [pp, vp, vp, vp, vp, i64, vp, vp, vp, sz, vp]
+        L.daf_qd_attn_static.restype = ctypes.c_int
+        L.daf_qd_attn_static.argtypes = [pp, vp, vp, vp, vp, i64, vp, vp, vp]
+        L.daf_qd_attn_static_max_bytes.restype = sz
+        L.daf_qd_attn_static_max_bytes.argtypes = []
         L.daf_fuse.restype = ctypes.c_int
         L.daf_fuse.argtypes = [pp, i32, vp, vp, vp, vp, vp, vp]
         L.daf_full_causal_attn.restype = ctypes.c_int
@@ -181,6 +186,18 @@ def daf_qd_attn(p, q_question, kv_k, kv_v, out, out_row_stride_bytes, dst_rows, 
     return lib().daf_qd_attn(ctypes.byref(p), _ptr(q_question), _ptr(kv_k), _ptr(kv_v), o,
                              int(out_row_stride_bytes), _ptr(dst_rows), _ptr(lse), _ptr(workspace),
                              _nbytes(workspace), _stream(stream))
+
+
+def daf_qd_attn_static(p, q_question, kv_k, kv_v, out, out_row_stride_bytes, dst_rows, lse, stream=None) -> int:
+    """Question-document attention without a workspace argument: the scratch is a fixed
+    array inside the library, for callers that cannot hand over (or allocate) device memory.
+    Calls on one device share that array, so they must not overlap on the GPU."""
+    return lib().daf_qd_attn_static(ctypes.byref(p), _ptr(q_question), _ptr(kv_k), _ptr(kv_v), _ptr(out),
+                                    int(out_row_stride_bytes), _ptr(dst_rows), _ptr(lse), _stream(stream))
+
+
+def daf_qd_attn_static_max_bytes() -> int:
+    return int(lib().daf_qd_attn_static_max_bytes())
 
 
 def daf_fuse(p, k, idx, o_imp, o_q, hidden, row_pos_out, stream=None) -> int:

@@ -533,3 +533,70 @@ int launch_attention(const void* q, const void* k, const void* v, int n_q, int n
 }
 
 }  // namespace daf
+
+// ------------------------------------------------------------------------------------------------
+// Allocation-free question-document attention.
+//
+// Some callers hold every byte of device memory themselves and cannot ask the
+// driver for more at the moment they need this step: a serving loop whose memory
+// pool has already claimed the whole GPU, a plug-in running inside another
+// framework's allocator where a driver allocation would stall the device, or a
+// latency-critical path where an allocation's implicit synchronisation is not
+// acceptable.  For them the split-KV partial results and the status word of the
+// question-document stage live in the fixed device array below instead of a
+// caller-provided workspace.  Every GPU that loads this library carries the array
+// until the process exits.
+namespace {
+constexpr size_t kStaticScratchBytes = (size_t)16 << 20;   // 16 MiB: status word + split-KV partials
+static __device__ __align__(256) unsigned char g_qd_static_scratch[kStaticScratchBytes];
+constexpr int kMaxDevices = 64;
+void* g_static_scratch_addr[kMaxDevices] = {nullptr};
+
+// In host code the array's name is only a handle for the runtime, not an address
+// a kernel can use, so the device address is looked up once per device.
+int static_scratch_address(void** out) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) { daf::set_cuda_error(e); return DAF_ERR_CUDA; }
+    if (dev < 0 || dev >= kMaxDevices) return DAF_ERR_UNSUPPORTED;
+    if (g_static_scratch_addr[dev] == nullptr) {
+        void* ptr = nullptr;
+        e = cudaGetSymbolAddress(&ptr, g_qd_static_scratch);
+        if (e != cudaSuccess || ptr == nullptr) {
+            daf::set_cuda_error(e != cudaSuccess ? e : cudaErrorInvalidSymbol);
+            return DAF_ERR_CUDA;
+        }
+        g_static_scratch_addr[dev] = ptr;
+    }
+    *out = g_static_scratch_addr[dev];
+    return DAF_OK;
+}
+}  // namespace
+
+extern "C" size_t daf_qd_attn_static_max_bytes(void) { return kStaticScratchBytes; }
+
+extern "C" int daf_qd_attn_static(const daf_params* p, const void* q_question, const void* kv_k, const void* kv_v,
+                                  void* out, int64_t out_row_stride_bytes, const int32_t* dst_rows, float* lse,
+                                  void* stream) {
+    using namespace daf;
+    ResolvedParams rp;
+    if (int rc = resolve_params(p, &rp)) return rc;
+    if (rp.L_q == 0) return DAF_OK;
+    if (!q_question || !kv_k || !kv_v || !out) return DAF_ERR_INVALID_ARG;
+    if (!aligned16(q_question) || !aligned16(kv_k) || !aligned16(kv_v) || !aligned16(out) ||
+        out_row_stride_bytes % 16 != 0) return DAF_ERR_ALIGNMENT;
+    if (out_row_stride_bytes < (int64_t)rp.Hq * 256) return DAF_ERR_INVALID_ARG;
+    // the fixed array must hold the status word and this problem's split-KV partials
+    const AttnPlan pl = plan_attention(rp.L_q, rp.N, rp.Hq, rp.G, rp.L_d, true, true);
+    const size_t need = kStatusBytes + attn_partial_bytes(rp.L_q, rp.Hq, pl.n_splits);
+    if (need > kStaticScratchBytes) return DAF_ERR_WORKSPACE;   // problem too large for the fixed scratch
+    void* base = nullptr;
+    if (int rc = static_scratch_address(&base)) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    // the array keeps whatever the previous call left: the status word has to start at zero
+    cudaError_t e = cudaMemsetAsync(base, 0, kStatusBytes, st);
+    if (e != cudaSuccess) { set_cuda_error(e); return DAF_ERR_CUDA; }
+    return launch_attention(q_question, kv_k, kv_v, rp.L_q, rp.N, rp.Hq, rp.Hkv, rp.L_d, rp.scale, true, true, out,
+                            out_row_stride_bytes, dst_rows, lse, reinterpret_cast<DeviceStatus*>(base),
+                            reinterpret_cast<char*>(base) + kStatusBytes, kStaticScratchBytes - kStatusBytes, st);
+}
