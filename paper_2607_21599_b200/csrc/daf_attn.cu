@@ -85,8 +85,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     if (skip_cta) return;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int pair = (int)gridDim.x - 1 - (int)blockIdx.x;          // heaviest causal work first
-    const int hb = blockIdx.y, split = blockIdx.z;
+    // blocks are dispatched x-fastest: all head blocks of the heaviest (last) query-tile pair go first
+    const int pair = (int)gridDim.y - 1 - (int)blockIdx.y;
+    const int hb = blockIdx.x, split = blockIdx.z;
     const int h0 = hb * a.Gp;
     const int g_kv = h0 / a.G;
 
@@ -254,40 +255,61 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) break;
             tc_fence_after();
+            // logits of this row: 128 fp32 values, fetched in two halves so that the row maximum of the
+            // first half is computed while the second half is still on its way from tensor memory
             uint32_t sr[4][32];
-#pragma unroll
-            for (int cchunk = 0; cchunk < 4; ++cchunk) tmem_ld32(s_addr + (uint32_t)(cchunk * 32), sr[cchunk]);
+            tmem_ld32(s_addr, sr[0]);
+            tmem_ld32(s_addr + 32u, sr[1]);
             tc_wait_ld();
+            tmem_ld32(s_addr + 64u, sr[2]);
+            tmem_ld32(s_addr + 96u, sr[3]);
             const int key0 = (j_begin + j) * kBlockN;
-            if (key0 + kBlockN - 1 > limit) {
+            const bool need_mask = key0 + kBlockN - 1 > limit;
+            float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-                for (int cchunk = 0; cchunk < 4; ++cchunk)
+            for (int half = 0; half < 2; ++half) {
+                if (half == 1) tc_wait_ld();
+                if (need_mask) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        if (key0 + cchunk * 32 + i > limit) sr[cchunk][i] = 0xFF800000u;  // -inf
+                    for (int cchunk = 2 * half; cchunk < 2 * half + 2; ++cchunk)
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            if (key0 + cchunk * 32 + i > limit) sr[cchunk][i] = 0xFF800000u;  // -inf
+                }
+#pragma unroll
+                for (int cchunk = 2 * half; cchunk < 2 * half + 2; ++cchunk)
+#pragma unroll
+                    for (int i = 0; i < 32; i += 8) {
+                        // four independent chains of 3-input maxima
+                        mx[0] = fmax3(mx[0], __uint_as_float(sr[cchunk][i + 0]), __uint_as_float(sr[cchunk][i + 1]));
+                        mx[1] = fmax3(mx[1], __uint_as_float(sr[cchunk][i + 2]), __uint_as_float(sr[cchunk][i + 3]));
+                        mx[2] = fmax3(mx[2], __uint_as_float(sr[cchunk][i + 4]), __uint_as_float(sr[cchunk][i + 5]));
+                        mx[3] = fmax3(mx[3], __uint_as_float(sr[cchunk][i + 6]), __uint_as_float(sr[cchunk][i + 7]));
+                    }
             }
-            float tmax = -INFINITY;
-#pragma unroll
-            for (int cchunk = 0; cchunk < 4; ++cchunk)
-#pragma unroll
-                for (int i = 0; i < 32; ++i) tmax = fmaxf(tmax, __uint_as_float(sr[cchunk][i]));
+            const float tmax = fmax3(mx[0], mx[1], fmaxf(mx[2], mx[3]));
             float m_new = fmaxf(m, tmax);
             // keep a slightly stale maximum: rescaling O is skipped while the growth stays below 2^8
             if (m != -INFINITY && (m_new - m) * c <= kRescaleThreshold) m_new = m;
             const float m_used = (m_new == -INFINITY) ? 0.f : m_new;
             const float alpha = (m == -INFINITY) ? 1.f : fast_exp2((m - m_new) * c);
             const float mc = m_used * c;
-            float rowsum = 0.f;
+            // p = 2^(s*c - m*c): packed two-wide FMA and adds, exponentials on the special-function unit
+            const uint64_t c2 = pack_f32x2(c, c), nmc2 = pack_f32x2(-mc, -mc);
+            uint64_t acc2[4] = {0ull, 0ull, 0ull, 0ull};
             uint32_t pr[2][32];
 #pragma unroll
             for (int cchunk = 0; cchunk < 4; ++cchunk)
 #pragma unroll
                 for (int i = 0; i < 32; i += 2) {
-                    const float p0 = fast_exp2(fmaf(__uint_as_float(sr[cchunk][i]), c, -mc));
-                    const float p1 = fast_exp2(fmaf(__uint_as_float(sr[cchunk][i + 1]), c, -mc));
-                    rowsum += p0 + p1;
+                    const uint64_t x2 = ffma2(pack_f32x2(__uint_as_float(sr[cchunk][i]), __uint_as_float(sr[cchunk][i + 1])), c2, nmc2);
+                    const float p0 = fast_exp2(f32x2_lo(x2));
+                    const float p1 = fast_exp2(f32x2_hi(x2));
+                    acc2[(i >> 1) & 3] = fadd2(acc2[(i >> 1) & 3], pack_f32x2(p0, p1));
                     pr[cchunk >> 1][(cchunk & 1) * 16 + (i >> 1)] = pack_bf16(p0, p1);
                 }
+            const uint64_t acc01 = fadd2(fadd2(acc2[0], acc2[1]), fadd2(acc2[2], acc2[3]));
+            const float rowsum = f32x2_lo(acc01) + f32x2_hi(acc01);
             l = l * alpha + rowsum;
             m = m_new;
             // P (bf16, two keys per 32-bit column) overlays the first 64 columns of S
@@ -386,18 +408,33 @@ attn_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ 
     const int lane = threadIdx.x & 31;
     if (row >= n_q * Hq) return;
     const int tok = row / Hq, head = row % Hq;
-    float mx = -INFINITY;
-    for (int s = 0; s < n_splits; ++s) mx = fmaxf(mx, part_lse[(size_t)s * n_q * Hq + row]);
+    // lane s holds the log-sum-exp of split s (n_splits <= 32), so all of them are fetched at once
+    const size_t stride = (size_t)n_q * Hq;
+    const float my_lse = lane < n_splits ? part_lse[(size_t)lane * stride + row] : -INFINITY;
+    float mx = my_lse;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
+    const float my_w = (my_lse == -INFINITY) ? 0.f : __expf(my_lse - mx);
+    float wsum = my_w;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) wsum += __shfl_xor_sync(0xFFFFFFFFu, wsum, o);
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    float wsum = 0.f;
-    for (int s = 0; s < n_splits; ++s) {
-        const float ls = part_lse[(size_t)s * n_q * Hq + row];
-        const float w = (ls == -INFINITY) ? 0.f : __expf(ls - mx);
-        if (w != 0.f) {
-            const float4 v = reinterpret_cast<const float4*>(part_o + ((size_t)s * n_q * Hq + row) * kD)[lane];
-            acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
-            wsum += w;
+    const float4* src = reinterpret_cast<const float4*>(part_o + (size_t)row * kD) + lane;
+    int s = 0;
+    for (; s + 4 <= n_splits; s += 4) {
+        float4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) v[u] = __ldcs(src + (size_t)(s + u) * stride * (kD / 4));
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const float w = __shfl_sync(0xFFFFFFFFu, my_w, s + u);
+            acc.x += w * v[u].x; acc.y += w * v[u].y; acc.z += w * v[u].z; acc.w += w * v[u].w;
         }
+    }
+    for (; s < n_splits; ++s) {
+        const float4 v = __ldcs(src + (size_t)s * stride * (kD / 4));
+        const float w = __shfl_sync(0xFFFFFFFFu, my_w, s);
+        acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
     }
     const float inv = wsum > 0.f ? 1.f / wsum : 0.f;
     const long long drow = dst_rows ? (long long)dst_rows[tok] : (long long)tok;
@@ -518,7 +555,7 @@ int launch_attention(const void* q, const void* k, const void* v, int n_q, int n
                                                             (size_t)pl.n_splits * n_q * Hq * kD * sizeof(float))
                                  : nullptr;
     a.status = status;
-    dim3 grid((unsigned)pl.pairs, (unsigned)pl.head_blocks, (unsigned)pl.n_splits);
+    dim3 grid((unsigned)pl.head_blocks, (unsigned)pl.pairs, (unsigned)pl.n_splits);
     attn_fwd_kernel<<<grid, kAttnThreads, kAttnSmemBytes, stream>>>(tq, tk, tv, a);
     count_launch();
     if (int rc = check_launch()) return rc;

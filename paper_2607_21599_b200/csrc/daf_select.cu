@@ -4,19 +4,25 @@
 // These steps move bytes and rank 32-bit keys; they are bound by HBM bandwidth
 // and launch latency, not by arithmetic, so they are plain coalesced 16-byte
 // kernels with no tensor-core work.
+#include <cooperative_groups.h>
+
 #include "daf_common.cuh"
 
 namespace daf {
 
 // ------------------------------------------------------------------ selection
-// One CTA ranks all L_d aggregated scores: an 8-bit-per-pass radix select finds
-// the key of the k-th largest score, then an ordered compaction emits the
-// selected positions in ascending order.  Ties at the threshold are broken by
-// position (lower first), which makes the result unique.
+// A cluster of 8 CTAs ranks all L_d aggregated scores.  Each CTA keeps a
+// contiguous slice of the keys in its shared memory.  Four passes of an
+// 8-bit radix select find the key of the k-th largest score: every CTA builds
+// a 256-bin histogram of its slice, the histograms are summed through
+// distributed shared memory, and every CTA picks the same digit.  An ordered
+// compaction then emits the selected positions in ascending order.  Ties at
+// the threshold are broken by position (lower first), so the result is unique.
 
-constexpr int kSelThreads = 1024;
+constexpr int kSelCluster = 8;
+constexpr int kSelThreads = 512;
 constexpr int kSelWarps = kSelThreads / 32;
-constexpr int kSelSmemKeys = 40960;  // keys kept in shared memory up to this L_d, in global scratch beyond
+constexpr int kSelSmemKeysPerCta = 40960;   // slice kept in shared memory up to this size, in global scratch beyond
 
 // Monotone map fp32 -> uint32: larger score <=> larger key; -0 == +0; NaN -> 0 (ranks lowest).
 __device__ __forceinline__ uint32_t score_key(float s) {
@@ -26,72 +32,94 @@ __device__ __forceinline__ uint32_t score_key(float s) {
     return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
 
-__global__ void __launch_bounds__(kSelThreads, 1)
+struct SelShared {
+    uint32_t hist[2][256];     // double-buffered so that a peer may still read pass p while pass p+1 is filled
+    uint32_t total[256];
+    uint32_t scan_gt[kSelWarps];
+    uint32_t scan_eq[kSelWarps];
+    uint32_t cta_counts[2];    // this CTA's number of keys above / equal to the threshold (read by peers)
+    uint32_t pick[2];          // chosen prefix, remaining rank
+};
+
+__global__ void __cluster_dims__(kSelCluster, 1, 1) __launch_bounds__(kSelThreads, 1)
 select_topk_kernel(const float* __restrict__ scores, int n_sig, int L_d, int k,
                    uint32_t* __restrict__ gkeys, int32_t* __restrict__ idx_out) {
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
     extern __shared__ __align__(16) unsigned char sel_smem[];
-    uint32_t* hist = reinterpret_cast<uint32_t*>(sel_smem);              // [kSelWarps][256]
-    uint32_t* total = hist + kSelWarps * 256;                             // [256]
-    uint32_t* scan_gt = total + 256;                                      // [kSelWarps]
-    uint32_t* scan_eq = scan_gt + kSelWarps;                              // [kSelWarps]
-    uint32_t* sh = scan_eq + kSelWarps;                                   // [4]: prefix, k_rem
-    uint32_t* skeys = sh + 4;
-    uint32_t* keys = (L_d <= kSelSmemKeys) ? skeys : gkeys;
+    SelShared* sh = reinterpret_cast<SelShared*>(sel_smem);
+    uint32_t* skeys = reinterpret_cast<uint32_t*>(sel_smem + sizeof(SelShared));
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int rank = (int)cluster.block_rank();
+    const int per_cta = (L_d + kSelCluster - 1) / kSelCluster;
+    const int lo_cta = min(L_d, rank * per_cta);
+    const int n_loc = min(L_d, lo_cta + per_cta) - lo_cta;
+    uint32_t* keys = (per_cta <= kSelSmemKeysPerCta) ? skeys : (gkeys + lo_cta);
 
     // aggregate the signal rows in ascending row order (fp32 adds, no fusing) and build keys
-    for (int i = tid; i < L_d; i += kSelThreads) {
-        float acc = scores[i];
-        for (int l = 1; l < n_sig; ++l) acc = __fadd_rn(acc, scores[(size_t)l * L_d + i]);
+    for (int i = tid; i < n_loc; i += kSelThreads) {
+        const int g = lo_cta + i;
+        float acc = scores[g];
+        for (int l = 1; l < n_sig; ++l) acc = __fadd_rn(acc, scores[(size_t)l * L_d + g]);
         keys[i] = score_key(acc);
     }
-    if (tid == 0) { sh[0] = 0u; sh[1] = (uint32_t)k; }
+    if (tid < 256) { sh->hist[0][tid] = 0u; sh->hist[1][tid] = 0u; }
+    if (tid == 0) { sh->pick[0] = 0u; sh->pick[1] = (uint32_t)k; }
     __syncthreads();
 
     uint32_t prefix = 0u, mask = 0u;
-    for (int shift = 24; shift >= 0; shift -= 8) {
-        for (int i = tid; i < kSelWarps * 256; i += kSelThreads) hist[i] = 0u;
-        __syncthreads();
-        const int n_round = (L_d + kSelThreads - 1) / kSelThreads * kSelThreads;
+    int pass = 0;
+    for (int shift = 24; shift >= 0; shift -= 8, ++pass) {
+        uint32_t* hist = sh->hist[pass & 1];
+        const int n_round = (n_loc + 31) / 32 * 32;
         for (int i = tid; i < n_round; i += kSelThreads) {
             bool in = false;
-            uint32_t bin = 0xFFFFFFFFu;
-            if (i < L_d) {
+            uint32_t bin = 0u;
+            if (i < n_loc) {
                 const uint32_t key = keys[i];
                 in = (key & mask) == prefix;
-                if (in) bin = (key >> shift) & 0xFFu;
+                bin = (key >> shift) & 0xFFu;
             }
-            // warp-aggregated histogram update: one atomic per distinct bin in the warp
-            const uint32_t peers = __match_any_sync(0xFFFFFFFFu, bin);
-            if (in && (int)(__ffs(peers) - 1) == lane) atomicAdd(&hist[warp * 256 + bin], (uint32_t)__popc(peers));
+            // a warp whose keys all fall in one bin adds once; otherwise every thread adds for itself
+            const uint32_t active = __ballot_sync(0xFFFFFFFFu, in);
+            if (active == 0u) continue;
+            const uint32_t lead_bin = __shfl_sync(0xFFFFFFFFu, bin, __ffs(active) - 1);
+            const uint32_t same = __ballot_sync(0xFFFFFFFFu, in && bin == lead_bin);
+            if (same == active) {
+                if (lane == __ffs(active) - 1) atomicAdd(&hist[lead_bin], (uint32_t)__popc(active));
+            } else if (in) {
+                atomicAdd(&hist[bin], 1u);
+            }
         }
-        __syncthreads();
+        cluster.sync();   // every CTA's histogram of this pass is complete
         if (tid < 256) {
-            uint32_t s = 0;
-            for (int w = 0; w < kSelWarps; ++w) s += hist[w * 256 + tid];
-            total[tid] = s;
+            uint32_t sum = 0;
+#pragma unroll
+            for (int r = 0; r < kSelCluster; ++r) sum += cluster.map_shared_rank(hist, r)[tid];
+            sh->total[tid] = sum;
+            sh->hist[(pass + 1) & 1][tid] = 0u;   // peers finished reading this buffer two syncs ago
         }
         __syncthreads();
         if (warp == 0) {
             // lane l owns bins [8*(31-l), 8*(31-l)+7]; lane 0 holds the highest bins
             const int base = 8 * (31 - lane);
-            uint32_t s = 0;
-            for (int b = 0; b < 8; ++b) s += total[base + b];
-            uint32_t incl = s;
+            uint32_t sgrp = 0;
+            for (int b = 0; b < 8; ++b) sgrp += sh->total[base + b];
+            uint32_t incl = sgrp;
             for (int o = 1; o < 32; o <<= 1) {
                 uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
                 if (lane >= o) incl += t;
             }
-            const uint32_t above = incl - s;
-            const uint32_t k_rem = sh[1];
+            const uint32_t above = incl - sgrp;
+            const uint32_t k_rem = sh->pick[1];
             if (k_rem > above && k_rem <= incl) {
                 uint32_t a = above;
                 for (int b = 7; b >= 0; --b) {
-                    const uint32_t c = total[base + b];
+                    const uint32_t c = sh->total[base + b];
                     if (k_rem <= a + c) {
-                        sh[0] = prefix | ((uint32_t)(base + b) << shift);
-                        sh[1] = k_rem - a;
+                        sh->pick[0] = prefix | ((uint32_t)(base + b) << shift);
+                        sh->pick[1] = k_rem - a;
                         break;
                     }
                     a += c;
@@ -99,15 +127,15 @@ select_topk_kernel(const float* __restrict__ scores, int n_sig, int L_d, int k,
             }
         }
         __syncthreads();
-        prefix = sh[0];
+        prefix = sh->pick[0];
         mask |= 0xFFu << shift;
     }
-    const uint32_t thr = prefix;       // key of the k-th largest score
-    const uint32_t need_eq = sh[1];    // how many keys equal to thr are taken (lowest positions first)
+    const uint32_t thr = prefix;           // key of the k-th largest score
+    const uint32_t need_eq = sh->pick[1];  // how many keys equal to thr are taken (lowest positions first)
 
-    // ordered compaction: thread t owns the contiguous positions [t*E, (t+1)*E)
-    const int E = (L_d + kSelThreads - 1) / kSelThreads;
-    const int lo = min(L_d, tid * E), hi = min(L_d, lo + E);
+    // ordered compaction: thread t owns the contiguous local positions [t*E, (t+1)*E)
+    const int E = (per_cta + kSelThreads - 1) / kSelThreads;
+    const int lo = min(n_loc, tid * E), hi = min(n_loc, lo + E);
     uint32_t n_gt = 0, n_eq = 0;
     for (int i = lo; i < hi; ++i) {
         const uint32_t key = keys[i];
@@ -119,30 +147,36 @@ select_topk_kernel(const float* __restrict__ scores, int n_sig, int L_d, int k,
         uint32_t a = __shfl_up_sync(0xFFFFFFFFu, in_gt, o), b = __shfl_up_sync(0xFFFFFFFFu, in_eq, o);
         if (lane >= o) { in_gt += a; in_eq += b; }
     }
-    if (lane == 31) { scan_gt[warp] = in_gt; scan_eq[warp] = in_eq; }
+    if (lane == 31) { sh->scan_gt[warp] = in_gt; sh->scan_eq[warp] = in_eq; }
     __syncthreads();
     if (warp == 0) {
-        uint32_t a = scan_gt[lane], b = scan_eq[lane];
+        uint32_t a = lane < kSelWarps ? sh->scan_gt[lane] : 0u, b = lane < kSelWarps ? sh->scan_eq[lane] : 0u;
         uint32_t ia = a, ib = b;
         for (int o = 1; o < 32; o <<= 1) {
             uint32_t x = __shfl_up_sync(0xFFFFFFFFu, ia, o), y = __shfl_up_sync(0xFFFFFFFFu, ib, o);
             if (lane >= o) { ia += x; ib += y; }
         }
-        scan_gt[lane] = ia - a;
-        scan_eq[lane] = ib - b;
+        if (lane < kSelWarps) { sh->scan_gt[lane] = ia - a; sh->scan_eq[lane] = ib - b; }
+        if (lane == kSelWarps - 1) { sh->cta_counts[0] = ia; sh->cta_counts[1] = ib; }
     }
-    __syncthreads();
-    uint32_t gt_before = scan_gt[warp] + in_gt - n_gt;
-    uint32_t eq_before = scan_eq[warp] + in_eq - n_eq;
+    cluster.sync();   // every CTA's counts are visible
+    uint32_t gt_before = sh->scan_gt[warp] + in_gt - n_gt;
+    uint32_t eq_before = sh->scan_eq[warp] + in_eq - n_eq;
+    for (int r = 0; r < rank; ++r) {
+        const uint32_t* c = cluster.map_shared_rank(sh->cta_counts, r);
+        gt_before += c[0];
+        eq_before += c[1];
+    }
     if (k > 0) {
         uint32_t pos = gt_before + min(eq_before, need_eq);
         for (int i = lo; i < hi; ++i) {
             const uint32_t key = keys[i];
             bool take = key > thr;
             if (key == thr) { take = eq_before < need_eq; ++eq_before; }
-            if (take) idx_out[pos++] = i;
+            if (take) idx_out[pos++] = lo_cta + i;
         }
     }
+    cluster.sync();   // no CTA may retire while a peer can still read its shared memory
 }
 
 // --------------------------------------------------- gather + hybrid KV update
@@ -223,12 +257,13 @@ fuse_rows_kernel(const FuseArgs a) {
 
 // ----------------------------------------------------------------- host side
 size_t select_scratch_bytes(int L_d) {
-    return L_d > kSelSmemKeys ? ((size_t)L_d * sizeof(uint32_t) + 255) / 256 * 256 : 0;
+    const int per_cta = (L_d + kSelCluster - 1) / kSelCluster;
+    return per_cta > kSelSmemKeysPerCta ? ((size_t)per_cta * kSelCluster * sizeof(uint32_t) + 255) / 256 * 256 : 0;
 }
 
 static size_t select_smem_bytes(int L_d) {
-    size_t fixed = (size_t)(kSelWarps * 256 + 256 + 2 * kSelWarps + 4) * sizeof(uint32_t);
-    return fixed + (L_d <= kSelSmemKeys ? (size_t)L_d * sizeof(uint32_t) : 0);
+    const int per_cta = (L_d + kSelCluster - 1) / kSelCluster;
+    return sizeof(SelShared) + (per_cta <= kSelSmemKeysPerCta ? (size_t)per_cta * sizeof(uint32_t) : 0);
 }
 
 int launch_select(const ResolvedParams& rp, const float* scores, int n_sig, const int32_t* idx_in,
@@ -237,15 +272,17 @@ int launch_select(const ResolvedParams& rp, const float* scores, int n_sig, cons
                   DeviceStatus* status, void* scratch, cudaStream_t stream) {
     const int32_t* idx_src = idx_in;
     if (scores != nullptr && rp.L_d > 0) {
-        static bool attr_set = false;
+        static bool attr_done[64] = {false};
         const size_t smem = select_smem_bytes(rp.L_d);
-        if (!attr_set) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        if (dev >= 0 && dev < 64 && !attr_done[dev]) {
             cudaError_t e = cudaFuncSetAttribute(select_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                 (int)select_smem_bytes(kSelSmemKeys));
+                                                 (int)(sizeof(SelShared) + (size_t)kSelSmemKeysPerCta * sizeof(uint32_t)));
             if (e != cudaSuccess) { set_cuda_error(e); return DAF_ERR_CUDA; }
-            attr_set = true;
+            attr_done[dev] = true;
         }
-        select_topk_kernel<<<1, kSelThreads, smem, stream>>>(scores, n_sig, rp.L_d, rp.k,
+        select_topk_kernel<<<kSelCluster, kSelThreads, smem, stream>>>(scores, n_sig, rp.L_d, rp.k,
                                                             reinterpret_cast<uint32_t*>(scratch), idx_out);
         count_launch();
         if (int rc = check_launch()) return rc;
