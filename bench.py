@@ -203,18 +203,42 @@ def run_ours(args, w: W.Workload):
     # every rank owns its own replica of the workload (distinct seeds per rank): weak scaling, no exchange
     bufs = [LayerBuffers(w, rank * w.layers + i, api, dev) for i in range(w.layers)]
     torch.cuda.synchronize()
-    stream = torch.cuda.current_stream()
+    Hq = w.n_q_heads
+    row_bytes = Hq * 256
 
+    # All launches below go to torch's current stream (the capture stream while a graph is recorded).
     def layer_call(b: LayerBuffers):
         L = b.L
-        st = api.daf_layer(p, L["scores"], b.n_sig, L["idx_in"], L["q_fresh"], L["k_fresh"], L["v_fresh"], b.kv_k,
-                           b.kv_v, b.idx_out, b.q_pack, b.k_pack, b.v_pack, b.hidden, None, ws, stream)
-        if st != 0:
-            api.check(st, "daf_layer")
+        api.check(api.daf_layer(p, L["scores"], b.n_sig, L["idx_in"], L["q_fresh"], L["k_fresh"], L["v_fresh"], b.kv_k,
+                                b.kv_v, b.idx_out, b.q_pack, b.k_pack, b.v_pack, b.hidden, None, ws), "daf_layer")
 
-    def step():
-        for b in bufs:
-            layer_call(b)
+    def st_select(b):
+        L = b.L
+        api.check(api.daf_select(p, L["scores"], b.n_sig, L["idx_in"], L["q_fresh"], L["k_fresh"], L["v_fresh"],
+                                 b.kv_k, b.kv_v, b.idx_out, b.q_pack, b.k_pack, b.v_pack, ws), "daf_select")
+
+    def st_imp(b):
+        api.check(api.daf_important_attn(p, b.k, b.q_pack, b.k_pack, b.v_pack, b.hidden, row_bytes, None, None, ws),
+                  "daf_important_attn")
+
+    def st_qd(b):
+        api.check(api.daf_qd_attn(p, b.L["q_fresh"][w.L_d:], b.kv_k, b.kv_v, b.hidden, row_bytes, None, None, ws,
+                                  out_offset_bytes=b.k * row_bytes), "daf_qd_attn")
+
+    n_full = min(len(bufs), 4)
+    pf = api.make_params(w.N, 0, 1.0, w.n_q_heads, w.n_kv_heads)
+    wsf = api.alloc_workspace(pf, dev)
+    full_out = torch.empty(w.N, Hq, 128, dtype=torch.bfloat16, device=dev)
+
+    def st_full(b):
+        api.check(api.daf_full_causal_attn(pf, w.N, b.L["q_fresh"], b.L["k_fresh"], b.L["v_fresh"], full_out, None,
+                                           wsf), "daf_full_causal_attn")
+
+    def over(fn, items):
+        def run():
+            for b in items:
+                fn(b)
+        return run
 
     def barrier():
         torch.cuda.synchronize()
@@ -222,22 +246,52 @@ def run_ours(args, w: W.Workload):
             dist.barrier()
             torch.cuda.synchronize()
 
-    for _ in range(max(args.warmup, 3)):
+    def capture(run):
+        """Records `run` (one pass over the layers) into a CUDA graph: a replay issues the same kernels
+        with the same arguments without host-side launch cost between them."""
+        launches_before = api.daf_launch_count()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            run()
+        return g, api.daf_launch_count() - launches_before
+
+    def time_replays(g, reps):
+        stream = torch.cuda.current_stream()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(reps):
+            g.replay()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps  # ms per replay
+
+    step = over(layer_call, bufs)
+    for _ in range(max(args.warmup, 3)):     # eager warm-up: also sets function attributes before capture
         step()
     barrier()
     api.check(api.daf_poll_status(ws), "warm-up (device status)")
 
+    use_graph = not args.no_graph
+    if use_graph:
+        g_step, launches_per_step = capture(step)
+        g_step.replay()
+        barrier()
+
+    stream = torch.cuda.current_stream()
     launches0 = api.daf_launch_count()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     with ClockSampler(local_rank) as clocks:
         barrier()
         e0.record(stream)
         for _ in range(args.steps):
-            step()
+            if use_graph:
+                g_step.replay()
+            else:
+                step()
         e1.record(stream)
         barrier()
     ms_total = e0.elapsed_time(e1)
-    launches = api.daf_launch_count() - launches0
+    launches = launches_per_step * args.steps if use_graph else api.daf_launch_count() - launches0
     api.check(api.daf_poll_status(ws), "timed region (device status)")
     if dist is not None:
         t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
@@ -250,55 +304,32 @@ def run_ours(args, w: W.Workload):
     daf_flops = flops["important"] + flops["question"]
     tflops = daf_flops * w.layers * world / (ms_per_step * 1e-3) / 1e12
 
-    # ---- per-stage timings (one launch group at a time, events on the launching stream)
-    def time_stage(fn, reps=3):
-        times = []
-        for _ in range(reps):
-            for b in bufs:
-                a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record(stream)
-                fn(b)
-                z.record(stream)
-                times.append((a, z))
+    # ---- per-stage timings: each stage's launches over all layers, replayed back to back (us per layer)
+    def time_stage(fn, items, reps=5):
+        run = over(fn, items)
+        run()
         torch.cuda.synchronize()
-        return statistics.mean(x.elapsed_time(y) for x, y in times) * 1e3  # us
+        if use_graph:
+            g, _ = capture(run)
+            g.replay()
+            torch.cuda.synchronize()
+            return time_replays(g, reps) * 1e3 / len(items)
+        stream2 = torch.cuda.current_stream()
+        a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream2)
+        for _ in range(reps):
+            run()
+        z.record(stream2)
+        torch.cuda.synchronize()
+        return a.elapsed_time(z) / reps * 1e3 / len(items)
 
-    Hq = w.n_q_heads
-    row_bytes = Hq * 256
-
-    def st_select(b):
-        L = b.L
-        api.check(api.daf_select(p, L["scores"], b.n_sig, L["idx_in"], L["q_fresh"], L["k_fresh"], L["v_fresh"],
-                                 b.kv_k, b.kv_v, b.idx_out, b.q_pack, b.k_pack, b.v_pack, ws, stream), "daf_select")
-
-    def st_imp(b):
-        api.check(api.daf_important_attn(p, b.k, b.q_pack, b.k_pack, b.v_pack, b.hidden, row_bytes, None, None, ws,
-                                         stream), "daf_important_attn")
-
-    def st_qd(b):
-        api.check(api.daf_qd_attn(p, b.L["q_fresh"][w.L_d:], b.kv_k, b.kv_v, b.hidden, row_bytes, None, None, ws,
-                                  stream, out_offset_bytes=b.k * row_bytes), "daf_qd_attn")
-
-    us_select = time_stage(st_select)
-    us_imp = time_stage(st_imp) if w.k > 0 else 0.0
-    us_qd = time_stage(st_qd) if w.L_q > 0 else 0.0
-
-    # ---- full recompute on the same kernels (comparison path), bounded number of layers
-    n_full = min(len(bufs), 4)
-    pf = api.make_params(w.N, 0, 1.0, w.n_q_heads, w.n_kv_heads)
-    wsf = api.alloc_workspace(pf, dev)
-    full_out = torch.empty(w.N, Hq, 128, dtype=torch.bfloat16, device=dev)
-
-    def st_full(b):
-        api.check(api.daf_full_causal_attn(pf, w.N, b.L["q_fresh"], b.L["k_fresh"], b.L["v_fresh"], full_out, None,
-                                           wsf, stream), "daf_full_causal_attn")
-
-    saved = bufs
-    bufs = bufs[:n_full]
-    time_stage(st_full, reps=1)
-    us_full = time_stage(st_full, reps=3)
-    bufs = saved
+    us_select = time_stage(st_select, bufs)
+    us_imp = time_stage(st_imp, bufs) if w.k > 0 else 0.0
+    us_qd = time_stage(st_qd, bufs) if w.L_q > 0 else 0.0
+    # full recompute on the same kernel (comparison path), bounded number of layers
+    us_full = time_stage(st_full, bufs[:n_full], reps=3)
     api.check(api.daf_poll_status(wsf), "full recompute (device status)")
+    api.check(api.daf_poll_status(ws), "stage timing (device status)")
 
     imp_tflops = flops["important"] / (us_imp * 1e-6) / 1e12 if us_imp else 0.0
     qd_tflops = flops["question"] / (us_qd * 1e-6) / 1e12 if us_qd else 0.0
@@ -338,7 +369,7 @@ def run_ours(args, w: W.Workload):
         def e2e_step():
             for h in host:
                 api.check(api.daf_layer_host(p, h["scores"], h["n_sig"], h["idx_in"], h["q_fresh"], h["k_fresh"],
-                                             h["v_fresh"], h["kv_k"], h["kv_v"], 0, h["hidden"], None, arena, stream),
+                                             h["v_fresh"], h["kv_k"], h["kv_v"], 0, h["hidden"], None, arena),
                           "daf_layer_host")
 
         e2e_steps = max(1, min(args.steps, 5))
@@ -395,6 +426,7 @@ def run_ours(args, w: W.Workload):
             "full_recompute": {"us_per_layer": us_full, "tflops": full_tflops, "frac": full_tflops / peaks["bf16_tflops"],
                                "speedup_daf_vs_full": us_full / us_per_layer / world if world == 1 else None,
                                "flop_ratio": flops["full"] / daf_flops, "layers_timed": n_full},
+            "launch_mode": "cuda_graph_replay" if use_graph else "eager",
             "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks.summary(),
             "peaks": peaks, "cpu_baseline": cpu_baseline,
         }
@@ -412,6 +444,7 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--config", default="c1", help="c0..c3 or a sweep point name (c4_L<L_d>_r<r>)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying a CUDA graph")
     args = ap.parse_args()
     if args.config in W.CONFIGS:
         w = W.CONFIGS[args.config]

@@ -22,32 +22,46 @@
 
 namespace daf {
 
-constexpr int kNQ = 2;                  // query tiles per CTA
 constexpr int kBlockM = 128;            // rows per query tile
 constexpr int kBlockN = 128;            // keys per KV tile
 constexpr int kD = 128;                 // head_dim
-constexpr int kStages = 4;              // KV ring slots (K and V tiles alternate through it)
 constexpr int kTileBytes = kBlockN * kD * 2;      // 32 KB: one Q, K or V tile
 constexpr int kHalfBytes = kTileBytes / 2;        // one 64-column half (128-byte rows)
-constexpr int kSoftmaxWarps = 4 * kNQ;
-constexpr int kTmaWarp = kSoftmaxWarps;
-constexpr int kMmaWarp = kSoftmaxWarps + 1;
-constexpr int kAttnThreads = 32 * (kSoftmaxWarps + 2);
-constexpr int kTmemCols = 512;          // S0 S1 O0 O1, 128 fp32 columns each
 constexpr int kMaxSplits = 32;
+constexpr int kNumSMs = 148;
 constexpr float kRescaleThreshold = 8.0f;   // in log2 units: keep a stale row maximum up to 2^8
 
+// Two shapes of the same kernel:
+//   NQ = 2: two query tiles per CTA share every K/V tile (half the shared-memory fill traffic), one CTA
+//           per SM with all 512 tensor-memory columns and a 4-slot ring: for large problems;
+//   NQ = 1: one query tile per CTA, 256 tensor-memory columns and a 2-slot ring, so that two CTAs live on
+//           an SM and cover each other's softmax, prologue and output stores: for problems with few tiles.
+template <int NQ>
+struct AttnCfg {
+    static constexpr int kStages = NQ == 2 ? 4 : 2;        // KV ring slots (K and V tiles alternate through it)
+    static constexpr int kSoftmaxWarps = 4 * NQ;
+    static constexpr int kTmaWarp = kSoftmaxWarps;
+    static constexpr int kMmaWarp = kSoftmaxWarps + 1;
+    static constexpr int kThreads = 32 * (kSoftmaxWarps + 2);
+    static constexpr int kTmemCols = 256 * NQ;             // per tile: S (128 fp32 columns) and O (128)
+    static constexpr int kCtasPerSM = NQ == 2 ? 1 : 2;
+};
+
+template <int NQ>
 struct AttnSmem {
-    uint64_t q_full[kNQ];
-    uint64_t kv_full[kStages];
-    uint64_t kv_empty[kStages];
-    uint64_t s_full[kNQ];
-    uint64_t p_full[kNQ];
-    uint64_t o_done[kNQ];
+    uint64_t q_full[NQ];
+    uint64_t kv_full[AttnCfg<NQ>::kStages];
+    uint64_t kv_empty[AttnCfg<NQ>::kStages];
+    uint64_t s_full[NQ];
+    uint64_t p_full[NQ];
+    uint64_t o_done[NQ];
     uint32_t tmem_base;
     int abort_flag;
 };
-constexpr size_t kAttnSmemBytes = 1024 /*alignment slack*/ + (size_t)(kNQ + kStages) * kTileBytes + sizeof(AttnSmem);
+template <int NQ>
+constexpr size_t attn_smem_bytes() {
+    return 1024 /*alignment slack*/ + (size_t)(NQ + AttnCfg<NQ>::kStages) * kTileBytes + sizeof(AttnSmem<NQ>);
+}
 
 struct AttnArgs {
     int n_q;            // query tokens
@@ -69,14 +83,32 @@ struct AttnArgs {
     DeviceStatus* status;
 };
 
-__global__ void __launch_bounds__(kAttnThreads, 1)
+#ifdef DAF_TRACE
+// Debug build only (-DDAF_TRACE): per-CTA time stamps for latency studies.
+__device__ unsigned long long g_trace[8 * 65536];
+#define DAF_STAMP(slot)                                                                         \
+    do {                                                                                        \
+        const unsigned cta_ = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);   \
+        if (cta_ < 65536u) g_trace[8 * cta_ + (slot)] = global_ns();                            \
+    } while (0)
+#else
+#define DAF_STAMP(slot) do {} while (0)
+#endif
+
+template <int NQ>
+__global__ void __launch_bounds__(AttnCfg<NQ>::kThreads, AttnCfg<NQ>::kCtasPerSM)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                 const __grid_constant__ CUtensorMap tmap_v, const AttnArgs a) {
+    constexpr int kNQ = NQ;
+    constexpr int kStages = AttnCfg<NQ>::kStages;
+    constexpr int kTmaWarp = AttnCfg<NQ>::kTmaWarp;
+    constexpr int kMmaWarp = AttnCfg<NQ>::kMmaWarp;
+    constexpr int kTmemCols = AttnCfg<NQ>::kTmemCols;
     extern __shared__ unsigned char attn_smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(attn_smem_raw) + 1023) & ~(uintptr_t)1023);
     unsigned char* q_smem = smem;                                   // kNQ tiles
     unsigned char* kv_smem = smem + (size_t)kNQ * kTileBytes;       // kStages tiles
-    AttnSmem* sm = reinterpret_cast<AttnSmem*>(kv_smem + (size_t)kStages * kTileBytes);
+    AttnSmem<NQ>* sm = reinterpret_cast<AttnSmem<NQ>*>(kv_smem + (size_t)kStages * kTileBytes);
 
     // a CTA of this grid (or an earlier kernel sharing the workspace) has already given up: do nothing
     __shared__ int skip_cta;
@@ -84,6 +116,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     __syncthreads();
     if (skip_cta) return;
 
+    if (threadIdx.x == 0) DAF_STAMP(0);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // blocks are dispatched x-fastest: all head blocks of the heaviest (last) query-tile pair go first
     const int pair = (int)gridDim.y - 1 - (int)blockIdx.y;
@@ -130,6 +163,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     tc_fence_after();
     const uint32_t tmem = sm->tmem_base;
     volatile int* abort_flag = &sm->abort_flag;
+    if (threadIdx.x == 0) DAF_STAMP(1);
 
     if (warp == kTmaWarp) {
         // ------------------------------------------------------------ TMA producer
@@ -221,6 +255,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                     tc_fence_after();
                     issue_pv(q, slot_of(seq_v), j == 0);
                     if (j + 1 < n_j[q]) { issue_qk(q, slot_of(seq_k)); tc_commit(&sm->s_full[q]); }
+                    else if (more) tc_commit(&sm->o_done[q]);   // this tile is done early: release its epilogue now
                     else last_tile[q] = true;
                 }
                 if (!ok) break;
@@ -239,8 +274,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         const int r = quad * 32 + lane;
         const int tok = t0[q] + r / a.Gp;
         const int head = h0 + r % a.Gp;
-        const bool row_valid = (r < a.Gp * a.Tt) && (tok < a.n_q) && (n_j[q] > 0 || a.n_splits > 1) &&
-                               (pair * kNQ + q < a.n_tb);
+        const bool row_valid_tile = (n_j[q] > 0 || a.n_splits > 1) && (pair * kNQ + q < a.n_tb);
+        const bool row_valid = (r < a.Gp * a.Tt) && (tok < a.n_q) && row_valid_tile;
         const long long lim_ll = (long long)tok + a.causal_off;
         const int limit = row_valid ? (int)min(lim_ll, (long long)a.n_kv - 1) : -1;   // last visible key
         const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
@@ -255,6 +290,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) break;
             tc_fence_after();
+            if (threadIdx.x == 0 && j == 0) DAF_STAMP(2);
             // logits of this row: 128 fp32 values, fetched in two halves so that the row maximum of the
             // first half is computed while the second half is still on its way from tensor memory
             uint32_t sr[4][32];
@@ -331,6 +367,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             tc_fence_before();
             mbar_arrive(&sm->p_full[q]);
         }
+        if (threadIdx.x == 0) DAF_STAMP(3);
         // ---- epilogue
         if (ok && n_j[q] > 0) {
             ok = mbar_wait(&sm->o_done[q], 0, abort_flag, a.status, 60 + q);
@@ -340,64 +377,118 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             tc_fence_after();
             const float inv_l = l > 0.f ? 1.f / l : 0.f;
             const float lse_val = l > 0.f ? m * a.scale + logf(l) : -INFINITY;
+            // Rows leave through shared memory so that global stores are whole 256-byte runs: each
+            // thread parks its own row (16-byte chunks, XOR-swizzled against bank conflicts) in the
+            // part of the Q tile that belongs to its warp (Q is dead once the last MMA has completed),
+            // then the warp writes its 32 rows out, 16 lanes per row.
+            unsigned char* stage = q_smem + (size_t)q * kTileBytes + (size_t)quad * 32 * 256;
+            auto park = [&](int chunk, uint4 w) {
+                *reinterpret_cast<uint4*>(stage + lane * 256 + ((chunk ^ (lane & 7)) << 4)) = w;
+            };
+            // copy phase: lanes 0-15 take row rr, lanes 16-31 row rr+1, rr advancing by 2; the row's
+            // (token, head) pair is tracked incrementally instead of dividing in the loop
+            const int sub = lane >> 4, cidx = lane & 15;
+            const int r_first = quad * 32 + sub;
+            const int step_t = 2 / a.Gp, step_h = 2 % a.Gp;
+            const int n_rows_tile = a.Gp * a.Tt;
             if (a.n_splits == 1) {
-                __nv_bfloat16* dst = nullptr;
-                if (row_valid) {
-                    const long long drow = a.dst_rows ? (long long)a.dst_rows[tok] : (long long)tok;
-                    dst = a.out + drow * a.out_row_stride + (long long)head * kD;
-                    if (a.lse != nullptr) a.lse[(size_t)head * a.n_q + tok] = lse_val;
-                }
+                if (row_valid && a.lse != nullptr) a.lse[(size_t)head * a.n_q + tok] = lse_val;
                 if (n_j[q] > 0) {
 #pragma unroll
                     for (int cchunk = 0; cchunk < 4; ++cchunk) {
                         uint32_t orr[32];
                         tmem_ld32(o_addr + (uint32_t)(cchunk * 32), orr);
                         tc_wait_ld();
-                        if (row_valid) {
-                            uint4* d4 = reinterpret_cast<uint4*>(dst + cchunk * 32);
 #pragma unroll
-                            for (int v = 0; v < 4; ++v) {
-                                uint4 w;
-                                w.x = pack_bf16(__uint_as_float(orr[v * 8 + 0]) * inv_l, __uint_as_float(orr[v * 8 + 1]) * inv_l);
-                                w.y = pack_bf16(__uint_as_float(orr[v * 8 + 2]) * inv_l, __uint_as_float(orr[v * 8 + 3]) * inv_l);
-                                w.z = pack_bf16(__uint_as_float(orr[v * 8 + 4]) * inv_l, __uint_as_float(orr[v * 8 + 5]) * inv_l);
-                                w.w = pack_bf16(__uint_as_float(orr[v * 8 + 6]) * inv_l, __uint_as_float(orr[v * 8 + 7]) * inv_l);
-                                d4[v] = w;
-                            }
+                        for (int v = 0; v < 4; ++v) {
+                            uint4 w;
+                            w.x = pack_bf16(__uint_as_float(orr[v * 8 + 0]) * inv_l, __uint_as_float(orr[v * 8 + 1]) * inv_l);
+                            w.y = pack_bf16(__uint_as_float(orr[v * 8 + 2]) * inv_l, __uint_as_float(orr[v * 8 + 3]) * inv_l);
+                            w.z = pack_bf16(__uint_as_float(orr[v * 8 + 4]) * inv_l, __uint_as_float(orr[v * 8 + 5]) * inv_l);
+                            w.w = pack_bf16(__uint_as_float(orr[v * 8 + 6]) * inv_l, __uint_as_float(orr[v * 8 + 7]) * inv_l);
+                            park(cchunk * 4 + v, w);
                         }
+                    }
+                    __syncwarp();
+                    int tok_r = t0[q] + r_first / a.Gp, head_off = r_first % a.Gp;
+#pragma unroll 4
+                    for (int i = 0; i < 16; ++i) {
+                        const int rr = 2 * i + sub;
+                        if (quad * 32 + rr < n_rows_tile && tok_r < a.n_q) {
+                            const long long drow = a.dst_rows ? (long long)a.dst_rows[tok_r] : (long long)tok_r;
+                            const uint4 w = *reinterpret_cast<const uint4*>(stage + rr * 256 + ((cidx ^ (rr & 7)) << 4));
+                            reinterpret_cast<uint4*>(a.out + drow * a.out_row_stride + (long long)(h0 + head_off) * kD)[cidx] = w;
+                        }
+                        head_off += step_h; tok_r += step_t;
+                        if (head_off >= a.Gp) { head_off -= a.Gp; ++tok_r; }
                     }
                 }
             } else {
-                const size_t prow = ((size_t)split * a.n_q + (size_t)max(tok, 0)) * a.Hq + head;
-                if (row_valid) a.part_lse[prow] = lse_val;
-                float4* d4 = reinterpret_cast<float4*>(a.part_o + prow * kD);
-                if (n_j[q] > 0) {
+                const size_t prow0 = (size_t)split * a.n_q;
+                if (row_valid) a.part_lse[(prow0 + (size_t)tok) * a.Hq + head] = lse_val;
 #pragma unroll
-                    for (int cchunk = 0; cchunk < 4; ++cchunk) {
-                        uint32_t orr[32];
-                        tmem_ld32(o_addr + (uint32_t)(cchunk * 32), orr);
-                        tc_wait_ld();
-                        if (row_valid) {
+                for (int half = 0; half < 2; ++half) {   // 64 fp32 columns (256 bytes per row) at a time
+                    if (n_j[q] > 0) {
 #pragma unroll
-                            for (int v = 0; v < 8; ++v)
-                                d4[cchunk * 8 + v] = make_float4(__uint_as_float(orr[v * 4 + 0]) * inv_l, __uint_as_float(orr[v * 4 + 1]) * inv_l,
-                                                                 __uint_as_float(orr[v * 4 + 2]) * inv_l, __uint_as_float(orr[v * 4 + 3]) * inv_l);
+                        for (int cc = 0; cc < 2; ++cc) {
+                            uint32_t orr[32];
+                            tmem_ld32(o_addr + (uint32_t)((half * 2 + cc) * 32), orr);
+                            tc_wait_ld();
+#pragma unroll
+                            for (int v = 0; v < 8; ++v) {
+                                uint4 w;
+                                w.x = __float_as_uint(__uint_as_float(orr[v * 4 + 0]) * inv_l);
+                                w.y = __float_as_uint(__uint_as_float(orr[v * 4 + 1]) * inv_l);
+                                w.z = __float_as_uint(__uint_as_float(orr[v * 4 + 2]) * inv_l);
+                                w.w = __float_as_uint(__uint_as_float(orr[v * 4 + 3]) * inv_l);
+                                park(cc * 8 + v, w);
+                            }
                         }
+                    } else {
+#pragma unroll
+                        for (int v = 0; v < 16; ++v) park(v, make_uint4(0u, 0u, 0u, 0u));
                     }
-                } else if (row_valid) {
-                    for (int v = 0; v < 32; ++v) d4[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    __syncwarp();
+                    int tok_r = t0[q] + r_first / a.Gp, head_off = r_first % a.Gp;
+#pragma unroll 4
+                    for (int i = 0; i < 16; ++i) {
+                        const int rr = 2 * i + sub;
+                        if (row_valid_tile && quad * 32 + rr < n_rows_tile && tok_r < a.n_q) {
+                            const uint4 w = *reinterpret_cast<const uint4*>(stage + rr * 256 + ((cidx ^ (rr & 7)) << 4));
+                            float* prow = a.part_o + ((prow0 + (size_t)tok_r) * a.Hq + (h0 + head_off)) * kD + half * 64;
+                            reinterpret_cast<uint4*>(prow)[cidx] = w;
+                        }
+                        head_off += step_h; tok_r += step_t;
+                        if (head_off >= a.Gp) { head_off -= a.Gp; ++tok_r; }
+                    }
+                    __syncwarp();
                 }
             }
         }
     }
 
+    if (threadIdx.x == 0) DAF_STAMP(4);
     tc_fence_before();
     __syncthreads();
     if (warp == kMmaWarp) {
         tc_fence_after();
         tmem_dealloc(tmem, kTmemCols);
     }
+#ifdef DAF_TRACE
+    if (threadIdx.x == 0) {
+        DAF_STAMP(5);
+        const unsigned cta = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
+        if (cta < 65536u) g_trace[8 * cta + 6] = (unsigned long long)n_j_max;
+    }
+#endif
 }
+
+#ifdef DAF_TRACE
+extern "C" void daf_dbg_force_nq(int nq);
+extern "C" int daf_dbg_read_trace(void* host, size_t bytes) {
+    return (int)cudaMemcpyFromSymbol(host, g_trace, bytes < sizeof(g_trace) ? bytes : sizeof(g_trace));
+}
+#endif
 
 // Merge of split-KV partials: one warp per (token, head) row.
 __global__ void __launch_bounds__(256)
@@ -483,14 +574,20 @@ static int make_tmap(CUtensorMap* m, const void* base, int tokens, int heads, in
 
 // How a problem is cut into CTAs.  Splitting the KV axis is only used for the
 // question rows, where there are few query tiles and a long KV axis.
+static int g_force_nq = 0;   // 0: choose by problem size (the tuning builds can pin a shape)
+
 AttnPlan plan_attention(int n_q, int n_kv, int Hq, int G, int causal_off, bool pack_group, bool allow_split) {
     AttnPlan pl;
     pl.Gp = pack_group ? G : 1;
     if (pl.Gp > 128) pl.Gp = 1;
     pl.Tt = kBlockM / pl.Gp;
     pl.n_tb = (n_q + pl.Tt - 1) / pl.Tt;
-    pl.pairs = (pl.n_tb + kNQ - 1) / kNQ;
     pl.head_blocks = Hq / pl.Gp;
+    // two tiles per CTA once that alone fills every SM twice over; otherwise one tile per CTA, two CTAs per SM
+    const int ctas_two = ((pl.n_tb + 1) / 2) * pl.head_blocks;
+    pl.nq = ctas_two >= 2 * kNumSMs ? 2 : 1;
+    if (g_force_nq == 1 || g_force_nq == 2) pl.nq = g_force_nq;
+    pl.pairs = (pl.n_tb + pl.nq - 1) / pl.nq;
     long long kv_hi = (long long)n_q - 1 + causal_off + 1;
     if (kv_hi > n_kv) kv_hi = n_kv;
     const int total_tiles = kv_hi > 0 ? (int)((kv_hi + kBlockN - 1) / kBlockN) : 0;
@@ -498,7 +595,8 @@ AttnPlan plan_attention(int n_q, int n_kv, int Hq, int G, int causal_off, bool p
     pl.tiles_per_split = total_tiles > 0 ? total_tiles : 1;
     if (allow_split && total_tiles > 1) {
         const int ctas = pl.pairs * pl.head_blocks;
-        int want = ctas > 0 ? 148 / ctas : 1;
+        const int slots = kNumSMs * (pl.nq == 2 ? 1 : 2);
+        int want = ctas > 0 ? slots / ctas : 1;
         if (want > kMaxSplits) want = kMaxSplits;
         if (want > total_tiles) want = total_tiles;
         if (want > 1) {
@@ -508,6 +606,10 @@ AttnPlan plan_attention(int n_q, int n_kv, int Hq, int G, int causal_off, bool p
     }
     return pl;
 }
+
+#ifdef DAF_TRACE
+extern "C" void daf_dbg_force_nq(int nq) { g_force_nq = nq; }
+#endif
 
 size_t attn_partial_bytes(int n_q, int Hq, int n_splits) {
     if (n_splits <= 1) return 0;
@@ -535,7 +637,9 @@ int launch_attention(const void* q, const void* k, const void* v, int n_q, int n
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !attr_done[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(attn_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttnSmemBytes);
+        cudaError_t e = cudaFuncSetAttribute(attn_fwd_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem_bytes<1>());
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(attn_fwd_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem_bytes<2>());
         if (e != cudaSuccess) { set_cuda_error(e); return DAF_ERR_CUDA; }
         attr_done[dev] = true;
     }
@@ -556,7 +660,8 @@ int launch_attention(const void* q, const void* k, const void* v, int n_q, int n
                                  : nullptr;
     a.status = status;
     dim3 grid((unsigned)pl.head_blocks, (unsigned)pl.pairs, (unsigned)pl.n_splits);
-    attn_fwd_kernel<<<grid, kAttnThreads, kAttnSmemBytes, stream>>>(tq, tk, tv, a);
+    if (pl.nq == 2) attn_fwd_kernel<2><<<grid, AttnCfg<2>::kThreads, attn_smem_bytes<2>(), stream>>>(tq, tk, tv, a);
+    else attn_fwd_kernel<1><<<grid, AttnCfg<1>::kThreads, attn_smem_bytes<1>(), stream>>>(tq, tk, tv, a);
     count_launch();
     if (int rc = check_launch()) return rc;
     if (pl.n_splits > 1) {
