@@ -108,6 +108,20 @@ def _dist_env():
     return int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
 
 
+def replica_layers(rank: int, w: W.Workload):
+    """Layer seeds of rank `rank`: every rank owns its own replica of the workload (weak scaling, no exchange)."""
+    return [rank * w.layers + i for i in range(w.layers)]
+
+
+def max_over_ranks(dist, value: float, device) -> float:
+    """A duration is reported as the maximum over ranks (single process: the value itself)."""
+    if dist is None:
+        return float(value)
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
 def _config_dict(w: W.Workload, n_gpus: int):
     return {"workload": f"{w.name}: {w.layers} layers, Hq={w.n_q_heads} Hkv={w.n_kv_heads} D={w.head_dim}, "
                         f"L_d={w.L_d} ({w.n_docs} docs of {w.doc_len}), L_q={w.L_q}, r={w.r} (k={w.k}), "
@@ -201,7 +215,7 @@ def run_ours(args, w: W.Workload):
     p = api.make_params(w.L_d, w.L_q, w.r, w.n_q_heads, w.n_kv_heads)
     ws = api.alloc_workspace(p, dev)
     # every rank owns its own replica of the workload (distinct seeds per rank): weak scaling, no exchange
-    bufs = [LayerBuffers(w, rank * w.layers + i, api, dev) for i in range(w.layers)]
+    bufs = [LayerBuffers(w, layer, api, dev) for layer in replica_layers(rank, w)]
     torch.cuda.synchronize()
     Hq = w.n_q_heads
     row_bytes = Hq * 256
@@ -293,10 +307,7 @@ def run_ours(args, w: W.Workload):
     ms_total = e0.elapsed_time(e1)
     launches = launches_per_step * args.steps if use_graph else api.daf_launch_count() - launches0
     api.check(api.daf_poll_status(ws), "timed region (device status)")
-    if dist is not None:
-        t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(dist, ms_total, dev)
     ms_per_step = ms_total / args.steps
     us_per_layer = ms_per_step * 1e3 / (w.layers * world)
 
@@ -380,10 +391,7 @@ def run_ours(args, w: W.Workload):
             e2e_step()
         torch.cuda.synchronize()
         dt = time.perf_counter() - t0
-        if dist is not None:
-            t = torch.tensor([dt], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            dt = float(t.item())
+        dt = max_over_ranks(dist, dt, dev)
         e2e = {"value": dt / e2e_steps / (n_e2e * world) * 1e6, "unit": UNIT,
                "h2d_bytes_per_step": int(per_layer_in * n_e2e), "d2h_bytes_per_step": int((w.k + w.L_q) * row_bytes * n_e2e),
                "layers_per_step": n_e2e, "steps": e2e_steps,

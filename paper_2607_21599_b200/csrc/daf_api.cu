@@ -103,9 +103,34 @@ static int check_out(const void* out, int64_t stride_bytes, int Hq) {
     return DAF_OK;
 }
 
+// A side stream and two events per device, created on first use and kept for the life of the
+// process (host-side state only; no device memory).
+struct SideStream { cudaStream_t stream; cudaEvent_t fork, join; };
+static SideStream* side_stream() {
+    static SideStream table[64];
+    static bool ready[64] = {false};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (!ready[dev]) {
+        SideStream s;
+        if (cudaStreamCreateWithFlags(&s.stream, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+        if (cudaEventCreateWithFlags(&s.fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        if (cudaEventCreateWithFlags(&s.join, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        table[dev] = s;
+        ready[dev] = true;
+    }
+    return &table[dev];
+}
+
 }  // namespace daf
 
 using namespace daf;
+
+#define DAF_CUDA_TRY(expr)                                                \
+    do {                                                                  \
+        cudaError_t e_ = (expr);                                          \
+        if (e_ != cudaSuccess) { set_cuda_error(e_); return DAF_ERR_CUDA; } \
+    } while (0)
 
 extern "C" {
 
@@ -208,19 +233,36 @@ int daf_layer(const daf_params* p, const float* scores, int32_t n_sig, const int
     if (int rc = do_select(rp, scores, n_sig, idx_in, q_fresh, k_fresh, v_fresh, kv_k, kv_v, idx_out, q_pack, k_pack,
                            v_pack, ws, st)) return rc;
     char* h = reinterpret_cast<char*>(hidden);
-    // state fusion is done by the attention epilogues: each stage writes its final rows
-    if (rp.k > 0) {
-        const int32_t* dst = rp.fuse_mode == 1 ? idx_out : nullptr;
-        if (int rc = launch_attention(q_pack, k_pack, v_pack, rp.k, rp.k, rp.Hq, rp.Hkv, 0, rp.scale, false, false, h,
-                                      row_bytes, dst, nullptr, ws.status, ws.attn_scratch, ws.attn_bytes, st)) return rc;
+    // State fusion is done by the attention epilogues: each stage writes its final rows.  The two
+    // stages are independent once step 1 is done, so the question stage runs on a side stream
+    // (forked and joined with events) and the GPU fills one stage's idle SMs with the other's CTAs.
+    const bool both = rp.k > 0 && rp.L_q > 0;
+    SideStream* side = both ? side_stream() : nullptr;
+    cudaStream_t st_q = st;
+    if (side != nullptr) {
+        DAF_CUDA_TRY(cudaEventRecord(side->fork, st));
+        DAF_CUDA_TRY(cudaStreamWaitEvent(side->stream, side->fork, 0));
+        st_q = side->stream;
     }
+    int rc_q = DAF_OK, rc_i = DAF_OK;
     if (rp.L_q > 0) {
         const int64_t first_row = rp.fuse_mode == 1 ? rp.L_d : rp.k;
         const char* qq = reinterpret_cast<const char*>(q_fresh) + (int64_t)rp.L_d * row_bytes;
-        if (int rc = launch_attention(qq, kv_k, kv_v, rp.L_q, rp.N, rp.Hq, rp.Hkv, rp.L_d, rp.scale, true, true,
-                                      h + first_row * row_bytes, row_bytes, nullptr, nullptr, ws.status,
-                                      ws.attn_scratch, ws.attn_bytes, st)) return rc;
+        rc_q = launch_attention(qq, kv_k, kv_v, rp.L_q, rp.N, rp.Hq, rp.Hkv, rp.L_d, rp.scale, true, true,
+                                h + first_row * row_bytes, row_bytes, nullptr, nullptr, ws.status, ws.attn_scratch,
+                                ws.attn_bytes, st_q);
     }
+    if (rp.k > 0) {
+        const int32_t* dst = rp.fuse_mode == 1 ? idx_out : nullptr;
+        rc_i = launch_attention(q_pack, k_pack, v_pack, rp.k, rp.k, rp.Hq, rp.Hkv, 0, rp.scale, false, false, h,
+                                row_bytes, dst, nullptr, ws.status, ws.attn_scratch, ws.attn_bytes, st);
+    }
+    if (side != nullptr) {   // always re-join, also after a failed launch, so that the streams stay consistent
+        DAF_CUDA_TRY(cudaEventRecord(side->join, side->stream));
+        DAF_CUDA_TRY(cudaStreamWaitEvent(st, side->join, 0));
+    }
+    if (rc_q != DAF_OK) return rc_q;
+    if (rc_i != DAF_OK) return rc_i;
     if (row_pos_out != nullptr) {
         if (int rc = launch_fuse(rp, idx_out, nullptr, nullptr, nullptr, row_pos_out, st)) return rc;
     }
@@ -267,11 +309,6 @@ size_t daf_layer_host_arena_bytes(const daf_params* p) {
     return a.total;
 }
 
-#define DAF_CUDA_TRY(expr)                                                \
-    do {                                                                  \
-        cudaError_t e_ = (expr);                                          \
-        if (e_ != cudaSuccess) { set_cuda_error(e_); return DAF_ERR_CUDA; } \
-    } while (0)
 
 int daf_layer_host(const daf_params* p, const float* h_scores, int32_t n_sig, const int32_t* h_idx_in,
                    const void* h_q_fresh, const void* h_k_fresh, const void* h_v_fresh,

@@ -222,13 +222,13 @@ __device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi) {
     return d;
 }
 __device__ __forceinline__ float f32x2_lo(uint64_t v) {
-    float lo, hi;
+    [[maybe_unused]] float lo, hi;
     asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
     (void)hi;
     return lo;
 }
 __device__ __forceinline__ float f32x2_hi(uint64_t v) {
-    float lo, hi;
+    [[maybe_unused]] float lo, hi;
     asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
     (void)lo;
     return hi;
