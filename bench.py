@@ -453,6 +453,7 @@ def main():
     ap.add_argument("--config", default="c1", help="c0..c3 or a sweep point name (c4_L<L_d>_r<r>)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying a CUDA graph")
+    ap.add_argument("--layers", type=int, default=0, help="use only the first LAYERS layers (profiling captures)")
     args = ap.parse_args()
     if args.config in W.CONFIGS:
         w = W.CONFIGS[args.config]
@@ -461,6 +462,9 @@ def main():
         if args.config not in pts:
             raise SystemExit(f"unknown config {args.config}; choose from {list(W.CONFIGS) + list(pts)}")
         w = pts[args.config]
+    if args.layers > 0:
+        import dataclasses
+        w = dataclasses.replace(w, layers=min(args.layers, w.layers))
     if args.impl == "reference":
         run_reference(args, w)
     else:

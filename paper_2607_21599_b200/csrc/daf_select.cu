@@ -179,6 +179,174 @@ select_topk_kernel(const float* __restrict__ scores, int n_sig, int L_d, int k,
     cluster.sync();   // no CTA may retire while a peer can still read its shared memory
 }
 
+// ------------------------------------------------ selection, one CTA (small L_d)
+// Latency matters more than bandwidth here (at most 160 KB of keys), so the common sizes run in
+// one CTA with no cluster traffic.  One pass over all keys histograms their top 12 bits and finds
+// the bin that holds the k-th largest key; only the keys of that bin (typically a few per cent)
+// go on to two 10-bit passes that fix the remaining 20 bits; an ordered compaction then emits the
+// positions.  If the bin holds more keys than the candidate list can take (many equal scores),
+// the two small passes walk all keys with a filter instead.
+constexpr int kSel1Threads = 1024;
+constexpr int kSel1Warps = kSel1Threads / 32;
+constexpr int kSel1MaxKeys = 40960;   // capacity of the one-CTA kernel (shared memory)
+constexpr int kSel1Bins = 4096;
+constexpr int kSel1CandMax = 4096;
+
+struct Sel1Shared {
+    uint32_t hist[kSel1Bins];
+    uint32_t cand[kSel1CandMax];
+    uint32_t warp_a[kSel1Warps];
+    uint32_t warp_b[kSel1Warps];
+    uint32_t pick[2];       // chosen digit, remaining rank
+    uint32_t n_cand;
+};
+
+// Exclusive prefix sums of (a, b) over the threads of the CTA, in thread order.
+__device__ __forceinline__ void block_excl_scan2(uint32_t a, uint32_t b, uint32_t* wa, uint32_t* wb,
+                                                 uint32_t& ex_a, uint32_t& ex_b, uint32_t& tot_a, uint32_t& tot_b) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t ia = a, ib = b;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t x = __shfl_up_sync(0xFFFFFFFFu, ia, o), y = __shfl_up_sync(0xFFFFFFFFu, ib, o);
+        if (lane >= o) { ia += x; ib += y; }
+    }
+    if (lane == 31) { wa[warp] = ia; wb[warp] = ib; }
+    __syncthreads();
+    uint32_t va = wa[lane], vb = wb[lane];   // kSel1Warps == 32: one warp total per lane
+    uint32_t sa = va, sb = vb;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t x = __shfl_up_sync(0xFFFFFFFFu, sa, o), y = __shfl_up_sync(0xFFFFFFFFu, sb, o);
+        if (lane >= o) { sa += x; sb += y; }
+    }
+    tot_a = __shfl_sync(0xFFFFFFFFu, sa, 31);
+    tot_b = __shfl_sync(0xFFFFFFFFu, sb, 31);
+    ex_a = __shfl_sync(0xFFFFFFFFu, sa - va, warp) + ia - a;
+    ex_b = __shfl_sync(0xFFFFFFFFu, sb - vb, warp) + ib - b;
+    __syncthreads();   // wa/wb may be reused by the next scan
+}
+
+// Adds one to hist[bin] for every thread with `in`; a warp whose keys share one bin adds once.
+__device__ __forceinline__ void hist_add(uint32_t* hist, bool in, uint32_t bin) {
+    const int lane = threadIdx.x & 31;
+    const uint32_t active = __ballot_sync(0xFFFFFFFFu, in);
+    if (active == 0u) return;
+    const int leader = __ffs(active) - 1;
+    const uint32_t lead_bin = __shfl_sync(0xFFFFFFFFu, bin, leader);
+    const uint32_t same = __ballot_sync(0xFFFFFFFFu, in && bin == lead_bin);
+    if (same == active) {
+        if (lane == leader) atomicAdd(&hist[lead_bin], (uint32_t)__popc(active));
+    } else if (in) {
+        atomicAdd(&hist[bin], 1u);
+    }
+}
+
+// Finds, from the top, the bin in which the k_rem-th element falls.  Thread t owns `per` consecutive
+// bins in descending order; the result goes to pick[0] (bin) and pick[1] (rank inside that bin).
+__device__ __forceinline__ void pick_bin(Sel1Shared* sh, int n_bins, int per) {
+    const int tid = threadIdx.x;
+    const int top = n_bins - 1 - tid * per;   // this thread's highest bin
+    uint32_t s = 0;
+    if (top >= 0)
+        for (int b = 0; b < per; ++b) s += sh->hist[top - b];
+    uint32_t above, dummy, tot, tot2;
+    block_excl_scan2(s, 0u, sh->warp_a, sh->warp_b, above, dummy, tot, tot2);
+    const uint32_t k_rem = sh->pick[1];
+    if (top >= 0 && k_rem > above && k_rem <= above + s) {
+        uint32_t a = above;
+        for (int b = 0; b < per; ++b) {
+            const uint32_t c = sh->hist[top - b];
+            if (k_rem <= a + c) { sh->pick[0] = (uint32_t)(top - b); sh->pick[1] = k_rem - a; break; }
+            a += c;
+        }
+    }
+    __syncthreads();
+}
+
+__global__ void __launch_bounds__(kSel1Threads, 1)
+select_topk_cta_kernel(const float* __restrict__ scores, int n_sig, int L_d, int k, int32_t* __restrict__ idx_out) {
+    extern __shared__ __align__(16) unsigned char sel_smem[];
+    Sel1Shared* sh = reinterpret_cast<Sel1Shared*>(sel_smem);
+    uint32_t* keys = reinterpret_cast<uint32_t*>(sel_smem + sizeof(Sel1Shared));
+    const int tid = threadIdx.x;
+
+    for (int i = tid; i < kSel1Bins; i += kSel1Threads) sh->hist[i] = 0u;
+    if (tid == 0) { sh->pick[0] = 0u; sh->pick[1] = (uint32_t)k; sh->n_cand = 0u; }
+    __syncthreads();
+    // pass 1 over all keys: aggregate the signal rows in ascending row order, build keys, histogram bits [31:20]
+    const int n_round = (L_d + 31) / 32 * 32;
+    for (int i = tid; i < n_round; i += kSel1Threads) {
+        uint32_t key = 0u;
+        if (i < L_d) {
+            float acc = scores[i];
+            for (int l = 1; l < n_sig; ++l) acc = __fadd_rn(acc, scores[(size_t)l * L_d + i]);
+            key = score_key(acc);
+            keys[i] = key;
+        }
+        hist_add(sh->hist, i < L_d, key >> 20);
+    }
+    __syncthreads();
+    pick_bin(sh, kSel1Bins, kSel1Bins / kSel1Threads);
+    const uint32_t d1 = sh->pick[0];
+    // candidates: keys whose top 12 bits equal d1
+    for (int i = tid; i < L_d; i += kSel1Threads) {
+        const uint32_t key = keys[i];
+        if ((key >> 20) == d1) {
+            const uint32_t slot = atomicAdd(&sh->n_cand, 1u);
+            if (slot < (uint32_t)kSel1CandMax) sh->cand[slot] = key;
+        }
+    }
+    for (int i = tid; i < 1024; i += kSel1Threads) sh->hist[i] = 0u;
+    __syncthreads();
+    const uint32_t n_cand = sh->n_cand;
+    const bool listed = n_cand <= (uint32_t)kSel1CandMax;
+    uint32_t prefix = d1 << 20, mask = 0xFFF00000u;
+    for (int shift = 10; shift >= 0; shift -= 10) {
+        if (listed) {
+            const int n_c_round = ((int)n_cand + 31) / 32 * 32;
+            for (int i = tid; i < n_c_round; i += kSel1Threads) {
+                const uint32_t key = i < (int)n_cand ? sh->cand[i] : 0u;
+                hist_add(sh->hist, i < (int)n_cand && (key & mask) == prefix, (key >> shift) & 0x3FFu);
+            }
+        } else {
+            for (int i = tid; i < n_round; i += kSel1Threads) {
+                const uint32_t key = i < L_d ? keys[i] : 0u;
+                hist_add(sh->hist, i < L_d && (key & mask) == prefix, (key >> shift) & 0x3FFu);
+            }
+        }
+        __syncthreads();
+        pick_bin(sh, 1024, 1);
+        prefix |= sh->pick[0] << shift;
+        mask |= 0x3FFu << shift;
+        if (tid < 1024) sh->hist[tid] = 0u;
+        __syncthreads();
+    }
+    const uint32_t thr = prefix;           // key of the k-th largest score
+    const uint32_t need_eq = sh->pick[1];  // how many keys equal to thr are taken (lowest positions first)
+
+    // ordered compaction: thread t owns the contiguous positions [t*E, (t+1)*E)
+    const int E = (L_d + kSel1Threads - 1) / kSel1Threads;
+    const int lo = min(L_d, tid * E), hi = min(L_d, lo + E);
+    uint32_t n_gt = 0, n_eq = 0;
+    for (int i = lo; i < hi; ++i) {
+        const uint32_t key = keys[i];
+        n_gt += key > thr;
+        n_eq += key == thr;
+    }
+    uint32_t gt_before, eq_before, tot_gt, tot_eq;
+    block_excl_scan2(n_gt, n_eq, sh->warp_a, sh->warp_b, gt_before, eq_before, tot_gt, tot_eq);
+    if (k > 0) {
+        uint32_t pos = gt_before + min(eq_before, need_eq);
+        for (int i = lo; i < hi; ++i) {
+            const uint32_t key = keys[i];
+            bool take = key > thr;
+            if (key == thr) { take = eq_before < need_eq; ++eq_before; }
+            if (take) idx_out[pos++] = i;
+        }
+    }
+}
+
 // --------------------------------------------------- gather + hybrid KV update
 // One CTA per row.  Rows 0..k-1 are the important tokens: their fresh Q/K/V rows
 // go to the packed buffers and (K/V) into the cache rows at their positions.
@@ -256,6 +424,13 @@ fuse_rows_kernel(const FuseArgs a) {
 }
 
 // ----------------------------------------------------------------- host side
+// Measured on B200: one CTA is faster up to about 2K tokens (3.8 vs 6.5 us at 1K); from 6K on the cluster's eight
+// histogram engines win (7.8 vs 18 us at 16K).
+static int g_sel1_max_keys = 2048;   // sizes up to this run in one CTA, larger ones in the cluster kernel
+#ifdef DAF_TRACE
+extern "C" void daf_dbg_sel1_max_keys(int n) { g_sel1_max_keys = n < kSel1MaxKeys ? n : kSel1MaxKeys; }
+#endif
+
 size_t select_scratch_bytes(int L_d) {
     const int per_cta = (L_d + kSelCluster - 1) / kSelCluster;
     return per_cta > kSelSmemKeysPerCta ? ((size_t)per_cta * kSelCluster * sizeof(uint32_t) + 255) / 256 * 256 : 0;
@@ -273,17 +448,25 @@ int launch_select(const ResolvedParams& rp, const float* scores, int n_sig, cons
     const int32_t* idx_src = idx_in;
     if (scores != nullptr && rp.L_d > 0) {
         static bool attr_done[64] = {false};
-        const size_t smem = select_smem_bytes(rp.L_d);
         int dev = 0;
         cudaGetDevice(&dev);
         if (dev >= 0 && dev < 64 && !attr_done[dev]) {
             cudaError_t e = cudaFuncSetAttribute(select_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                  (int)(sizeof(SelShared) + (size_t)kSelSmemKeysPerCta * sizeof(uint32_t)));
+            if (e == cudaSuccess)
+                e = cudaFuncSetAttribute(select_topk_cta_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)(sizeof(Sel1Shared) + (size_t)kSel1MaxKeys * sizeof(uint32_t)));
             if (e != cudaSuccess) { set_cuda_error(e); return DAF_ERR_CUDA; }
             attr_done[dev] = true;
         }
-        select_topk_kernel<<<kSelCluster, kSelThreads, smem, stream>>>(scores, n_sig, rp.L_d, rp.k,
-                                                            reinterpret_cast<uint32_t*>(scratch), idx_out);
+        if (rp.L_d <= g_sel1_max_keys) {
+            const size_t smem1 = sizeof(Sel1Shared) + (size_t)rp.L_d * sizeof(uint32_t);
+            select_topk_cta_kernel<<<1, kSel1Threads, smem1, stream>>>(scores, n_sig, rp.L_d, rp.k, idx_out);
+        } else {
+            const size_t smem = select_smem_bytes(rp.L_d);
+            select_topk_kernel<<<kSelCluster, kSelThreads, smem, stream>>>(scores, n_sig, rp.L_d, rp.k,
+                                                                reinterpret_cast<uint32_t*>(scratch), idx_out);
+        }
         count_launch();
         if (int rc = check_launch()) return rc;
         idx_src = idx_out;

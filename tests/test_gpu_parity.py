@@ -57,6 +57,8 @@ def _normal(shape, seed, scale=1.0):
     (1024, 0.15, 1, "lognormal"), (6144, 0.15, 1, "lognormal"), (16384, 0.10, 3, "lognormal"),
     (32768, 0.20, 1, "pareto"), (1000, 0.1, 2, "ties"), (777, 1.0, 1, "lognormal"), (130, 0.5, 1, "special"),
     (50000, 0.07, 1, "lognormal"), (33, 0.03, 1, "ties"), (4096, 0.25, 1, "constant"),
+    (16384, 0.10, 1, "constant"), (20000, 0.3, 2, "ties"), (40960, 0.2, 1, "lognormal"), (40961, 0.2, 1, "lognormal"),
+    (7, 0.5, 1, "lognormal"), (1, 1.0, 1, "lognormal"),
 ])
 def test_select_indices_bit_exact(L_d, r, n_sig, kind):
     if kind == "pareto":
