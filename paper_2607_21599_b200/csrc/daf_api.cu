@@ -238,24 +238,26 @@ int daf_layer(const daf_params* p, const float* scores, int32_t n_sig, const int
     // (forked and joined with events) and the GPU fills one stage's idle SMs with the other's CTAs.
     const bool both = rp.k > 0 && rp.L_q > 0;
     SideStream* side = both ? side_stream() : nullptr;
-    cudaStream_t st_q = st;
+    cudaStream_t st_i = st;   // the important-token stage moves to the side stream when both stages run
     if (side != nullptr) {
         DAF_CUDA_TRY(cudaEventRecord(side->fork, st));
         DAF_CUDA_TRY(cudaStreamWaitEvent(side->stream, side->fork, 0));
-        st_q = side->stream;
+        st_i = side->stream;
     }
     int rc_q = DAF_OK, rc_i = DAF_OK;
     if (rp.L_q > 0) {
+        // launched right behind the gather kernel of this call on the same stream: may overlap its tail
         const int64_t first_row = rp.fuse_mode == 1 ? rp.L_d : rp.k;
         const char* qq = reinterpret_cast<const char*>(q_fresh) + (int64_t)rp.L_d * row_bytes;
         rc_q = launch_attention(qq, kv_k, kv_v, rp.L_q, rp.N, rp.Hq, rp.Hkv, rp.L_d, rp.scale, true, true,
                                 h + first_row * row_bytes, row_bytes, nullptr, nullptr, ws.status, ws.attn_scratch,
-                                ws.attn_bytes, st_q);
+                                ws.attn_bytes, st, /*after_kernel=*/true);
     }
     if (rp.k > 0) {
         const int32_t* dst = rp.fuse_mode == 1 ? idx_out : nullptr;
         rc_i = launch_attention(q_pack, k_pack, v_pack, rp.k, rp.k, rp.Hq, rp.Hkv, 0, rp.scale, false, false, h,
-                                row_bytes, dst, nullptr, ws.status, ws.attn_scratch, ws.attn_bytes, st);
+                                row_bytes, dst, nullptr, ws.status, ws.attn_scratch, ws.attn_bytes, st_i,
+                                /*after_kernel=*/side == nullptr);
     }
     if (side != nullptr) {   // always re-join, also after a failed launch, so that the streams stay consistent
         DAF_CUDA_TRY(cudaEventRecord(side->join, side->stream));

@@ -110,6 +110,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     unsigned char* kv_smem = smem + (size_t)kNQ * kTileBytes;       // kStages tiles
     AttnSmem<NQ>* sm = reinterpret_cast<AttnSmem<NQ>*>(kv_smem + (size_t)kStages * kTileBytes);
 
+    pdl_wait();                // inputs may come from the kernel launched just before (gather / hybrid-cache update)
+    pdl_launch_dependents();   // a dependent kernel (the split merge) may start launching; it waits for this grid
+
     // a CTA of this grid (or an earlier kernel sharing the workspace) has already given up: do nothing
     __shared__ int skip_cta;
     if (threadIdx.x == 0) skip_cta = (a.status != nullptr && *reinterpret_cast<volatile int*>(&a.status->code) != 0) ? 1 : 0;
@@ -495,6 +498,7 @@ __global__ void __launch_bounds__(256)
 attn_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_lse, int n_splits, int n_q, int Hq,
                     __nv_bfloat16* __restrict__ out, long long out_row_stride, const int32_t* __restrict__ dst_rows,
                     float* __restrict__ lse) {
+    pdl_wait();                // partial results come from the attention kernel launched just before
     const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (row >= n_q * Hq) return;
@@ -621,7 +625,7 @@ size_t attn_partial_bytes(int n_q, int Hq, int n_splits) {
 int launch_attention(const void* q, const void* k, const void* v, int n_q, int n_kv, int Hq, int Hkv, int causal_off,
                      float scale, bool pack_group, bool allow_split, void* out, long long out_row_stride_bytes,
                      const int32_t* dst_rows, float* lse, DeviceStatus* status, void* scratch, size_t scratch_bytes,
-                     cudaStream_t stream) {
+                     cudaStream_t stream, bool after_kernel) {
     if (n_q <= 0) return DAF_OK;
     const int G = Hq / Hkv;
     AttnPlan pl = plan_attention(n_q, n_kv, Hq, G, causal_off, pack_group, allow_split);
@@ -660,15 +664,19 @@ int launch_attention(const void* q, const void* k, const void* v, int n_q, int n
                                  : nullptr;
     a.status = status;
     dim3 grid((unsigned)pl.head_blocks, (unsigned)pl.pairs, (unsigned)pl.n_splits);
-    if (pl.nq == 2) attn_fwd_kernel<2><<<grid, AttnCfg<2>::kThreads, attn_smem_bytes<2>(), stream>>>(tq, tk, tv, a);
-    else attn_fwd_kernel<1><<<grid, AttnCfg<1>::kThreads, attn_smem_bytes<1>(), stream>>>(tq, tk, tv, a);
+    cudaError_t e;
+    if (pl.nq == 2) e = launch_kernel(attn_fwd_kernel<2>, grid, dim3(AttnCfg<2>::kThreads), attn_smem_bytes<2>(), stream, after_kernel, tq, tk, tv, a);
+    else e = launch_kernel(attn_fwd_kernel<1>, grid, dim3(AttnCfg<1>::kThreads), attn_smem_bytes<1>(), stream, after_kernel, tq, tk, tv, a);
     count_launch();
+    if (e != cudaSuccess) { set_cuda_error(e); return DAF_ERR_CUDA; }
     if (int rc = check_launch()) return rc;
     if (pl.n_splits > 1) {
         const int rows = n_q * Hq;
-        attn_combine_kernel<<<(rows + 7) / 8, 256, 0, stream>>>(a.part_o, a.part_lse, pl.n_splits, n_q, Hq, a.out,
-                                                                a.out_row_stride, dst_rows, lse);
+        e = launch_kernel(attn_combine_kernel, dim3((unsigned)((rows + 7) / 8)), dim3(256), 0, stream, /*after_kernel=*/true,
+                          (const float*)a.part_o, (const float*)a.part_lse, pl.n_splits, n_q, Hq, a.out, a.out_row_stride,
+                          dst_rows, lse);
         count_launch();
+        if (e != cudaSuccess) { set_cuda_error(e); return DAF_ERR_CUDA; }
         if (int rc = check_launch()) return rc;
     }
     return DAF_OK;

@@ -49,10 +49,33 @@ size_t attn_partial_bytes(int n_q, int Hq, int n_splits);
 int launch_attention(const void* q, const void* k, const void* v, int n_q, int n_kv, int Hq, int Hkv, int causal_off,
                      float scale, bool pack_group, bool allow_split, void* out, long long out_row_stride_bytes,
                      const int32_t* dst_rows, float* lse, DeviceStatus* status, void* scratch, size_t scratch_bytes,
-                     cudaStream_t stream);
+                     cudaStream_t stream, bool after_kernel = false);
 
 // ---------------------------------------------------------------- device side
 #ifdef __CUDACC__
+
+// Launch helper.  With `after_kernel` the launch carries the programmatic-serialization attribute:
+// the kernel may start while the previous kernel of the stream is still draining and must call
+// pdl_wait() before it touches anything that kernel wrote.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                 bool after_kernel, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = after_kernel ? 1 : 0;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
+// Programmatic dependent launch: wait for the preceding kernel's results / let the next kernel start launching.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 __device__ __forceinline__ void report_status(DeviceStatus* st, int code, int where, int detail) {
     if (st != nullptr && atomicCAS(&st->code, 0, code) == 0) {

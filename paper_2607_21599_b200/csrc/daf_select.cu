@@ -46,6 +46,7 @@ select_topk_kernel(const float* __restrict__ scores, int n_sig, int L_d, int k,
                    uint32_t* __restrict__ gkeys, int32_t* __restrict__ idx_out) {
     namespace cg = cooperative_groups;
     cg::cluster_group cluster = cg::this_cluster();
+    pdl_launch_dependents();   // the gather kernel may start launching; it waits for this grid before reading idx
     extern __shared__ __align__(16) unsigned char sel_smem[];
     SelShared* sh = reinterpret_cast<SelShared*>(sel_smem);
     uint32_t* skeys = reinterpret_cast<uint32_t*>(sel_smem + sizeof(SelShared));
@@ -184,11 +185,10 @@ select_topk_kernel(const float* __restrict__ scores, int n_sig, int L_d, int k,
 // one CTA with no cluster traffic.  One pass over all keys histograms their top 12 bits and finds
 // the bin that holds the k-th largest key; only the keys of that bin (typically a few per cent)
 // go on to two 10-bit passes that fix the remaining 20 bits; an ordered compaction then emits the
-// positions.  If the bin holds more keys than the candidate list can take (many equal scores),
-// the two small passes walk all keys with a filter instead.
+// positions.
 constexpr int kSel1Threads = 1024;
 constexpr int kSel1Warps = kSel1Threads / 32;
-constexpr int kSel1MaxKeys = 40960;   // capacity of the one-CTA kernel (shared memory)
+constexpr int kSel1MaxKeys = 4096;    // capacity of the one-CTA kernel (= candidate list size)
 constexpr int kSel1Bins = 4096;
 constexpr int kSel1CandMax = 4096;
 
@@ -270,6 +270,7 @@ select_topk_cta_kernel(const float* __restrict__ scores, int n_sig, int L_d, int
     Sel1Shared* sh = reinterpret_cast<Sel1Shared*>(sel_smem);
     uint32_t* keys = reinterpret_cast<uint32_t*>(sel_smem + sizeof(Sel1Shared));
     const int tid = threadIdx.x;
+    pdl_launch_dependents();   // the gather kernel may start launching; it waits for this grid before reading idx
 
     for (int i = tid; i < kSel1Bins; i += kSel1Threads) sh->hist[i] = 0u;
     if (tid == 0) { sh->pick[0] = 0u; sh->pick[1] = (uint32_t)k; sh->n_cand = 0u; }
@@ -293,27 +294,18 @@ select_topk_cta_kernel(const float* __restrict__ scores, int n_sig, int L_d, int
     for (int i = tid; i < L_d; i += kSel1Threads) {
         const uint32_t key = keys[i];
         if ((key >> 20) == d1) {
-            const uint32_t slot = atomicAdd(&sh->n_cand, 1u);
-            if (slot < (uint32_t)kSel1CandMax) sh->cand[slot] = key;
+            sh->cand[atomicAdd(&sh->n_cand, 1u)] = key;
         }
     }
     for (int i = tid; i < 1024; i += kSel1Threads) sh->hist[i] = 0u;
     __syncthreads();
-    const uint32_t n_cand = sh->n_cand;
-    const bool listed = n_cand <= (uint32_t)kSel1CandMax;
+    const int n_cand = (int)sh->n_cand;    // at most L_d <= kSel1CandMax, so the list never overflows
     uint32_t prefix = d1 << 20, mask = 0xFFF00000u;
     for (int shift = 10; shift >= 0; shift -= 10) {
-        if (listed) {
-            const int n_c_round = ((int)n_cand + 31) / 32 * 32;
-            for (int i = tid; i < n_c_round; i += kSel1Threads) {
-                const uint32_t key = i < (int)n_cand ? sh->cand[i] : 0u;
-                hist_add(sh->hist, i < (int)n_cand && (key & mask) == prefix, (key >> shift) & 0x3FFu);
-            }
-        } else {
-            for (int i = tid; i < n_round; i += kSel1Threads) {
-                const uint32_t key = i < L_d ? keys[i] : 0u;
-                hist_add(sh->hist, i < L_d && (key & mask) == prefix, (key >> shift) & 0x3FFu);
-            }
+        const int n_c_round = (n_cand + 31) / 32 * 32;
+        for (int i = tid; i < n_c_round; i += kSel1Threads) {
+            const uint32_t key = i < n_cand ? sh->cand[i] : 0u;
+            hist_add(sh->hist, i < n_cand && (key & mask) == prefix, (key >> shift) & 0x3FFu);
         }
         __syncthreads();
         pick_bin(sh, 1024, 1);
@@ -366,6 +358,8 @@ struct GatherArgs {
 
 __global__ void __launch_bounds__(kRowThreads)
 gather_update_kernel(const GatherArgs a) {
+    pdl_wait();                // idx comes from the selection kernel launched just before
+    pdl_launch_dependents();   // the attention kernel may start launching; it waits for this grid
     const int row = blockIdx.x;
     const int per_row = a.cq + 2 * a.ckv;
     if (row < a.k) {
@@ -488,8 +482,10 @@ int launch_select(const ResolvedParams& rp, const float* scores, int n_sig, cons
         a.cq = rp.Hq * 16; a.ckv = rp.Hkv * 16;
         a.overwrite = rp.overwrite;
         a.status = status;
-        gather_update_kernel<<<rows, kRowThreads, 0, stream>>>(a);
+        cudaError_t e = launch_kernel(gather_update_kernel, dim3((unsigned)rows), dim3(kRowThreads), 0, stream,
+                                      /*after_kernel=*/idx_src == idx_out && scores != nullptr, a);
         count_launch();
+        if (e != cudaSuccess) { set_cuda_error(e); return DAF_ERR_CUDA; }
         if (int rc = check_launch()) return rc;
     }
     return DAF_OK;
