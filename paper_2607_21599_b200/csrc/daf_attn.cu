@@ -590,6 +590,10 @@ AttnPlan plan_attention(int n_q, int n_kv, int Hq, int G, int causal_off, bool p
     // two tiles per CTA once that alone fills every SM twice over; otherwise one tile per CTA, two CTAs per SM
     const int ctas_two = ((pl.n_tb + 1) / 2) * pl.head_blocks;
     pl.nq = ctas_two >= 2 * kNumSMs ? 2 : 1;
+    // The question stage streams a long KV axis through few query tiles: sharing every K/V tile between
+    // two tiles halves the L2-to-SM traffic, which is what bounds the one-tile shape there
+    // (measured at 32k context: 96 us with one tile per CTA, about 70 us with two).
+    if (allow_split && pl.n_tb >= 2) pl.nq = 2;
     if (g_force_nq == 1 || g_force_nq == 2) pl.nq = g_force_nq;
     pl.pairs = (pl.n_tb + pl.nq - 1) / pl.nq;
     long long kv_hi = (long long)n_q - 1 + causal_off + 1;
