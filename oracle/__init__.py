@@ -15,6 +15,7 @@ from .daf_oracle import (  # noqa: F401
     qd_attn,
     full_causal_attn,
     fuse,
+    deviation_scores,
     daf_layer,
     num_threads,
 )

@@ -31,9 +31,10 @@
  * hand-worked rational example in tests/golden/), against a brute-force masked
  * N x N attention over the concatenated context, and the selection against a
  * library stable argsort and an O(L_d^2) rank count.
- * Parity unpinned: the *meaning* of the importance scores (the paper gives no
- * formula for the per-layer deviation signal); the selection rule applied to
- * given scores is pinned.
+ * Parity unpinned: the *formula* of the per-layer deviation signal (the paper names
+ * the signal but gives no formula; daf_oracle_deviation_scores states the reading
+ * taken).  The selection rule applied to given scores is pinned, and so is the
+ * arithmetic of the chosen deviation formula.
  */
 #include <math.h>
 #include <stdint.h>
@@ -217,6 +218,29 @@ void daf_oracle_full_causal_attn(const float *q, const float *k, const float *v,
                                  const int32_t *rows, int32_t n_rows, double *out, double *lse)
 {
     attention_rows(q, k, v, n, n, Hq, Hkv, D, scale, 0, rows, n_rows, out, lse);
+}
+
+/* Per-layer importance signal (Methods, item 1: important tokens are found from the
+ * deviation between the freshly computed and the offline KV states of a layer).  The
+ * paper names the signal but prints no formula; the reading taken here is the squared
+ * Euclidean deviation of a token's K and V rows, summed over heads and channels:
+ *   s[i] = sum_{h,d} (Kf[i,h,d] - Kc[i,h,d])^2 + (Vf[i,h,d] - Vc[i,h,d])^2 .
+ * Parity unpinned as far as the choice of formula goes; the arithmetic of this
+ * formula is pinned (zero for equal tensors, c^2 for one element off by c, a
+ * hand-worked case, a library sum of squares). */
+void daf_oracle_deviation_scores(const float *k_fresh, const float *v_fresh, const float *k_cached,
+                                 const float *v_cached, int32_t L_d, int64_t row_elems, double *s_out)
+{
+#pragma omp parallel for schedule(static)
+    for (int32_t i = 0; i < L_d; ++i) {
+        double acc = 0.0;
+        for (int64_t e = 0; e < row_elems; ++e) {
+            const double dk = (double)k_fresh[(int64_t)i * row_elems + e] - (double)k_cached[(int64_t)i * row_elems + e];
+            const double dv = (double)v_fresh[(int64_t)i * row_elems + e] - (double)v_cached[(int64_t)i * row_elems + e];
+            acc += dk * dk + dv * dv;
+        }
+        s_out[i] = acc;
+    }
 }
 
 /* State fusion (Methods, item 3).  mode 0: compact concatenation, important rows

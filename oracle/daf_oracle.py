@@ -56,6 +56,8 @@ def _load():
         lib.daf_oracle_qd_attn.argtypes = [c_f, c_f, c_f, i32, i32, i32, i32, i32, f64, c_i, i32, c_d, c_d]
         lib.daf_oracle_full_causal_attn.restype = None
         lib.daf_oracle_full_causal_attn.argtypes = [c_f, c_f, c_f, i32, i32, i32, i32, f64, c_i, i32, c_d, c_d]
+        lib.daf_oracle_deviation_scores.restype = None
+        lib.daf_oracle_deviation_scores.argtypes = [c_f, c_f, c_f, c_f, i32, i64, c_d]
         lib.daf_oracle_fuse.restype = None
         lib.daf_oracle_fuse.argtypes = [c_d, c_d, c_i, i32, i32, i32, i64, i32, c_d, c_i]
         lib.daf_oracle_num_threads.restype = i32
@@ -180,6 +182,17 @@ def full_causal_attn(q, k, v, scale: float, rows=None, return_lse: bool = False)
                                         n, Hq, Hkv, D, float(scale), _p(rows_a, ctypes.c_int32), n_rows,
                                         _p(out, ctypes.c_double), _p(lse, ctypes.c_double))
     return (out, lse) if return_lse else out
+
+
+def deviation_scores(k_fresh, v_fresh, k_cached, v_cached, L_d: int) -> np.ndarray:
+    """fp64 [L_d]: squared deviation of each document token's fresh K/V rows from its cached rows."""
+    kf, vf, kc, vc = _f32(k_fresh), _f32(v_fresh), _f32(k_cached), _f32(v_cached)
+    assert kf.shape[0] >= L_d and kc.shape[0] >= L_d and kf.shape[1:] == kc.shape[1:] == vf.shape[1:] == vc.shape[1:]
+    row_elems = int(np.prod(kf.shape[1:]))
+    out = np.zeros(L_d, dtype=np.float64)
+    _load().daf_oracle_deviation_scores(_p(kf, ctypes.c_float), _p(vf, ctypes.c_float), _p(kc, ctypes.c_float),
+                                        _p(vc, ctypes.c_float), int(L_d), row_elems, _p(out, ctypes.c_double))
+    return out
 
 
 def fuse(o_imp, o_q, idx, L_d: int, mode: int = 0, hidden: Optional[np.ndarray] = None):

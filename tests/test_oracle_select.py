@@ -101,3 +101,28 @@ def test_gather_hybrid_and_fuse_placement():
     exp1[idx] = o_imp
     exp1[L_d:] = o_q
     assert np.array_equal(hid1, exp1) and list(pos1) == list(pos)
+
+
+def test_deviation_scores_closed_forms_and_library_sum():
+    rng = np.random.default_rng(8)
+    L_d, H, D = 9, 2, 4
+    kf = rng.standard_normal((L_d + 3, H, D)).astype(np.float32)   # fresh tensors carry question rows too
+    vf = rng.standard_normal((L_d + 3, H, D)).astype(np.float32)
+    kc, vc = kf[:L_d].copy(), vf[:L_d].copy()
+    assert np.all(oracle.deviation_scores(kf, vf, kc, vc, L_d) == 0.0)          # equal tensors: no deviation
+    kc[4, 1, 2] += 0.5                                                           # one element off by c: c^2
+    vc[6, 0, 0] -= 2.0
+    s = oracle.deviation_scores(kf, vf, kc, vc, L_d)
+    want = np.zeros(L_d)
+    want[4], want[6] = 0.25, 4.0
+    np.testing.assert_allclose(s, want, atol=1e-6)
+    # hand-worked: K differs by (1,2,...,8), V by (1,1,...,1) on token 0 -> 204 + 8
+    kc2, vc2 = kf[:L_d].copy(), vf[:L_d].copy()
+    kc2[0] -= np.arange(1, 9, dtype=np.float32).reshape(H, D)
+    vc2[0] -= 1.0
+    assert abs(oracle.deviation_scores(kf, vf, kc2, vc2, L_d)[0] - 212.0) < 1e-4
+    # library sum of squares on random tensors
+    kc3 = rng.standard_normal((L_d, H, D)).astype(np.float32)
+    vc3 = rng.standard_normal((L_d, H, D)).astype(np.float32)
+    lib = ((kf[:L_d].astype(np.float64) - kc3) ** 2 + (vf[:L_d].astype(np.float64) - vc3) ** 2).sum(axis=(1, 2))
+    np.testing.assert_allclose(oracle.deviation_scores(kf, vf, kc3, vc3, L_d), lib, rtol=1e-12)
