@@ -334,6 +334,13 @@ def run_ours(args, w: W.Workload):
         torch.cuda.synchronize()
         return a.elapsed_time(z) / reps * 1e3 / len(items)
 
+    dev_scores = torch.empty(w.L_d, dtype=torch.float32, device=dev)
+
+    def st_dev(b):
+        api.check(api.daf_deviation_scores(p, b.L["k_fresh"], b.L["v_fresh"], b.L["k_cached"], b.L["v_cached"],
+                                           dev_scores), "daf_deviation_scores")
+
+    us_dev = time_stage(st_dev, bufs)
     us_select = time_stage(st_select, bufs)
     us_imp = time_stage(st_imp, bufs) if w.k > 0 else 0.0
     us_qd = time_stage(st_qd, bufs) if w.L_q > 0 else 0.0
@@ -346,6 +353,7 @@ def run_ours(args, w: W.Workload):
     qd_tflops = flops["question"] / (us_qd * 1e-6) / 1e12 if us_qd else 0.0
     full_tflops = flops["full"] / (us_full * 1e-6) / 1e12
     gather_bytes = 2 * w.k * (w.n_q_heads + 2 * w.n_kv_heads) * 256 + (w.k + 2 * w.L_q) * 2 * w.n_kv_heads * 256
+    dev_bytes = 4 * w.L_d * w.n_kv_heads * 256 + 4 * w.L_d
 
     dominant_is_imp = flops["important"] >= flops["question"]
     roofline = {
@@ -427,6 +435,9 @@ def run_ours(args, w: W.Workload):
                 "important_attn": {"bound": "tensor", "tflops": imp_tflops, "frac": imp_tflops / peaks["bf16_tflops"]},
                 "question_attn": {"bound": "tensor", "tflops": qd_tflops, "frac": qd_tflops / peaks["bf16_tflops"],
                                   "kv_gbs": 2 * w.N * w.n_kv_heads * 256 / (us_qd * 1e-6) / 1e9 if us_qd else None},
+                "deviation_scores": {"bound": "hbm", "us": us_dev, "gbs": dev_bytes / (us_dev * 1e-6) / 1e9,
+                                     "frac": dev_bytes / (us_dev * 1e-6) / 1e9 / peaks["hbm_gbs"],
+                                     "note": "signal layers only; not part of the per-layer step"},
                 "select_gather_update": {"bound": "hbm", "gbs": gather_bytes / (us_select * 1e-6) / 1e9,
                                          "frac": gather_bytes / (us_select * 1e-6) / 1e9 / peaks["hbm_gbs"],
                                          "note": "includes the latency-bound top-k kernel"},

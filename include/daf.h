@@ -74,6 +74,17 @@ size_t daf_workspace_bytes(const daf_params* p);
  * per workspace before its first use (a workspace that is all zero bytes needs no call). */
 int daf_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
 
+/* Per-layer importance signal (Methods item 1: tokens are ranked by the deviation between the
+ * fresh and the offline KV states of a layer; signals of several layers are then aggregated by
+ * daf_select).  The paper gives no formula; this library takes, for document token i,
+ *     s[i] = sum over heads and channels of (Kf - Kc)^2 + (Vf - Vc)^2      (fp32 accumulation).
+ *   k_fresh, v_fresh    [>= L_d, n_kv_heads, 128] fresh K/V of one layer (rows >= L_d are ignored)
+ *   k_cached, v_cached  [>= L_d, n_kv_heads, 128] offline K/V of the same layer
+ *   scores_row          fp32 [L_d] out: one row of the [n_sig, L_d] matrix daf_select takes
+ */
+int daf_deviation_scores(const daf_params* p, const void* k_fresh, const void* v_fresh, const void* k_cached,
+                         const void* v_cached, float* scores_row, void* stream);
+
 /* Step 1 (Methods item 1 "selection", "gather"; item 2 "hybrid KV cache").
  *   scores   fp32 [n_sig, L_d] per-layer importance signals, summed over n_sig in
  *            ascending row order in fp32; the k highest sums are selected (ties:

@@ -187,6 +187,17 @@ int daf_qd_attn(const daf_params* p, const void* q_question, const void* kv_k, c
                             (cudaStream_t)stream);
 }
 
+int daf_deviation_scores(const daf_params* p, const void* k_fresh, const void* v_fresh, const void* k_cached,
+                         const void* v_cached, float* scores_row, void* stream) {
+    ResolvedParams rp;
+    if (int rc = resolve_params(p, &rp)) return rc;
+    if (rp.L_d == 0) return DAF_OK;
+    if (!k_fresh || !v_fresh || !k_cached || !v_cached || !scores_row) return DAF_ERR_INVALID_ARG;
+    if (!aligned16(k_fresh) || !aligned16(v_fresh) || !aligned16(k_cached) || !aligned16(v_cached) ||
+        (reinterpret_cast<uintptr_t>(scores_row) & 3u) != 0) return DAF_ERR_ALIGNMENT;
+    return launch_deviation_scores(rp, k_fresh, v_fresh, k_cached, v_cached, scores_row, (cudaStream_t)stream);
+}
+
 int daf_fuse(const daf_params* p, int32_t k, const int32_t* idx, const void* o_imp, const void* o_q,
              void* hidden, int32_t* row_pos_out, void* stream) {
     ResolvedParams rp;

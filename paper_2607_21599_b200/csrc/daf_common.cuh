@@ -43,6 +43,8 @@ int launch_select(const ResolvedParams& rp, const float* scores, int n_sig, cons
                   DeviceStatus* status, void* scratch, cudaStream_t stream);
 int launch_fuse(const ResolvedParams& rp, const int32_t* idx, const void* o_imp, const void* o_q, void* hidden,
                 int32_t* row_pos_out, cudaStream_t stream);
+int launch_deviation_scores(const ResolvedParams& rp, const void* k_fresh, const void* v_fresh, const void* k_cached,
+                            const void* v_cached, float* scores, cudaStream_t stream);
 struct AttnPlan { int Gp, Tt, n_tb, nq, pairs, head_blocks, n_splits, tiles_per_split; };
 AttnPlan plan_attention(int n_q, int n_kv, int Hq, int G, int causal_off, bool pack_group, bool allow_split);
 size_t attn_partial_bytes(int n_q, int Hq, int n_splits);

@@ -417,6 +417,44 @@ fuse_rows_kernel(const FuseArgs a) {
     for (int c = threadIdx.x; c < a.cq; c += kRowThreads) dst[c] = __ldg(src + c);
 }
 
+// ------------------------------------------------------------ deviation signal
+// Per-layer importance signal of a document token: squared deviation of its fresh K and V rows from
+// the cached ones, summed over heads and channels (Methods, item 1; the formula is this library's
+// reading).  A streaming reduction: one warp per token, 16-byte loads, fp32 accumulation, a fixed
+// shuffle tree, so the result does not depend on the launch shape.
+__device__ __forceinline__ float sq_dev8(const int4 a, const int4 b) {
+    const __nv_bfloat162* x = reinterpret_cast<const __nv_bfloat162*>(&a);
+    const __nv_bfloat162* y = reinterpret_cast<const __nv_bfloat162*>(&b);
+    float acc = 0.f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float2 fx = __bfloat1622float2(x[i]), fy = __bfloat1622float2(y[i]);
+        const float d0 = fx.x - fy.x, d1 = fx.y - fy.y;
+        acc = fmaf(d0, d0, acc);
+        acc = fmaf(d1, d1, acc);
+    }
+    return acc;
+}
+
+__global__ void __launch_bounds__(256)
+deviation_scores_kernel(const int4* __restrict__ k_fresh, const int4* __restrict__ v_fresh,
+                        const int4* __restrict__ k_cached, const int4* __restrict__ v_cached,
+                        int L_d, int chunks_per_row, float* __restrict__ scores) {
+    const int lane = threadIdx.x & 31;
+    const int warps_per_grid = (int)(gridDim.x * (blockDim.x >> 5));
+    for (int tok = (int)(blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)); tok < L_d; tok += warps_per_grid) {
+        const size_t base = (size_t)tok * chunks_per_row;
+        float acc = 0.f;
+        for (int c = lane; c < chunks_per_row; c += 32) {
+            acc += sq_dev8(__ldg(k_fresh + base + c), __ldg(k_cached + base + c));
+            acc += sq_dev8(__ldg(v_fresh + base + c), __ldg(v_cached + base + c));
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+        if (lane == 0) scores[tok] = acc;
+    }
+}
+
 // ----------------------------------------------------------------- host side
 // Measured on B200: one CTA is faster up to about 2K tokens (3.8 vs 6.5 us at 1K); from 6K on the cluster's eight
 // histogram engines win (7.8 vs 18 us at 16K).
@@ -489,6 +527,20 @@ int launch_select(const ResolvedParams& rp, const float* scores, int n_sig, cons
         if (int rc = check_launch()) return rc;
     }
     return DAF_OK;
+}
+
+int launch_deviation_scores(const ResolvedParams& rp, const void* k_fresh, const void* v_fresh, const void* k_cached,
+                            const void* v_cached, float* scores, cudaStream_t stream) {
+    if (rp.L_d == 0) return DAF_OK;
+    const int warps = 8;
+    int blocks = (rp.L_d + warps - 1) / warps;
+    const int max_blocks = 148 * 8;          // a few waves of 256-thread CTAs; each warp then walks several tokens
+    if (blocks > max_blocks) blocks = max_blocks;
+    deviation_scores_kernel<<<blocks, warps * 32, 0, stream>>>(
+        reinterpret_cast<const int4*>(k_fresh), reinterpret_cast<const int4*>(v_fresh),
+        reinterpret_cast<const int4*>(k_cached), reinterpret_cast<const int4*>(v_cached), rp.L_d, rp.Hkv * 16, scores);
+    count_launch();
+    return check_launch();
 }
 
 int launch_fuse(const ResolvedParams& rp, const int32_t* idx, const void* o_imp, const void* o_q, void* hidden,

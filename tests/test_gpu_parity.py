@@ -92,6 +92,39 @@ def test_select_indices_bit_exact(L_d, r, n_sig, kind):
     assert np.array_equal(idx_out[:k].cpu().numpy(), ref)
 
 
+# --------------------------------------------------------------------------- deviation signal
+@pytest.mark.parametrize("L_d,L_q,Hkv", [(1024, 32, 4), (777, 0, 8), (6144, 64, 4), (5, 3, 1), (40000, 16, 8)])
+def test_deviation_scores_match_oracle(L_d, L_q, Hkv):
+    N = L_d + L_q
+    kf, vf = _normal((N, Hkv, 128), 71), _normal((N, Hkv, 128), 72)
+    kc, vc = _normal((L_d, Hkv, 128), 73), _normal((L_d, Hkv, 128), 74)
+    kc[: min(3, L_d)] = kf[: min(3, L_d)]          # tokens whose K did not move
+    p = api.make_params(L_d, L_q, 0.1, 4 * Hkv, Hkv)
+    s = torch.full((L_d + 1,), -1.0, dtype=torch.float32, device="cuda")
+    api.check(api.daf_deviation_scores(p, kf.cuda(), vf.cuda(), kc.cuda(), vc.cuda(), s), "daf_deviation_scores")
+    torch.cuda.synchronize()
+    ref = oracle.deviation_scores(_f(kf), _f(vf), _f(kc), _f(vc), L_d)
+    # fp32 accumulation of Hkv*256 non-negative terms against the fp64 oracle
+    np.testing.assert_allclose(s[:L_d].cpu().numpy().astype(np.float64), ref, rtol=2e-5, atol=0)
+    assert float(s[L_d]) == -1.0, "wrote past the end"
+    # the selection that follows ranks exactly these fp32 scores: the rows it keeps must dominate the rest
+    # in the oracle's scores up to the fp32 rounding of the signal
+    k = api.daf_num_important(L_d, 0.1)
+    if k > 0 and k < L_d:
+        ws = api.alloc_workspace(p)
+        z = torch.zeros(N, 4 * Hkv, 128, dtype=torch.bfloat16, device="cuda")
+        kk = torch.zeros(N, Hkv, 128, dtype=torch.bfloat16, device="cuda")
+        idx_out = torch.zeros(k, dtype=torch.int32, device="cuda")
+        qp = torch.zeros(k, 4 * Hkv, 128, dtype=torch.bfloat16, device="cuda")
+        kp = torch.zeros(k, Hkv, 128, dtype=torch.bfloat16, device="cuda")
+        _ok(api.daf_select(p, s[:L_d].contiguous(), 1, None, z, kk, kk.clone(), kk.clone(), kk.clone(), idx_out, qp, kp,
+                           kp.clone(), ws), ws, "daf_select on deviation scores")
+        sel = np.zeros(L_d, dtype=bool)
+        sel[idx_out.cpu().numpy()] = True
+        assert sel.sum() == k
+        assert ref[sel].min() >= ref[~sel].max() * (1 - 1e-4)
+
+
 # --------------------------------------------------------------------------- gather / hybrid cache / fusion
 @pytest.mark.parametrize("name,Hq,Hkv,L_d,L_q,r", [("c0", 28, 4, 1024, 32, 0.15), ("x", 8, 8, 300, 7, 0.4),
                                                   ("y", 40, 8, 513, 0, 0.2), ("z", 4, 1, 64, 5, 0.0)])
