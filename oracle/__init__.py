@@ -16,6 +16,7 @@ from .daf_oracle import (  # noqa: F401
     full_causal_attn,
     fuse,
     deviation_scores,
+    blend_attn,
     daf_layer,
     num_threads,
 )

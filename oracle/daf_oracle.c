@@ -136,14 +136,15 @@ void daf_oracle_hybrid_kv(const float *cached, const float *fresh, const int32_t
 }
 
 /* Softmax attention of selected query rows, grouped-query heads, causal with an
- * offset: query row p sees keys t <= p + offset (and t < n_kv).
+ * offset: query row p sees keys t <= p + offset (and t < n_kv); when `last_key` is
+ * given, row p sees keys t <= last_key[p] instead.
  *   q   [n_q , Hq , D]   k, v [n_kv, Hkv, D]   token-major, fp32 values
  *   rows: n_rows query-row numbers to evaluate, or NULL for rows 0..n_rows-1
  *   out [n_rows, Hq, D] fp64;  lse [n_rows, Hq] fp64 (may be NULL)
  * Query head h reads KV head h / (Hq / Hkv). */
 static void attention_rows(const float *q, const float *k, const float *v,
                            int32_t n_q, int32_t n_kv, int32_t Hq, int32_t Hkv, int32_t D,
-                           double scale, int64_t offset,
+                           double scale, int64_t offset, const int32_t *last_key,
                            const int32_t *rows, int32_t n_rows, double *out, double *lse)
 {
     const int32_t G = Hq / Hkv;
@@ -156,7 +157,7 @@ static void attention_rows(const float *q, const float *k, const float *v,
             for (int32_t h = 0; h < Hq; ++h) {
                 const int32_t p = rows ? rows[a] : a;
                 const int32_t g = h / G;
-                int64_t n_vis = (int64_t)p + offset + 1;
+                int64_t n_vis = last_key ? (int64_t)last_key[p] + 1 : (int64_t)p + offset + 1;
                 if (n_vis > n_kv) n_vis = n_kv;
                 double *o = out + ((int64_t)a * Hq + h) * D;
                 for (int32_t d = 0; d < D; ++d) o[d] = 0.0;
@@ -198,7 +199,7 @@ void daf_oracle_important_attn(const float *q_pack, const float *k_pack, const f
                                int32_t k, int32_t Hq, int32_t Hkv, int32_t D, double scale,
                                const int32_t *rows, int32_t n_rows, double *out, double *lse)
 {
-    attention_rows(q_pack, k_pack, v_pack, k, k, Hq, Hkv, D, scale, 0, rows, n_rows, out, lse);
+    attention_rows(q_pack, k_pack, v_pack, k, k, Hq, Hkv, D, scale, 0, NULL, rows, n_rows, out, lse);
 }
 
 /* Question-document attention (Methods, item 2): an L_q x (L_d + L_q) attention;
@@ -208,7 +209,7 @@ void daf_oracle_qd_attn(const float *q_question, const float *kv_k, const float 
                         int32_t L_d, int32_t L_q, int32_t Hq, int32_t Hkv, int32_t D, double scale,
                         const int32_t *rows, int32_t n_rows, double *out, double *lse)
 {
-    attention_rows(q_question, kv_k, kv_v, L_q, L_d + L_q, Hq, Hkv, D, scale, L_d, rows, n_rows, out, lse);
+    attention_rows(q_question, kv_k, kv_v, L_q, L_d + L_q, Hq, Hkv, D, scale, L_d, NULL, rows, n_rows, out, lse);
 }
 
 /* Full recomputation (the comparison path of the experiments): causal attention
@@ -217,7 +218,20 @@ void daf_oracle_full_causal_attn(const float *q, const float *k, const float *v,
                                  int32_t n, int32_t Hq, int32_t Hkv, int32_t D, double scale,
                                  const int32_t *rows, int32_t n_rows, double *out, double *lse)
 {
-    attention_rows(q, k, v, n, n, Hq, Hkv, D, scale, 0, rows, n_rows, out, lse);
+    attention_rows(q, k, v, n, n, Hq, Hkv, D, scale, 0, NULL, rows, n_rows, out, lse);
+}
+
+/* Selective recomputation over the full context (Complexity Analysis: the scheme DAF is
+ * compared with lets the important rows and the question rows attend the whole context, at a
+ * cost of about r L_d^2 + L_d L_q, against r^2 L_d^2 + L_q (L_d + L_q) for DAF).  The compact
+ * rows (important rows in position order, then the question rows) each attend every key of
+ * the hybrid cache up to their own position row_pos[j].  Built only to measure that cost
+ * ratio on the same kernels; it is not part of the DAF path. */
+void daf_oracle_blend_attn(const float *q_rows, const float *kv_k, const float *kv_v, const int32_t *row_pos,
+                           int32_t n_q, int32_t n_kv, int32_t Hq, int32_t Hkv, int32_t D, double scale,
+                           const int32_t *rows, int32_t n_rows, double *out, double *lse)
+{
+    attention_rows(q_rows, kv_k, kv_v, n_q, n_kv, Hq, Hkv, D, scale, 0, row_pos, rows, n_rows, out, lse);
 }
 
 /* Per-layer importance signal (Methods, item 1: important tokens are found from the

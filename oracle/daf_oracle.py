@@ -56,6 +56,8 @@ def _load():
         lib.daf_oracle_qd_attn.argtypes = [c_f, c_f, c_f, i32, i32, i32, i32, i32, f64, c_i, i32, c_d, c_d]
         lib.daf_oracle_full_causal_attn.restype = None
         lib.daf_oracle_full_causal_attn.argtypes = [c_f, c_f, c_f, i32, i32, i32, i32, f64, c_i, i32, c_d, c_d]
+        lib.daf_oracle_blend_attn.restype = None
+        lib.daf_oracle_blend_attn.argtypes = [c_f, c_f, c_f, c_i, i32, i32, i32, i32, i32, f64, c_i, i32, c_d, c_d]
         lib.daf_oracle_deviation_scores.restype = None
         lib.daf_oracle_deviation_scores.argtypes = [c_f, c_f, c_f, c_f, i32, i64, c_d]
         lib.daf_oracle_fuse.restype = None
@@ -181,6 +183,21 @@ def full_causal_attn(q, k, v, scale: float, rows=None, return_lse: bool = False)
     _load().daf_oracle_full_causal_attn(_p(q, ctypes.c_float), _p(k, ctypes.c_float), _p(v, ctypes.c_float),
                                         n, Hq, Hkv, D, float(scale), _p(rows_a, ctypes.c_int32), n_rows,
                                         _p(out, ctypes.c_double), _p(lse, ctypes.c_double))
+    return (out, lse) if return_lse else out
+
+
+def blend_attn(q_rows, kv_k, kv_v, row_pos, scale: float, rows=None, return_lse: bool = False):
+    """Compact rows (positions row_pos, ascending) attend every key t <= row_pos[j] of kv_k / kv_v."""
+    q, k, v, Hq, Hkv, D = _attn_shapes(q_rows, kv_k, kv_v)
+    pos = _i32(row_pos)
+    n_q = q.shape[0]
+    assert pos.shape[0] == n_q and (n_q == 0 or int(pos.max()) < k.shape[0])
+    rows_a, n_rows = _rows_arg(rows, n_q)
+    out = np.zeros((n_rows, Hq, D), dtype=np.float64)
+    lse = np.zeros((n_rows, Hq), dtype=np.float64)
+    _load().daf_oracle_blend_attn(_p(q, ctypes.c_float), _p(k, ctypes.c_float), _p(v, ctypes.c_float),
+                                  _p(pos, ctypes.c_int32), n_q, k.shape[0], Hq, Hkv, D, float(scale),
+                                  _p(rows_a, ctypes.c_int32), n_rows, _p(out, ctypes.c_double), _p(lse, ctypes.c_double))
     return (out, lse) if return_lse else out
 
 

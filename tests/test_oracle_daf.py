@@ -128,3 +128,30 @@ def test_flop_model_matches_complexity_terms():
           for n in W.CONFIGS}
     assert abs(gf["c0"] - 0.648) < 0.001 and abs(gf["c1"] - 11.77) < 0.01
     assert abs(gf["c2"] - 56.5) < 0.1 and abs(gf["c3"] - 368.2) < 0.1
+
+
+def test_full_context_variant_against_masked_library_attention():
+    """Rows at positions row_pos attend every key up to their position (selective recomputation over the
+    full context): pinned by a library attention with an explicit mask, by the identity position map
+    (plain causal attention) and by the question rows of the DAF layer."""
+    w = W.tiny(L_d=40, doc_len=8, L_q=4, r=0.25, n_q_heads=6, n_kv_heads=2, head_dim=8)
+    L = W.make_layer(w, 7)
+    q, kf, vf, kc, vc = (_np(L[n]) for n in ("q_fresh", "k_fresh", "v_fresh", "k_cached", "v_cached"))
+    base = oracle.daf_layer(q, kf, vf, kc, vc, 40, 4, w.softmax_scale, scores=L["scores"].numpy(), r=0.25)
+    pos = base["row_pos"]
+    q_rows = q[pos]
+    got = oracle.blend_attn(q_rows, base["kv_k"], base["kv_v"], pos, w.softmax_scale)
+    qt = torch.from_numpy(q_rows).double().permute(1, 0, 2)[None]
+    kt = torch.from_numpy(base["kv_k"]).double().permute(1, 0, 2)[None].repeat_interleave(3, 1)
+    vt = torch.from_numpy(base["kv_v"]).double().permute(1, 0, 2)[None].repeat_interleave(3, 1)
+    mask = torch.arange(44)[None, :] <= torch.from_numpy(pos.astype(np.int64))[:, None]
+    ref = torch.nn.functional.scaled_dot_product_attention(qt, kt, vt, attn_mask=mask, scale=w.softmax_scale)
+    np.testing.assert_allclose(got, ref[0].permute(1, 0, 2).numpy(), rtol=0, atol=1e-12)
+    # the question rows of this variant are the question stage of DAF
+    np.testing.assert_allclose(got[len(base["idx"]):], base["o_q"], rtol=0, atol=1e-13)
+    # identity position map: plain causal attention
+    ident = oracle.blend_attn(q, kf, vf, np.arange(44), w.softmax_scale)
+    np.testing.assert_allclose(ident, oracle.full_causal_attn(q, kf, vf, w.softmax_scale), rtol=0, atol=1e-13)
+    # a row subset is the same rows
+    sub = oracle.blend_attn(q_rows, base["kv_k"], base["kv_v"], pos, w.softmax_scale, rows=[0, 5, len(pos) - 1])
+    assert np.array_equal(sub, got[[0, 5, len(pos) - 1]])
