@@ -74,6 +74,19 @@ size_t daf_workspace_bytes(const daf_params* p);
  * per workspace before its first use (a workspace that is all zero bytes needs no call). */
 int daf_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
 
+/* Comparison variant, not part of the DAF path (Complexity Analysis paragraph: selective recomputation
+ * in which the important rows and the question rows attend the FULL context costs about
+ * r L_d^2 + L_d L_q, against r^2 L_d^2 + L_q (L_d + L_q) for DAF).  Same kernel, with a position per row:
+ *   q_rows   [n_rows, n_q_heads, 128] compact query rows (important rows in position order, then question rows)
+ *   kv_k, kv_v  [N, n_kv_heads, 128]  the hybrid cache
+ *   row_pos  int32 [n_rows] ascending original positions (as daf_fuse / daf_layer report in row_pos_out);
+ *            row j attends keys t <= row_pos[j]
+ *   out      bf16 rows j at out + j * out_row_stride_bytes; lse optional fp32 [n_q_heads, n_rows]
+ */
+int daf_blend_attn(const daf_params* p, int32_t n_rows, const void* q_rows, const void* kv_k, const void* kv_v,
+                   const int32_t* row_pos, void* out, int64_t out_row_stride_bytes, float* lse,
+                   void* workspace, size_t workspace_bytes, void* stream);
+
 /* Per-layer importance signal (Methods item 1: tokens are ranked by the deviation between the
  * fresh and the offline KV states of a layer; signals of several layers are then aggregated by
  * daf_select).  The paper gives no formula; this library takes, for document token i,

@@ -30,7 +30,7 @@ EXPORTS = [
     "daf_num_important", "daf_workspace_bytes", "daf_workspace_init", "daf_select", "daf_important_attn",
     "daf_qd_attn", "daf_fuse", "daf_full_causal_attn", "daf_layer", "daf_layer_host_arena_bytes",
     "daf_layer_host", "daf_poll_status", "daf_strerror", "daf_last_cuda_error", "daf_launch_count",
-    "daf_qd_attn_static", "daf_qd_attn_static_max_bytes", "daf_deviation_scores",
+    "daf_qd_attn_static", "daf_qd_attn_static_max_bytes", "daf_deviation_scores", "daf_blend_attn",
 ]
 
 
@@ -89,6 +89,8 @@ def lib() -> ctypes.CDLL:
         L.daf_qd_attn_static.argtypes = [pp, vp, vp, vp, vp, i64, vp, vp, vp]
         L.daf_qd_attn_static_max_bytes.restype = sz
         L.daf_qd_attn_static_max_bytes.argtypes = []
+        L.daf_blend_attn.restype = ctypes.c_int
+        L.daf_blend_attn.argtypes = [pp, i32, vp, vp, vp, vp, vp, i64, vp, vp, sz, vp]
         L.daf_deviation_scores.restype = ctypes.c_int
         L.daf_deviation_scores.argtypes = [pp, vp, vp, vp, vp, vp, vp]
         L.daf_fuse.restype = ctypes.c_int
@@ -200,6 +202,12 @@ def daf_qd_attn_static(p, q_question, kv_k, kv_v, out, out_row_stride_bytes, dst
 
 def daf_qd_attn_static_max_bytes() -> int:
     return int(lib().daf_qd_attn_static_max_bytes())
+
+
+def daf_blend_attn(p, n_rows, q_rows, kv_k, kv_v, row_pos, out, out_row_stride_bytes, lse, workspace, stream=None) -> int:
+    return lib().daf_blend_attn(ctypes.byref(p), int(n_rows), _ptr(q_rows), _ptr(kv_k), _ptr(kv_v), _ptr(row_pos),
+                                _ptr(out), int(out_row_stride_bytes), _ptr(lse), _ptr(workspace), _nbytes(workspace),
+                                _stream(stream))
 
 
 def daf_deviation_scores(p, k_fresh, v_fresh, k_cached, v_cached, scores_row, stream=None) -> int:

@@ -187,6 +187,24 @@ int daf_qd_attn(const daf_params* p, const void* q_question, const void* kv_k, c
                             (cudaStream_t)stream);
 }
 
+int daf_blend_attn(const daf_params* p, int32_t n_rows, const void* q_rows, const void* kv_k, const void* kv_v,
+                   const int32_t* row_pos, void* out, int64_t out_row_stride_bytes, float* lse,
+                   void* workspace, size_t workspace_bytes_, void* stream) {
+    ResolvedParams rp;
+    if (int rc = resolve_params(p, &rp)) return rc;
+    if (n_rows < 0 || n_rows > rp.N) return DAF_ERR_INVALID_ARG;
+    Workspace ws;
+    if (int rc = carve_workspace(rp, workspace, workspace_bytes_, &ws)) return rc;
+    if (n_rows == 0) return DAF_OK;
+    if (!q_rows || !kv_k || !kv_v || !row_pos) return DAF_ERR_INVALID_ARG;
+    if (!aligned16(q_rows) || !aligned16(kv_k) || !aligned16(kv_v) || (reinterpret_cast<uintptr_t>(row_pos) & 3u)) return DAF_ERR_ALIGNMENT;
+    if (int rc = check_out(out, out_row_stride_bytes, rp.Hq)) return rc;
+    // causal_off = N - n_rows only sizes the launch (last row sees at most N keys); the limits come from row_pos
+    return launch_attention(q_rows, kv_k, kv_v, n_rows, rp.N, rp.Hq, rp.Hkv, rp.N - n_rows, rp.scale, false, false, out,
+                            out_row_stride_bytes, nullptr, lse, ws.status, ws.attn_scratch, ws.attn_bytes,
+                            (cudaStream_t)stream, false, row_pos);
+}
+
 int daf_deviation_scores(const daf_params* p, const void* k_fresh, const void* v_fresh, const void* k_cached,
                          const void* v_cached, float* scores_row, void* stream) {
     ResolvedParams rp;

@@ -70,7 +70,8 @@ struct AttnArgs {
     int Gp;             // query heads per tile (1 or G)
     int Tt;             // tokens per tile = 128 / Gp
     int n_tb;           // token blocks = ceil(n_q / Tt)
-    int causal_off;     // token t sees keys <= t + causal_off
+    int causal_off;     // token t sees keys <= t + causal_off ...
+    const int32_t* q_pos; // ... or, when given, keys <= q_pos[t] (ascending positions of the query tokens)
     int n_splits;       // KV splits (1: write final rows; >1: write partials)
     int tiles_per_split;
     float scale;        // softmax scale
@@ -138,7 +139,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         int nj = 0;
         if (tb < a.n_tb) {
             const int max_tok = min(a.n_q, t0[q] + a.Tt) - 1;
-            const long long kv_hi = min((long long)a.n_kv, (long long)max_tok + a.causal_off + 1);
+            const long long last_key = a.q_pos ? (long long)__ldg(a.q_pos + max_tok) : (long long)max_tok + a.causal_off;
+            const long long kv_hi = min((long long)a.n_kv, last_key + 1);
             const int tiles_total = kv_hi > 0 ? (int)((kv_hi + kBlockN - 1) / kBlockN) : 0;
             nj = max(0, min(tiles_total, j_begin + a.tiles_per_split) - j_begin);
         }
@@ -279,7 +281,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         const int head = h0 + r % a.Gp;
         const bool row_valid_tile = (n_j[q] > 0 || a.n_splits > 1) && (pair * kNQ + q < a.n_tb);
         const bool row_valid = (r < a.Gp * a.Tt) && (tok < a.n_q) && row_valid_tile;
-        const long long lim_ll = (long long)tok + a.causal_off;
+        const long long lim_ll = (a.q_pos && tok < a.n_q) ? (long long)__ldg(a.q_pos + tok) : (long long)tok + a.causal_off;
         const int limit = row_valid ? (int)min(lim_ll, (long long)a.n_kv - 1) : -1;   // last visible key
         const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
         const uint32_t s_addr = tmem + lane_addr + (uint32_t)(q * kBlockN);
@@ -629,7 +631,7 @@ size_t attn_partial_bytes(int n_q, int Hq, int n_splits) {
 int launch_attention(const void* q, const void* k, const void* v, int n_q, int n_kv, int Hq, int Hkv, int causal_off,
                      float scale, bool pack_group, bool allow_split, void* out, long long out_row_stride_bytes,
                      const int32_t* dst_rows, float* lse, DeviceStatus* status, void* scratch, size_t scratch_bytes,
-                     cudaStream_t stream, bool after_kernel) {
+                     cudaStream_t stream, bool after_kernel, const int32_t* q_pos) {
     if (n_q <= 0) return DAF_OK;
     const int G = Hq / Hkv;
     AttnPlan pl = plan_attention(n_q, n_kv, Hq, G, causal_off, pack_group, allow_split);
@@ -656,6 +658,7 @@ int launch_attention(const void* q, const void* k, const void* v, int n_q, int n
     a.n_q = n_q; a.n_kv = n_kv; a.Hq = Hq; a.G = G;
     a.Gp = pl.Gp; a.Tt = pl.Tt; a.n_tb = pl.n_tb;
     a.causal_off = causal_off;
+    a.q_pos = q_pos;
     a.n_splits = pl.n_splits; a.tiles_per_split = pl.tiles_per_split;
     a.scale = scale; a.scale_log2 = scale * 1.4426950408889634f;
     a.out = reinterpret_cast<__nv_bfloat16*>(out);

@@ -51,7 +51,7 @@ size_t attn_partial_bytes(int n_q, int Hq, int n_splits);
 int launch_attention(const void* q, const void* k, const void* v, int n_q, int n_kv, int Hq, int Hkv, int causal_off,
                      float scale, bool pack_group, bool allow_split, void* out, long long out_row_stride_bytes,
                      const int32_t* dst_rows, float* lse, DeviceStatus* status, void* scratch, size_t scratch_bytes,
-                     cudaStream_t stream, bool after_kernel = false);
+                     cudaStream_t stream, bool after_kernel = false, const int32_t* q_pos = nullptr);
 
 // ---------------------------------------------------------------- device side
 #ifdef __CUDACC__

@@ -244,6 +244,32 @@ def test_full_causal_attention_matches_oracle(n, Hq, Hkv):
     _assert_close(out, ref, f"full causal n={n}")
 
 
+@pytest.mark.parametrize("L_d,L_q,r,Hq,Hkv", [(1024, 32, 0.15, 28, 4), (700, 5, 0.3, 8, 2), (2048, 128, 0.05, 40, 8),
+                                               (300, 0, 1.0, 4, 4)])
+def test_full_context_variant_matches_oracle(L_d, L_q, r, Hq, Hkv):
+    w = W.Workload("b", 31, Hq, Hkv, 128, 1, L_d, L_d, L_q, r, "lognormal")
+    L = W.make_layer(w, 0)
+    k = api.daf_num_important(L_d, r)
+    idx = oracle.select(L["scores"].numpy(), k)
+    pos = np.concatenate([idx, np.arange(L_d, L_d + L_q, dtype=np.int32)]).astype(np.int32)
+    kv_k = torch.cat([L["k_cached"], L["k_fresh"][L_d:]], 0)
+    kv_v = torch.cat([L["v_cached"], L["v_fresh"][L_d:]], 0)
+    it = torch.from_numpy(idx).long()
+    kv_k[it], kv_v[it] = L["k_fresh"][it], L["v_fresh"][it]
+    q_rows = L["q_fresh"][torch.from_numpy(pos).long()].contiguous()
+    p = api.make_params(L_d, L_q, r, Hq, Hkv)
+    ws = api.alloc_workspace(p)
+    n = len(pos)
+    out = torch.full((n + 1, Hq, 128), 5.0, dtype=torch.bfloat16, device="cuda")
+    lse = torch.zeros(Hq, n, dtype=torch.float32, device="cuda")
+    _ok(api.daf_blend_attn(p, n, q_rows.cuda(), kv_k.cuda(), kv_v.cuda(), torch.from_numpy(pos).cuda(), out, Hq * 256,
+                           lse, ws), ws, "daf_blend_attn")
+    ref, ref_lse = oracle.blend_attn(_f(q_rows), _f(kv_k), _f(kv_v), pos, 1.0 / math.sqrt(128), return_lse=True)
+    _assert_close(out[:n], ref, f"full-context variant L_d={L_d}")
+    assert torch.all(out[n] == 5.0)
+    np.testing.assert_allclose(lse.cpu().numpy().T, ref_lse, atol=2e-3, rtol=0)
+
+
 def test_closed_forms_on_the_gpu():
     """Zero keys give the running mean of the values; constant values come back unchanged."""
     n, Hq, Hkv = 260, 4, 2
