@@ -415,3 +415,56 @@ def test_fresh_change_at_non_important_row_is_invisible():
     finally:
         W.make_layer = orig
     assert np.array_equal(idx, idx2) and torch.equal(hidden, hidden2)
+
+
+# --------------------------------------------------------------------------- device-side status, edge shapes
+def test_status_word_makes_kernels_stand_down_and_is_reported_once():
+    """A failure recorded in the workspace makes later attention kernels return without touching their
+    outputs; daf_poll_status reports it once and clears it (no GPU fault is involved anywhere)."""
+    n, Hq, Hkv = 300, 4, 2
+    q, k, v = _normal((n, Hq, 128), 81), _normal((n, Hkv, 128), 82), _normal((n, Hkv, 128), 83)
+    p = api.make_params(n, 0, 1.0, Hq, Hkv)
+    ws = api.alloc_workspace(p)
+    ws.view(torch.int32)[0] = api.DAF_ERR_TIMEOUT          # as a CTA whose bounded wait ran out would leave it
+    out = torch.full((n, Hq, 128), 5.0, dtype=torch.bfloat16, device="cuda")
+    api.check(api.daf_important_attn(p, n, q.cuda(), k.cuda(), v.cuda(), out, Hq * 256, None, None, ws), "launch")
+    torch.cuda.synchronize()
+    assert torch.all(out == 5.0), "a kernel ran although the workspace carried a failure"
+    assert api.daf_poll_status(ws) == api.DAF_ERR_TIMEOUT
+    assert api.daf_poll_status(ws) == api.DAF_OK            # reported once, then cleared
+    _ok(api.daf_important_attn(p, n, q.cuda(), k.cuda(), v.cuda(), out, Hq * 256, None, None, ws), ws, "after clearing")
+    _assert_close(out, oracle.important_attn(_f(q), _f(k), _f(v), 1.0 / math.sqrt(128)), "after clearing")
+
+
+def test_out_of_range_index_is_skipped_and_reported():
+    L_d, L_q, Hq, Hkv = 64, 2, 4, 2
+    p = api.make_params(L_d, L_q, 4 / 64, Hq, Hkv)
+    assert api.daf_num_important(L_d, 4 / 64) == 4
+    ws = api.alloc_workspace(p)
+    dev = "cuda"
+    qf = _normal((L_d + L_q, Hq, 128), 84).to(dev)
+    kf, vf = _normal((L_d + L_q, Hkv, 128), 85).to(dev), _normal((L_d + L_q, Hkv, 128), 86).to(dev)
+    kvk, kvv = torch.zeros_like(kf), torch.zeros_like(kf)
+    idx_in = torch.tensor([3, 9, 1000, 40], dtype=torch.int32, device=dev)     # 1000 is outside [0, L_d)
+    idx_out = torch.zeros(4, dtype=torch.int32, device=dev)
+    qp = torch.full((4, Hq, 128), 3.0, dtype=torch.bfloat16, device=dev)
+    kp = torch.full((4, Hkv, 128), 3.0, dtype=torch.bfloat16, device=dev)
+    vp = torch.full_like(kp, 3.0)
+    api.check(api.daf_select(p, None, 0, idx_in, qf, kf, vf, kvk, kvv, idx_out, qp, kp, vp, ws), "daf_select")
+    torch.cuda.synchronize()
+    assert api.daf_poll_status(ws) == api.DAF_ERR_BOUNDS
+    assert torch.all(qp[2] == 3.0) and torch.equal(qp[0], qf[3]) and torch.equal(qp[3], qf[40])
+
+
+@pytest.mark.parametrize("L_d,L_q,r,Hq,Hkv,n_sig", [(900, 300, 0.2, 4, 4, 1), (512, 40, 1.0, 16, 2, 8),
+                                                     (1500, 130, 0.1, 8, 1, 2), (257, 129, 0.5, 12, 4, 3)])
+def test_layer_edge_shapes(L_d, L_q, r, Hq, Hkv, n_sig):
+    """More than one question token block, group sizes 1 and 8, r = 1 with a question, several signal rows."""
+    w = W.Workload("e", 41, Hq, Hkv, 128, 1, L_d, L_d, L_q, r, "lognormal", n_sig)
+    for fuse_mode in (0, 1):
+        L, hidden, idx, row_pos, kv_k, kv_v = _run_layer(w, 0, fuse_mode)
+        ref = _oracle_layer(w, L, fuse_mode)
+        assert np.array_equal(idx, ref["idx"]) and np.array_equal(row_pos, ref["row_pos"])
+        assert np.array_equal(_f(kv_k), ref["kv_k"]) and np.array_equal(_f(kv_v), ref["kv_v"])
+        rows = np.arange(len(ref["row_pos"])) if fuse_mode == 0 else ref["row_pos"]
+        _assert_close(hidden[rows], ref["hidden"][rows], f"edge shape L_d={L_d} L_q={L_q} mode={fuse_mode}")
