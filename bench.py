@@ -481,13 +481,15 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--config", default="c1", help="c0..c3 or a sweep point name (c4_L<L_d>_r<r>)")
+    ap.add_argument("--config", default="c1", help="c0..c3, a sweep point name (c4_L<L_d>_r<r>) or x136k")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying a CUDA graph")
     ap.add_argument("--layers", type=int, default=0, help="use only the first LAYERS layers (profiling captures)")
     args = ap.parse_args()
     if args.config in W.CONFIGS:
         w = W.CONFIGS[args.config]
+    elif args.config in W.EXTRA_CONFIGS:
+        w = W.EXTRA_CONFIGS[args.config]
     else:
         pts = {x.name: x for x in W.sweep_points()}
         if args.config not in pts:

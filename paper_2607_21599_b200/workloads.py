@@ -141,6 +141,13 @@ CONFIGS: Dict[str, Workload] = {
 }
 
 
+# Beyond the five stated configurations: the shape of the paper's longest evaluation point (a 136k-token
+# context with r = 0.3, Table 1), four layers of it.  Used by the benchmark and one sampled parity test.
+EXTRA_CONFIGS: Dict[str, Workload] = {
+    "x136k": Workload("x136k", 5, 28, 4, 128, 4, 139264, 512, 128, 0.30, "lognormal"),
+}
+
+
 def sweep_points() -> List[Workload]:
     """The single-layer sweep on the Qwen2.5-14B attention shape."""
     pts = []

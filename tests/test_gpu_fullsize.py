@@ -44,6 +44,8 @@ def _check(got_rows_bf16, ref, what):
 def _workload(name):
     if name in W.CONFIGS:
         return W.CONFIGS[name]
+    if name in W.EXTRA_CONFIGS:
+        return W.EXTRA_CONFIGS[name]
     return {w.name: w for w in W.sweep_points()}[name]
 
 
@@ -53,6 +55,7 @@ def _workload(name):
     ("c3", 27, 100, 32, 32),
     ("c4_L32768_r0.30", 0, 64, 24, 0),
     ("c4_L2048_r0.05", 0, 103, 128, 64),
+    ("x136k", 1, 24, 12, 0),
 ])
 def test_layer_at_benchmark_size(name, layer, n_imp_rows, n_q_rows, n_full_rows):
     assert torch.cuda.is_available()
