@@ -62,8 +62,18 @@ static size_t qd_partial_bytes(const ResolvedParams& rp) {
     return attn_partial_bytes(rp.L_q, rp.Hq, pl.n_splits);
 }
 
+// The attention scratch serves the stand-alone question stage and the joint launch of steps 2 and 3.
+static size_t attn_scratch_bytes(const ResolvedParams& rp) {
+    size_t need = qd_partial_bytes(rp);
+    if (rp.k > 0 && rp.L_q > 0) {
+        const size_t joint = joint_partial_bytes(plan_joint(rp.k, rp.L_q, rp.L_d, rp.Hq, rp.G));
+        if (joint > need) need = joint;
+    }
+    return need;
+}
+
 static size_t workspace_bytes(const ResolvedParams& rp) {
-    return kStatusBytes + select_scratch_bytes(rp.L_d) + qd_partial_bytes(rp);
+    return kStatusBytes + select_scratch_bytes(rp.L_d) + attn_scratch_bytes(rp);
 }
 
 static int carve_workspace(const ResolvedParams& rp, void* workspace, size_t bytes, Workspace* ws) {
@@ -101,25 +111,6 @@ static int check_out(const void* out, int64_t stride_bytes, int Hq) {
     if (!aligned16(out) || stride_bytes % 16 != 0) return DAF_ERR_ALIGNMENT;
     if (stride_bytes < (int64_t)Hq * 256) return DAF_ERR_INVALID_ARG;
     return DAF_OK;
-}
-
-// A side stream and two events per device, created on first use and kept for the life of the
-// process (host-side state only; no device memory).
-struct SideStream { cudaStream_t stream; cudaEvent_t fork, join; };
-static SideStream* side_stream() {
-    static SideStream table[64];
-    static bool ready[64] = {false};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
-    if (!ready[dev]) {
-        SideStream s;
-        if (cudaStreamCreateWithFlags(&s.stream, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
-        if (cudaEventCreateWithFlags(&s.fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
-        if (cudaEventCreateWithFlags(&s.join, cudaEventDisableTiming) != cudaSuccess) return nullptr;
-        table[dev] = s;
-        ready[dev] = true;
-    }
-    return &table[dev];
 }
 
 }  // namespace daf
@@ -262,38 +253,25 @@ int daf_layer(const daf_params* p, const float* scores, int32_t n_sig, const int
     if (int rc = do_select(rp, scores, n_sig, idx_in, q_fresh, k_fresh, v_fresh, kv_k, kv_v, idx_out, q_pack, k_pack,
                            v_pack, ws, st)) return rc;
     char* h = reinterpret_cast<char*>(hidden);
-    // State fusion is done by the attention epilogues: each stage writes its final rows.  The two
-    // stages are independent once step 1 is done, so the question stage runs on a side stream
-    // (forked and joined with events) and the GPU fills one stage's idle SMs with the other's CTAs.
-    const bool both = rp.k > 0 && rp.L_q > 0;
-    SideStream* side = both ? side_stream() : nullptr;
-    cudaStream_t st_i = st;   // the important-token stage moves to the side stream when both stages run
-    if (side != nullptr) {
-        DAF_CUDA_TRY(cudaEventRecord(side->fork, st));
-        DAF_CUDA_TRY(cudaStreamWaitEvent(side->stream, side->fork, 0));
-        st_i = side->stream;
+    // State fusion is done by the attention epilogues: each stage writes its final rows.  When both
+    // stages have rows they run as one list of work items in one launch, right behind the gather
+    // kernel of this call (the launch may overlap that kernel's tail).
+    const int64_t first_row = rp.fuse_mode == 1 ? rp.L_d : rp.k;
+    const char* qq = reinterpret_cast<const char*>(q_fresh) + (int64_t)rp.L_d * row_bytes;
+    const int32_t* dst = rp.fuse_mode == 1 ? idx_out : nullptr;
+    if (rp.k > 0 && rp.L_q > 0) {
+        if (int rc = launch_attention_joint(q_pack, k_pack, v_pack, rp.k, h, dst, qq, kv_k, kv_v, rp.L_q, rp.L_d,
+                                            h + first_row * row_bytes, row_bytes, rp.Hq, rp.Hkv, rp.scale, ws.status,
+                                            ws.attn_scratch, ws.attn_bytes, st, /*after_kernel=*/true)) return rc;
+    } else if (rp.L_q > 0) {
+        if (int rc = launch_attention(qq, kv_k, kv_v, rp.L_q, rp.N, rp.Hq, rp.Hkv, rp.L_d, rp.scale, true, true,
+                                      h + first_row * row_bytes, row_bytes, nullptr, nullptr, ws.status, ws.attn_scratch,
+                                      ws.attn_bytes, st, /*after_kernel=*/true)) return rc;
+    } else {
+        if (int rc = launch_attention(q_pack, k_pack, v_pack, rp.k, rp.k, rp.Hq, rp.Hkv, 0, rp.scale, false, false, h,
+                                      row_bytes, dst, nullptr, ws.status, ws.attn_scratch, ws.attn_bytes, st,
+                                      /*after_kernel=*/true)) return rc;
     }
-    int rc_q = DAF_OK, rc_i = DAF_OK;
-    if (rp.L_q > 0) {
-        // launched right behind the gather kernel of this call on the same stream: may overlap its tail
-        const int64_t first_row = rp.fuse_mode == 1 ? rp.L_d : rp.k;
-        const char* qq = reinterpret_cast<const char*>(q_fresh) + (int64_t)rp.L_d * row_bytes;
-        rc_q = launch_attention(qq, kv_k, kv_v, rp.L_q, rp.N, rp.Hq, rp.Hkv, rp.L_d, rp.scale, true, true,
-                                h + first_row * row_bytes, row_bytes, nullptr, nullptr, ws.status, ws.attn_scratch,
-                                ws.attn_bytes, st, /*after_kernel=*/true);
-    }
-    if (rp.k > 0) {
-        const int32_t* dst = rp.fuse_mode == 1 ? idx_out : nullptr;
-        rc_i = launch_attention(q_pack, k_pack, v_pack, rp.k, rp.k, rp.Hq, rp.Hkv, 0, rp.scale, false, false, h,
-                                row_bytes, dst, nullptr, ws.status, ws.attn_scratch, ws.attn_bytes, st_i,
-                                /*after_kernel=*/side == nullptr);
-    }
-    if (side != nullptr) {   // always re-join, also after a failed launch, so that the streams stay consistent
-        DAF_CUDA_TRY(cudaEventRecord(side->join, side->stream));
-        DAF_CUDA_TRY(cudaStreamWaitEvent(st, side->join, 0));
-    }
-    if (rc_q != DAF_OK) return rc_q;
-    if (rc_i != DAF_OK) return rc_i;
     if (row_pos_out != nullptr) {
         if (int rc = launch_fuse(rp, idx_out, nullptr, nullptr, nullptr, row_pos_out, st)) return rc;
     }

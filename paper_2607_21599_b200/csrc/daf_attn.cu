@@ -17,6 +17,7 @@
 // attention; Gp = group size for the question rows, so that one pass over the
 // KV cache serves every query head of the group.
 #include <math.h>
+#include <string.h>
 
 #include "daf_common.cuh"
 
@@ -63,7 +64,8 @@ constexpr size_t attn_smem_bytes() {
     return 1024 /*alignment slack*/ + (size_t)(NQ + AttnCfg<NQ>::kStages) * kTileBytes + sizeof(AttnSmem<NQ>);
 }
 
-struct AttnArgs {
+// One attention problem and how it is cut into work items.
+struct SegArgs {
     int n_q;            // query tokens
     int n_kv;           // key rows
     int Hq, G;          // query heads; group size Hq / Hkv
@@ -72,15 +74,28 @@ struct AttnArgs {
     int n_tb;           // token blocks = ceil(n_q / Tt)
     int causal_off;     // token t sees keys <= t + causal_off ...
     const int32_t* q_pos; // ... or, when given, keys <= q_pos[t] (ascending positions of the query tokens)
-    int n_splits;       // KV splits (1: write final rows; >1: write partials)
-    int tiles_per_split;
+    // Work items.  A unit is NQ adjacent token blocks (the tiles one CTA owns).  Either every unit is cut
+    // into the same n_splits KV ranges of tiles_per_split tiles (chunk == 0), or -- packed causal attention
+    // only, where unit u sees min(NQ (u + 1), n_tb) tiles -- units [g chunk, (g + 1) chunk) are cut into
+    // g + 1 balanced ranges each, so that no item walks more than about NQ * chunk tiles.
+    int head_blocks, n_units;
+    int n_splits, tiles_per_split;
+    int chunk, n_slots;    // n_slots: number of (unit, range) pairs = partial-result slots
+    int n_items;           // head_blocks * (n_units * n_splits  or  n_slots)
     float scale;        // softmax scale
     float scale_log2;   // scale * log2(e)
     __nv_bfloat16* out; long long out_row_stride;  // elements
     const int32_t* dst_rows;
     float* lse;         // [Hq, n_q] or null
-    float* part_o;      // [n_splits, n_q, Hq, 128] fp32, normalised per split
-    float* part_lse;    // [n_splits, n_q, Hq]
+    float* part_o;      // partial results, fp32, normalised per range: [slot rows][Hq][128]
+    float* part_lse;    // [slot rows][Hq]
+};
+
+// A launch runs one problem on a 3-D grid (head block, unit, split), or two problems from one list of
+// items on a 1-D grid (joint): the items of seg[1] first, then those of seg[0], heaviest units first.
+struct AttnArgs {
+    SegArgs seg[2];
+    int joint;
     DeviceStatus* status;
 };
 
@@ -98,8 +113,10 @@ __device__ unsigned long long g_trace[8 * 65536];
 
 template <int NQ>
 __global__ void __launch_bounds__(AttnCfg<NQ>::kThreads, AttnCfg<NQ>::kCtasPerSM)
-attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
-                const __grid_constant__ CUtensorMap tmap_v, const AttnArgs a) {
+attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_constant__ CUtensorMap tmap_k0,
+                const __grid_constant__ CUtensorMap tmap_v0, const __grid_constant__ CUtensorMap tmap_q1,
+                const __grid_constant__ CUtensorMap tmap_k1, const __grid_constant__ CUtensorMap tmap_v1,
+                const AttnArgs args) {
     constexpr int kNQ = NQ;
     constexpr int kStages = AttnCfg<NQ>::kStages;
     constexpr int kTmaWarp = AttnCfg<NQ>::kTmaWarp;
@@ -116,25 +133,76 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
 
     // a CTA of this grid (or an earlier kernel sharing the workspace) has already given up: do nothing
     __shared__ int skip_cta;
-    if (threadIdx.x == 0) skip_cta = (a.status != nullptr && *reinterpret_cast<volatile int*>(&a.status->code) != 0) ? 1 : 0;
+    if (threadIdx.x == 0) skip_cta = (args.status != nullptr && *reinterpret_cast<volatile int*>(&args.status->code) != 0) ? 1 : 0;
     __syncthreads();
     if (skip_cta) return;
 
     if (threadIdx.x == 0) DAF_STAMP(0);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    // blocks are dispatched x-fastest: all head blocks of the heaviest (last) query-tile pair go first
-    const int pair = (int)gridDim.y - 1 - (int)blockIdx.y;
-    const int hb = blockIdx.x, split = blockIdx.z;
+
+    // ---- which item is this CTA's (uniform across the CTA)
+    int seg_id = 0, item = (int)blockIdx.x;
+    if (args.joint) {
+        if (item < args.seg[1].n_items) seg_id = 1;
+        else item -= args.seg[1].n_items;
+    }
+#define DAF_SEG(field) (seg_id ? args.seg[1].field : args.seg[0].field)
+    struct { int n_q, n_kv, G, Gp, Tt, n_tb, causal_off; const int32_t* q_pos; float scale_log2; } a;
+    a.n_q = DAF_SEG(n_q); a.n_kv = DAF_SEG(n_kv); a.G = DAF_SEG(G); a.Gp = DAF_SEG(Gp); a.Tt = DAF_SEG(Tt);
+    a.n_tb = DAF_SEG(n_tb); a.causal_off = DAF_SEG(causal_off); a.q_pos = DAF_SEG(q_pos); a.scale_log2 = DAF_SEG(scale_log2);
+    const CUtensorMap* tmap_q = seg_id ? &tmap_q1 : &tmap_q0;
+    const CUtensorMap* tmap_k = seg_id ? &tmap_k1 : &tmap_k0;
+    const CUtensorMap* tmap_v = seg_id ? &tmap_v1 : &tmap_v0;
+    DeviceStatus* const status = args.status;
+
+    int hb, unit, j_begin, j_end, item_splits, tok_base;
+    long long part_row0;      // this item's first row in the partial-result arrays, in tokens
+    if (!args.joint || DAF_SEG(chunk) == 0) {
+        int split;
+        if (!args.joint) {
+            // blocks are dispatched x-fastest: all head blocks of the heaviest (last) unit go first
+            hb = (int)blockIdx.x; unit = (int)gridDim.y - 1 - (int)blockIdx.y; split = (int)blockIdx.z;
+        } else {
+            const int n_hb = DAF_SEG(head_blocks), n_units = DAF_SEG(n_units);
+            hb = item % n_hb;
+            const int rest = item / n_hb;
+            unit = n_units - 1 - rest % n_units;
+            split = rest / n_units;
+        }
+        const int tps = DAF_SEG(tiles_per_split);
+        j_begin = split * tps;
+        j_end = j_begin + tps;
+        item_splits = DAF_SEG(n_splits);
+        part_row0 = (long long)split * a.n_q;
+        tok_base = 0;
+    } else {
+        // packed causal attention cut into balanced ranges: slot numbers ascend with the unit, the
+        // grid walks them from the top so that the longest items start first
+        const int n_hb = DAF_SEG(head_blocks), chunk = DAF_SEG(chunk);
+        hb = item % n_hb;
+        const int slot = DAF_SEG(n_slots) - 1 - item / n_hb;
+        int g = (int)((sqrtf(1.f + 8.f * (float)slot / (float)chunk) - 1.f) * 0.5f);
+        while (chunk * (g + 1) * (g + 2) / 2 <= slot) ++g;
+        while (g > 0 && chunk * g * (g + 1) / 2 > slot) --g;
+        const int rem = slot - chunk * g * (g + 1) / 2;
+        unit = g * chunk + rem / (g + 1);
+        const int range = rem % (g + 1);
+        const int n_tiles = min(kNQ * (unit + 1), a.n_tb);
+        j_begin = range * n_tiles / (g + 1);
+        j_end = (range + 1) * n_tiles / (g + 1);
+        item_splits = g + 1;
+        part_row0 = (long long)slot * (kNQ * kBlockM);
+        tok_base = unit * (kNQ * kBlockM);
+    }
     const int h0 = hb * a.Gp;
     const int g_kv = h0 / a.G;
 
     // per-tile geometry (uniform across the CTA)
     int t0[kNQ], n_j[kNQ];
-    const int j_begin = split * a.tiles_per_split;
     int n_j_max = 0;
 #pragma unroll
     for (int q = 0; q < kNQ; ++q) {
-        const int tb = pair * kNQ + q;
+        const int tb = unit * kNQ + q;
         t0[q] = tb * a.Tt;
         int nj = 0;
         if (tb < a.n_tb) {
@@ -142,7 +210,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             const long long last_key = a.q_pos ? (long long)__ldg(a.q_pos + max_tok) : (long long)max_tok + a.causal_off;
             const long long kv_hi = min((long long)a.n_kv, last_key + 1);
             const int tiles_total = kv_hi > 0 ? (int)((kv_hi + kBlockN - 1) / kBlockN) : 0;
-            nj = max(0, min(tiles_total, j_begin + a.tiles_per_split) - j_begin);
+            nj = max(0, min(tiles_total, j_end) - j_begin);
         }
         n_j[q] = nj;
         n_j_max = max(n_j_max, nj);
@@ -173,16 +241,16 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     if (warp == kTmaWarp) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            tma_prefetch_desc(&tmap_q);
-            tma_prefetch_desc(&tmap_k);
-            tma_prefetch_desc(&tmap_v);
+            tma_prefetch_desc(tmap_q);
+            tma_prefetch_desc(tmap_k);
+            tma_prefetch_desc(tmap_v);
             const uint32_t q_tx = 2u * 128u * (uint32_t)(a.Gp * a.Tt);
             for (int q = 0; q < kNQ; ++q) {
                 if (n_j[q] > 0) {
                     unsigned char* dst = q_smem + (size_t)q * kTileBytes;
                     mbar_arrive_expect_tx(&sm->q_full[q], q_tx);
-                    tma_load_3d(dst, &tmap_q, &sm->q_full[q], 0, h0, t0[q]);
-                    tma_load_3d(dst + kHalfBytes, &tmap_q, &sm->q_full[q], 64, h0, t0[q]);
+                    tma_load_3d(dst, tmap_q, &sm->q_full[q], 0, h0, t0[q]);
+                    tma_load_3d(dst + kHalfBytes, tmap_q, &sm->q_full[q], 64, h0, t0[q]);
                 }
             }
             bool ok = true;
@@ -192,10 +260,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 for (int kv = 0; kv < 2 && ok; ++kv, ++seq) {
                     const int slot = seq % kStages;
                     const uint32_t round = (uint32_t)(seq / kStages);
-                    if (round > 0) ok = mbar_wait(&sm->kv_empty[slot], (round - 1) & 1u, abort_flag, a.status, 10 + slot);
+                    if (round > 0) ok = mbar_wait(&sm->kv_empty[slot], (round - 1) & 1u, abort_flag, status, 10 + slot);
                     if (!ok) break;
                     unsigned char* dst = kv_smem + (size_t)slot * kTileBytes;
-                    const CUtensorMap* tm = kv == 0 ? &tmap_k : &tmap_v;
+                    const CUtensorMap* tm = kv == 0 ? tmap_k : tmap_v;
                     mbar_arrive_expect_tx(&sm->kv_full[slot], (uint32_t)kTileBytes);
                     tma_load_3d(dst, tm, &sm->kv_full[slot], 0, g_kv, key0);
                     tma_load_3d(dst + kHalfBytes, tm, &sm->kv_full[slot], 64, g_kv, key0);
@@ -214,7 +282,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             constexpr uint32_t idesc_pv = make_idesc_bf16(kBlockM, kD, 1);
             bool ok = true;
             for (int q = 0; q < kNQ && ok; ++q)
-                if (n_j[q] > 0) ok = mbar_wait(&sm->q_full[q], 0, abort_flag, a.status, 20 + q);
+                if (n_j[q] > 0) ok = mbar_wait(&sm->q_full[q], 0, abort_flag, status, 20 + q);
             auto slot_of = [](int seq) { return seq % kStages; };
             auto parity_of = [](int seq) { return (uint32_t)((seq / kStages) & 1); };
             auto issue_qk = [&](int q, int slot) {
@@ -237,7 +305,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                               (first && kk == 0) ? 0u : 1u);
                 }
             };
-            if (ok) ok = mbar_wait(&sm->kv_full[slot_of(0)], parity_of(0), abort_flag, a.status, 30);
+            if (ok) ok = mbar_wait(&sm->kv_full[slot_of(0)], parity_of(0), abort_flag, status, 30);
             if (ok) {
                 tc_fence_after();
                 for (int q = 0; q < kNQ; ++q)
@@ -247,15 +315,15 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             for (int j = 0; j < n_j_max && ok; ++j) {
                 const int seq_v = 2 * j + 1, seq_k = 2 * j + 2;
                 const bool more = j + 1 < n_j_max;
-                ok = mbar_wait(&sm->kv_full[slot_of(seq_v)], parity_of(seq_v), abort_flag, a.status, 31);
-                if (ok && more) ok = mbar_wait(&sm->kv_full[slot_of(seq_k)], parity_of(seq_k), abort_flag, a.status, 32);
+                ok = mbar_wait(&sm->kv_full[slot_of(seq_v)], parity_of(seq_v), abort_flag, status, 31);
+                if (ok && more) ok = mbar_wait(&sm->kv_full[slot_of(seq_k)], parity_of(seq_k), abort_flag, status, 32);
                 if (!ok) break;
                 tc_fence_after();
                 bool last_tile[kNQ];
                 for (int q = 0; q < kNQ && ok; ++q) {
                     last_tile[q] = false;
                     if (j >= n_j[q]) continue;
-                    ok = mbar_wait(&sm->p_full[q], (uint32_t)(j & 1), abort_flag, a.status, 40 + q);
+                    ok = mbar_wait(&sm->p_full[q], (uint32_t)(j & 1), abort_flag, status, 40 + q);
                     if (!ok) break;
                     tc_fence_after();
                     issue_pv(q, slot_of(seq_v), j == 0);
@@ -279,7 +347,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         const int r = quad * 32 + lane;
         const int tok = t0[q] + r / a.Gp;
         const int head = h0 + r % a.Gp;
-        const bool row_valid_tile = (n_j[q] > 0 || a.n_splits > 1) && (pair * kNQ + q < a.n_tb);
+        const bool row_valid_tile = (n_j[q] > 0 || item_splits > 1) && (unit * kNQ + q < a.n_tb);
         const bool row_valid = (r < a.Gp * a.Tt) && (tok < a.n_q) && row_valid_tile;
         const long long lim_ll = (a.q_pos && tok < a.n_q) ? (long long)__ldg(a.q_pos + tok) : (long long)tok + a.causal_off;
         const int limit = row_valid ? (int)min(lim_ll, (long long)a.n_kv - 1) : -1;   // last visible key
@@ -291,7 +359,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         float m = -INFINITY, l = 0.f;
         bool ok = true;
         for (int j = 0; j < n_j[q]; ++j) {
-            ok = mbar_wait(&sm->s_full[q], (uint32_t)(j & 1), abort_flag, a.status, 50 + q);
+            ok = mbar_wait(&sm->s_full[q], (uint32_t)(j & 1), abort_flag, status, 50 + q);
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) break;
             tc_fence_after();
@@ -375,13 +443,19 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         if (threadIdx.x == 0) DAF_STAMP(3);
         // ---- epilogue
         if (ok && n_j[q] > 0) {
-            ok = mbar_wait(&sm->o_done[q], 0, abort_flag, a.status, 60 + q);
+            ok = mbar_wait(&sm->o_done[q], 0, abort_flag, status, 60 + q);
             ok = __all_sync(0xFFFFFFFFu, ok);
         }
         if (ok) {
             tc_fence_after();
+            // the fields only the epilogue needs are picked here, not held in registers through the loop
+            struct { int n_q, Gp, Tt, Hq; __nv_bfloat16* out; long long out_row_stride; const int32_t* dst_rows;
+                     float* lse; float* part_o; float* part_lse; } e;
+            e.n_q = a.n_q; e.Gp = a.Gp; e.Tt = a.Tt; e.Hq = DAF_SEG(Hq);
+            e.out = DAF_SEG(out); e.out_row_stride = DAF_SEG(out_row_stride); e.dst_rows = DAF_SEG(dst_rows);
+            e.lse = DAF_SEG(lse); e.part_o = DAF_SEG(part_o); e.part_lse = DAF_SEG(part_lse);
             const float inv_l = l > 0.f ? 1.f / l : 0.f;
-            const float lse_val = l > 0.f ? m * a.scale + logf(l) : -INFINITY;
+            const float lse_val = l > 0.f ? m * DAF_SEG(scale) + logf(l) : -INFINITY;
             // Rows leave through shared memory so that global stores are whole 256-byte runs: each
             // thread parks its own row (16-byte chunks, XOR-swizzled against bank conflicts) in the
             // part of the Q tile that belongs to its warp (Q is dead once the last MMA has completed),
@@ -394,10 +468,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             // (token, head) pair is tracked incrementally instead of dividing in the loop
             const int sub = lane >> 4, cidx = lane & 15;
             const int r_first = quad * 32 + sub;
-            const int step_t = 2 / a.Gp, step_h = 2 % a.Gp;
-            const int n_rows_tile = a.Gp * a.Tt;
-            if (a.n_splits == 1) {
-                if (row_valid && a.lse != nullptr) a.lse[(size_t)head * a.n_q + tok] = lse_val;
+            const int step_t = 2 / e.Gp, step_h = 2 % e.Gp;
+            const int n_rows_tile = e.Gp * e.Tt;
+            if (item_splits == 1) {
+                if (row_valid && e.lse != nullptr) e.lse[(size_t)head * e.n_q + tok] = lse_val;
                 if (n_j[q] > 0) {
 #pragma unroll
                     for (int cchunk = 0; cchunk < 4; ++cchunk) {
@@ -415,22 +489,22 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                         }
                     }
                     __syncwarp();
-                    int tok_r = t0[q] + r_first / a.Gp, head_off = r_first % a.Gp;
+                    int tok_r = t0[q] + r_first / e.Gp, head_off = r_first % e.Gp;
 #pragma unroll 4
                     for (int i = 0; i < 16; ++i) {
                         const int rr = 2 * i + sub;
-                        if (quad * 32 + rr < n_rows_tile && tok_r < a.n_q) {
-                            const long long drow = a.dst_rows ? (long long)a.dst_rows[tok_r] : (long long)tok_r;
+                        if (quad * 32 + rr < n_rows_tile && tok_r < e.n_q) {
+                            const long long drow = e.dst_rows ? (long long)e.dst_rows[tok_r] : (long long)tok_r;
                             const uint4 w = *reinterpret_cast<const uint4*>(stage + rr * 256 + ((cidx ^ (rr & 7)) << 4));
-                            reinterpret_cast<uint4*>(a.out + drow * a.out_row_stride + (long long)(h0 + head_off) * kD)[cidx] = w;
+                            reinterpret_cast<uint4*>(e.out + drow * e.out_row_stride + (long long)(h0 + head_off) * kD)[cidx] = w;
                         }
                         head_off += step_h; tok_r += step_t;
-                        if (head_off >= a.Gp) { head_off -= a.Gp; ++tok_r; }
+                        if (head_off >= e.Gp) { head_off -= e.Gp; ++tok_r; }
                     }
                 }
             } else {
-                const size_t prow0 = (size_t)split * a.n_q;
-                if (row_valid) a.part_lse[(prow0 + (size_t)tok) * a.Hq + head] = lse_val;
+                const long long prow0 = part_row0 - tok_base;
+                if (row_valid) e.part_lse[(prow0 + tok) * e.Hq + head] = lse_val;
 #pragma unroll
                 for (int half = 0; half < 2; ++half) {   // 64 fp32 columns (256 bytes per row) at a time
                     if (n_j[q] > 0) {
@@ -454,17 +528,17 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                         for (int v = 0; v < 16; ++v) park(v, make_uint4(0u, 0u, 0u, 0u));
                     }
                     __syncwarp();
-                    int tok_r = t0[q] + r_first / a.Gp, head_off = r_first % a.Gp;
+                    int tok_r = t0[q] + r_first / e.Gp, head_off = r_first % e.Gp;
 #pragma unroll 4
                     for (int i = 0; i < 16; ++i) {
                         const int rr = 2 * i + sub;
-                        if (row_valid_tile && quad * 32 + rr < n_rows_tile && tok_r < a.n_q) {
+                        if (row_valid_tile && quad * 32 + rr < n_rows_tile && tok_r < e.n_q) {
                             const uint4 w = *reinterpret_cast<const uint4*>(stage + rr * 256 + ((cidx ^ (rr & 7)) << 4));
-                            float* prow = a.part_o + ((prow0 + (size_t)tok_r) * a.Hq + (h0 + head_off)) * kD + half * 64;
+                            float* prow = e.part_o + ((prow0 + tok_r) * e.Hq + (h0 + head_off)) * kD + half * 64;
                             reinterpret_cast<uint4*>(prow)[cidx] = w;
                         }
                         head_off += step_h; tok_r += step_t;
-                        if (head_off >= a.Gp) { head_off -= a.Gp; ++tok_r; }
+                        if (head_off >= e.Gp) { head_off -= e.Gp; ++tok_r; }
                     }
                     __syncwarp();
                 }
@@ -479,6 +553,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         tc_fence_after();
         tmem_dealloc(tmem, kTmemCols);
     }
+#undef DAF_SEG
 #ifdef DAF_TRACE
     if (threadIdx.x == 0) {
         DAF_STAMP(5);
@@ -489,25 +564,52 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
 }
 
 #ifdef DAF_TRACE
-extern "C" void daf_dbg_force_nq(int nq);
 extern "C" int daf_dbg_read_trace(void* host, size_t bytes) {
     return (int)cudaMemcpyFromSymbol(host, g_trace, bytes < sizeof(g_trace) ? bytes : sizeof(g_trace));
 }
 #endif
 
-// Merge of split-KV partials: one warp per (token, head) row.
+// Merge of partial results: one warp per (token, head) row.  A launch merges the rows of up to two
+// problems (those of s0 first).  A row's partials sit `stride` rows apart; how many there are is the
+// same for every row (n_splits) or, for a problem cut into balanced ranges, follows from its unit.
+struct CombineSeg {
+    const float* part_o; const float* part_lse;
+    int n_q, Hq;
+    int tok_first;       // rows of tokens below this were written in final form by the attention kernel
+    int n_rows;          // (n_q - tok_first) * Hq
+    int n_splits;        // > 0: every row has this many partials, n_q * Hq rows apart
+    int unit_tokens, chunk;   // n_splits == 0: tokens per unit, units per group (see SegArgs)
+    __nv_bfloat16* out; long long out_row_stride; const int32_t* dst_rows; float* lse;
+};
+
 __global__ void __launch_bounds__(256)
-attn_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_lse, int n_splits, int n_q, int Hq,
-                    __nv_bfloat16* __restrict__ out, long long out_row_stride, const int32_t* __restrict__ dst_rows,
-                    float* __restrict__ lse) {
+attn_combine_kernel(const CombineSeg s0, const CombineSeg s1) {
     pdl_wait();                // partial results come from the attention kernel launched just before
-    const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
+    int row = blockIdx.x * 8 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
-    if (row >= n_q * Hq) return;
-    const int tok = row / Hq, head = row % Hq;
-    // lane s holds the log-sum-exp of split s (n_splits <= 32), so all of them are fetched at once
-    const size_t stride = (size_t)n_q * Hq;
-    const float my_lse = lane < n_splits ? part_lse[(size_t)lane * stride + row] : -INFINITY;
+    const bool second = row >= s0.n_rows;
+    if (second) row -= s0.n_rows;
+#define DAF_CS(field) (second ? s1.field : s0.field)
+    if (row >= DAF_CS(n_rows)) return;
+    const int Hq = DAF_CS(Hq), n_q = DAF_CS(n_q);
+    const int tok = DAF_CS(tok_first) + row / Hq, head = row % Hq;
+    int n_splits = DAF_CS(n_splits);
+    size_t first, stride;      // in rows of the partial arrays
+    if (n_splits > 0) {
+        first = (size_t)tok * Hq + head;
+        stride = (size_t)n_q * Hq;
+    } else {
+        const int ut = DAF_CS(unit_tokens), chunk = DAF_CS(chunk);
+        const int unit = tok / ut, g = unit / chunk;
+        n_splits = g + 1;
+        const int slot0 = chunk * g * (g + 1) / 2 + (unit - g * chunk) * (g + 1);
+        first = ((size_t)slot0 * ut + (size_t)(tok - unit * ut)) * Hq + head;
+        stride = (size_t)ut * Hq;
+    }
+    const float* part_o = DAF_CS(part_o);
+    const float* part_lse = DAF_CS(part_lse);
+    // lane s holds the log-sum-exp of partial s (at most 32 of them), so all of them are fetched at once
+    const float my_lse = lane < n_splits ? part_lse[first + (size_t)lane * stride] : -INFINITY;
     float mx = my_lse;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
@@ -516,7 +618,7 @@ attn_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ 
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) wsum += __shfl_xor_sync(0xFFFFFFFFu, wsum, o);
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    const float4* src = reinterpret_cast<const float4*>(part_o + (size_t)row * kD) + lane;
+    const float4* src = reinterpret_cast<const float4*>(part_o + first * kD) + lane;
     int s = 0;
     for (; s + 4 <= n_splits; s += 4) {
         float4 v[4];
@@ -534,12 +636,15 @@ attn_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ 
         acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
     }
     const float inv = wsum > 0.f ? 1.f / wsum : 0.f;
+    const int32_t* dst_rows = DAF_CS(dst_rows);
     const long long drow = dst_rows ? (long long)dst_rows[tok] : (long long)tok;
     uint2 w2;
     w2.x = pack_bf16(acc.x * inv, acc.y * inv);
     w2.y = pack_bf16(acc.z * inv, acc.w * inv);
-    reinterpret_cast<uint2*>(out + drow * out_row_stride + (long long)head * kD)[lane] = w2;
+    reinterpret_cast<uint2*>(DAF_CS(out) + drow * DAF_CS(out_row_stride) + (long long)head * kD)[lane] = w2;
+    float* lse = DAF_CS(lse);
     if (lse != nullptr && lane == 0) lse[(size_t)head * n_q + tok] = wsum > 0.f ? mx + logf(wsum) : -INFINITY;
+#undef DAF_CS
 }
 
 // ----------------------------------------------------------------- host side
@@ -578,9 +683,24 @@ static int make_tmap(CUtensorMap* m, const void* base, int tokens, int heads, in
     return DAF_OK;
 }
 
-// How a problem is cut into CTAs.  Splitting the KV axis is only used for the
+static int set_kernel_attributes() {
+    static bool attr_done[64] = {false};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !attr_done[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(attn_fwd_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem_bytes<1>());
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(attn_fwd_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem_bytes<2>());
+        if (e != cudaSuccess) { set_cuda_error(e); return DAF_ERR_CUDA; }
+        attr_done[dev] = true;
+    }
+    return DAF_OK;
+}
+
+// How a single problem is cut into CTAs.  Splitting the KV axis is only used for the
 // question rows, where there are few query tiles and a long KV axis.
-static int g_force_nq = 0;   // 0: choose by problem size (the tuning builds can pin a shape)
+static int g_force_nq = 0;        // 0: choose by problem size (the tuning builds can pin a shape)
+static float g_joint_factor = 1.0f;   // longest item of a joint launch, as a fraction of the mean load of a CTA slot
 
 AttnPlan plan_attention(int n_q, int n_kv, int Hq, int G, int causal_off, bool pack_group, bool allow_split) {
     AttnPlan pl;
@@ -592,9 +712,8 @@ AttnPlan plan_attention(int n_q, int n_kv, int Hq, int G, int causal_off, bool p
     // two tiles per CTA once that alone fills every SM twice over; otherwise one tile per CTA, two CTAs per SM
     const int ctas_two = ((pl.n_tb + 1) / 2) * pl.head_blocks;
     pl.nq = ctas_two >= 2 * kNumSMs ? 2 : 1;
-    // The question stage streams a long KV axis through few query tiles: sharing every K/V tile between
-    // two tiles halves the L2-to-SM traffic, which is what bounds the one-tile shape there
-    // (measured at 32k context: 96 us with one tile per CTA, about 70 us with two).
+    // The question stage streams a long KV axis through few query tiles: there two tiles per CTA that share
+    // every K/V tile measured faster (at 32k context: 96 us with one tile per CTA, about 70 us with two).
     if (allow_split && pl.n_tb >= 2) pl.nq = 2;
     if (g_force_nq == 1 || g_force_nq == 2) pl.nq = g_force_nq;
     pl.pairs = (pl.n_tb + pl.nq - 1) / pl.nq;
@@ -617,15 +736,105 @@ AttnPlan plan_attention(int n_q, int n_kv, int Hq, int G, int causal_off, bool p
     return pl;
 }
 
-#ifdef DAF_TRACE
-extern "C" void daf_dbg_force_nq(int nq) { g_force_nq = nq; }
-#endif
-
 size_t attn_partial_bytes(int n_q, int Hq, int n_splits) {
     if (n_splits <= 1) return 0;
     size_t o = (size_t)n_splits * n_q * Hq * kD * sizeof(float);
     size_t l = ((size_t)n_splits * n_q * Hq * sizeof(float) + 255) / 256 * 256;
     return o + l;
+}
+
+// Number of (unit, range) slots of units [0, n_units) when groups of `chunk` units are cut into 1, 2, 3, ... ranges.
+static int slots_before(int n_units, int chunk) {
+    const int g = n_units / chunk;
+    return chunk * g * (g + 1) / 2 + (n_units - g * chunk) * (g + 1);
+}
+
+// Steps 2 and 3 of one layer as one list of work items.  The longest item is held to a fraction of the
+// mean load of a CTA slot: long causal chains of the important-token stage are cut into ranges (merged
+// afterwards like the KV splits of the question stage), short ones are left whole.
+JointPlan plan_joint(int k, int L_q, int L_d, int Hq, int G) {
+    JointPlan jp;
+    const int N = L_d + L_q;
+    jp.n_tb_i = (k + kBlockM - 1) / kBlockM;
+    jp.nq = ((jp.n_tb_i + 1) / 2) * Hq >= 2 * kNumSMs ? 2 : 1;
+    if (g_force_nq == 1 || g_force_nq == 2) jp.nq = g_force_nq;
+    jp.n_units_i = (jp.n_tb_i + jp.nq - 1) / jp.nq;
+    jp.Gp_q = G > 128 ? 1 : G;
+    jp.Tt_q = kBlockM / jp.Gp_q;
+    jp.n_tb_q = (L_q + jp.Tt_q - 1) / jp.Tt_q;
+    jp.head_blocks_q = Hq / jp.Gp_q;
+    jp.n_units_q = (jp.n_tb_q + jp.nq - 1) / jp.nq;
+    const int tiles_q = (N + kBlockN - 1) / kBlockN;
+    long long work = 0;   // in CTA steps (one K/V tile through the CTA's tiles)
+    for (int u = 0; u < jp.n_units_i; ++u) work += (long long)Hq * (jp.nq * (u + 1) < jp.n_tb_i ? jp.nq * (u + 1) : jp.n_tb_i);
+    work += (long long)jp.head_blocks_q * jp.n_units_q * tiles_q;
+    const int slots = kNumSMs * (jp.nq == 2 ? 1 : 2);
+    int longest = (int)ceilf(g_joint_factor * (float)work / (float)slots);
+    if (longest < 2) longest = 2;
+    auto set_chunk = [&](int chunk) {
+        if (chunk < 1) chunk = 1;
+        if (chunk < (jp.n_units_i + 31) / 32) chunk = (jp.n_units_i + 31) / 32;   // at most 32 ranges per unit
+        if (chunk > jp.n_units_i) chunk = jp.n_units_i;
+        jp.chunk = chunk;
+        jp.n_slots = slots_before(jp.n_units_i, chunk);
+        jp.part_bytes_i = 0;
+        if (chunk < jp.n_units_i) {
+            const size_t rows = (size_t)jp.n_slots * jp.nq * kBlockM * Hq;
+            jp.part_bytes_i = rows * kD * sizeof(float) + (rows * sizeof(float) + 255) / 256 * 256;
+        }
+    };
+    set_chunk(longest / jp.nq);
+    if (jp.part_bytes_i > ((size_t)256 << 20)) set_chunk(jp.n_units_i);   // partials of a large problem: not worth their traffic
+    jp.items_i = Hq * jp.n_slots;
+    int want = (tiles_q + longest - 1) / longest;
+    if (want > kMaxSplits) want = kMaxSplits;
+    if (want < 1) want = 1;
+    jp.tiles_per_split_q = (tiles_q + want - 1) / want;
+    jp.n_splits_q = (tiles_q + jp.tiles_per_split_q - 1) / jp.tiles_per_split_q;
+    jp.items_q = jp.head_blocks_q * jp.n_units_q * jp.n_splits_q;
+    jp.part_bytes_q = attn_partial_bytes(L_q, Hq, jp.n_splits_q);
+    return jp;
+}
+
+#ifdef DAF_TRACE
+extern "C" void daf_dbg_force_nq(int nq) { g_force_nq = nq; }
+extern "C" void daf_dbg_joint_factor(float f) { g_joint_factor = f; }
+#endif
+
+static void fill_problem(SegArgs* s, int n_q, int n_kv, int Hq, int G, int Gp, int causal_off, const int32_t* q_pos,
+                         float scale, void* out, long long out_row_stride_bytes, const int32_t* dst_rows, float* lse) {
+    s->n_q = n_q; s->n_kv = n_kv; s->Hq = Hq; s->G = G;
+    s->Gp = Gp; s->Tt = kBlockM / Gp; s->n_tb = (n_q + s->Tt - 1) / s->Tt;
+    s->causal_off = causal_off;
+    s->q_pos = q_pos;
+    s->head_blocks = Hq / Gp;
+    s->scale = scale; s->scale_log2 = scale * 1.4426950408889634f;
+    s->out = reinterpret_cast<__nv_bfloat16*>(out);
+    s->out_row_stride = out_row_stride_bytes / 2;
+    s->dst_rows = dst_rows;
+    s->lse = lse;
+}
+
+static void fill_combine(CombineSeg* c, const SegArgs& s, int unit_tokens) {
+    c->part_o = s.part_o; c->part_lse = s.part_lse;
+    c->n_q = s.n_q; c->Hq = s.Hq;
+    c->n_splits = s.chunk == 0 ? s.n_splits : 0;
+    c->unit_tokens = unit_tokens; c->chunk = s.chunk > 0 ? s.chunk : 1;
+    c->tok_first = 0;
+    if (s.chunk == 0 && s.n_splits <= 1) c->tok_first = s.n_q;                    // nothing to merge
+    if (s.chunk > 0) c->tok_first = s.chunk * unit_tokens < s.n_q ? s.chunk * unit_tokens : s.n_q;
+    c->n_rows = (s.n_q - c->tok_first) * s.Hq;
+    c->out = s.out; c->out_row_stride = s.out_row_stride; c->dst_rows = s.dst_rows; c->lse = s.lse;
+}
+
+static int launch_combine(const CombineSeg& c0, const CombineSeg& c1, cudaStream_t stream) {
+    const int rows = c0.n_rows + c1.n_rows;
+    if (rows <= 0) return DAF_OK;
+    cudaError_t e = launch_kernel(attn_combine_kernel, dim3((unsigned)((rows + 7) / 8)), dim3(256), 0, stream,
+                                  /*after_kernel=*/true, c0, c1);
+    count_launch();
+    if (e != cudaSuccess) { set_cuda_error(e); return DAF_ERR_CUDA; }
+    return check_launch();
 }
 
 int launch_attention(const void* q, const void* k, const void* v, int n_q, int n_kv, int Hq, int Hkv, int causal_off,
@@ -642,51 +851,94 @@ int launch_attention(const void* q, const void* k, const void* v, int n_q, int n
     if (int rc = make_tmap(&tq, q, n_q, Hq, pl.Gp, pl.Tt)) return rc;
     if (int rc = make_tmap(&tk, k, n_kv, Hkv, 1, kBlockN)) return rc;
     if (int rc = make_tmap(&tv, v, n_kv, Hkv, 1, kBlockN)) return rc;
-
-    static bool attr_done[64] = {false};
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (dev >= 0 && dev < 64 && !attr_done[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(attn_fwd_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem_bytes<1>());
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(attn_fwd_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem_bytes<2>());
-        if (e != cudaSuccess) { set_cuda_error(e); return DAF_ERR_CUDA; }
-        attr_done[dev] = true;
-    }
+    if (int rc = set_kernel_attributes()) return rc;
 
     AttnArgs a;
-    a.n_q = n_q; a.n_kv = n_kv; a.Hq = Hq; a.G = G;
-    a.Gp = pl.Gp; a.Tt = pl.Tt; a.n_tb = pl.n_tb;
-    a.causal_off = causal_off;
-    a.q_pos = q_pos;
-    a.n_splits = pl.n_splits; a.tiles_per_split = pl.tiles_per_split;
-    a.scale = scale; a.scale_log2 = scale * 1.4426950408889634f;
-    a.out = reinterpret_cast<__nv_bfloat16*>(out);
-    a.out_row_stride = out_row_stride_bytes / 2;
-    a.dst_rows = dst_rows;
-    a.lse = lse;
-    a.part_o = reinterpret_cast<float*>(scratch);
-    a.part_lse = pl.n_splits > 1 ? reinterpret_cast<float*>(reinterpret_cast<char*>(scratch) +
+    memset(&a, 0, sizeof(a));
+    SegArgs& s = a.seg[0];
+    fill_problem(&s, n_q, n_kv, Hq, G, pl.Gp, causal_off, q_pos, scale, out, out_row_stride_bytes, dst_rows, lse);
+    s.n_units = pl.pairs;
+    s.n_splits = pl.n_splits; s.tiles_per_split = pl.tiles_per_split;
+    s.chunk = 0; s.n_slots = 0;
+    s.n_items = pl.head_blocks * pl.pairs * pl.n_splits;
+    s.part_o = reinterpret_cast<float*>(scratch);
+    s.part_lse = pl.n_splits > 1 ? reinterpret_cast<float*>(reinterpret_cast<char*>(scratch) +
                                                             (size_t)pl.n_splits * n_q * Hq * kD * sizeof(float))
                                  : nullptr;
+    a.joint = 0;
     a.status = status;
     dim3 grid((unsigned)pl.head_blocks, (unsigned)pl.pairs, (unsigned)pl.n_splits);
     cudaError_t e;
-    if (pl.nq == 2) e = launch_kernel(attn_fwd_kernel<2>, grid, dim3(AttnCfg<2>::kThreads), attn_smem_bytes<2>(), stream, after_kernel, tq, tk, tv, a);
-    else e = launch_kernel(attn_fwd_kernel<1>, grid, dim3(AttnCfg<1>::kThreads), attn_smem_bytes<1>(), stream, after_kernel, tq, tk, tv, a);
+    if (pl.nq == 2) e = launch_kernel(attn_fwd_kernel<2>, grid, dim3(AttnCfg<2>::kThreads), attn_smem_bytes<2>(), stream, after_kernel, tq, tk, tv, tq, tk, tv, a);
+    else e = launch_kernel(attn_fwd_kernel<1>, grid, dim3(AttnCfg<1>::kThreads), attn_smem_bytes<1>(), stream, after_kernel, tq, tk, tv, tq, tk, tv, a);
     count_launch();
     if (e != cudaSuccess) { set_cuda_error(e); return DAF_ERR_CUDA; }
     if (int rc = check_launch()) return rc;
     if (pl.n_splits > 1) {
-        const int rows = n_q * Hq;
-        e = launch_kernel(attn_combine_kernel, dim3((unsigned)((rows + 7) / 8)), dim3(256), 0, stream, /*after_kernel=*/true,
-                          (const float*)a.part_o, (const float*)a.part_lse, pl.n_splits, n_q, Hq, a.out, a.out_row_stride,
-                          dst_rows, lse);
-        count_launch();
-        if (e != cudaSuccess) { set_cuda_error(e); return DAF_ERR_CUDA; }
-        if (int rc = check_launch()) return rc;
+        CombineSeg c0, c1;
+        fill_combine(&c0, s, pl.nq * kBlockM);
+        memset(&c1, 0, sizeof(c1));
+        return launch_combine(c0, c1, stream);
     }
     return DAF_OK;
+}
+
+size_t joint_partial_bytes(const JointPlan& jp) { return jp.part_bytes_q + jp.part_bytes_i; }
+
+int launch_attention_joint(const void* q_imp, const void* k_imp, const void* v_imp, int k, void* out_imp,
+                           const int32_t* dst_rows_imp, const void* q_question, const void* kv_k, const void* kv_v,
+                           int L_q, int L_d, void* out_question, long long out_row_stride_bytes, int Hq, int Hkv,
+                           float scale, DeviceStatus* status, void* scratch, size_t scratch_bytes, cudaStream_t stream,
+                           bool after_kernel) {
+    const int G = Hq / Hkv, N = L_d + L_q;
+    const JointPlan jp = plan_joint(k, L_q, L_d, Hq, G);
+    if (joint_partial_bytes(jp) > scratch_bytes) return DAF_ERR_WORKSPACE;
+
+    CUtensorMap tq0, tk0, tv0, tq1, tk1, tv1;
+    if (int rc = make_tmap(&tq0, q_imp, k, Hq, 1, kBlockM)) return rc;
+    if (int rc = make_tmap(&tk0, k_imp, k, Hkv, 1, kBlockN)) return rc;
+    if (int rc = make_tmap(&tv0, v_imp, k, Hkv, 1, kBlockN)) return rc;
+    if (int rc = make_tmap(&tq1, q_question, L_q, Hq, jp.Gp_q, jp.Tt_q)) return rc;
+    if (int rc = make_tmap(&tk1, kv_k, N, Hkv, 1, kBlockN)) return rc;
+    if (int rc = make_tmap(&tv1, kv_v, N, Hkv, 1, kBlockN)) return rc;
+    if (int rc = set_kernel_attributes()) return rc;
+
+    AttnArgs a;
+    memset(&a, 0, sizeof(a));
+    char* sc = reinterpret_cast<char*>(scratch);
+    // question rows: every unit cut into the same KV splits
+    SegArgs& sq = a.seg[1];
+    fill_problem(&sq, L_q, N, Hq, G, jp.Gp_q, L_d, nullptr, scale, out_question, out_row_stride_bytes, nullptr, nullptr);
+    sq.n_units = jp.n_units_q;
+    sq.n_splits = jp.n_splits_q; sq.tiles_per_split = jp.tiles_per_split_q;
+    sq.chunk = 0; sq.n_slots = 0;
+    sq.n_items = jp.items_q;
+    sq.part_o = reinterpret_cast<float*>(sc);
+    sq.part_lse = reinterpret_cast<float*>(sc + (size_t)jp.n_splits_q * L_q * Hq * kD * sizeof(float));
+    // important tokens: packed causal attention, long chains cut into balanced ranges
+    SegArgs& si = a.seg[0];
+    fill_problem(&si, k, k, Hq, G, 1, 0, nullptr, scale, out_imp, out_row_stride_bytes, dst_rows_imp, nullptr);
+    si.n_units = jp.n_units_i;
+    si.n_splits = 1; si.tiles_per_split = jp.n_tb_i;
+    si.chunk = jp.chunk; si.n_slots = jp.n_slots;
+    si.n_items = jp.items_i;
+    const size_t rows_i = (size_t)jp.n_slots * jp.nq * kBlockM * Hq;
+    si.part_o = reinterpret_cast<float*>(sc + jp.part_bytes_q);
+    si.part_lse = reinterpret_cast<float*>(sc + jp.part_bytes_q + rows_i * kD * sizeof(float));
+    a.joint = 1;
+    a.status = status;
+
+    dim3 grid((unsigned)(jp.items_q + jp.items_i), 1, 1);
+    cudaError_t e;
+    if (jp.nq == 2) e = launch_kernel(attn_fwd_kernel<2>, grid, dim3(AttnCfg<2>::kThreads), attn_smem_bytes<2>(), stream, after_kernel, tq0, tk0, tv0, tq1, tk1, tv1, a);
+    else e = launch_kernel(attn_fwd_kernel<1>, grid, dim3(AttnCfg<1>::kThreads), attn_smem_bytes<1>(), stream, after_kernel, tq0, tk0, tv0, tq1, tk1, tv1, a);
+    count_launch();
+    if (e != cudaSuccess) { set_cuda_error(e); return DAF_ERR_CUDA; }
+    if (int rc = check_launch()) return rc;
+    CombineSeg ci, cq;
+    fill_combine(&ci, si, jp.nq * kBlockM);
+    fill_combine(&cq, sq, jp.nq * kBlockM);
+    return launch_combine(ci, cq, stream);
 }
 
 }  // namespace daf

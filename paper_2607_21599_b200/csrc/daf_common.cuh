@@ -52,6 +52,20 @@ int launch_attention(const void* q, const void* k, const void* v, int n_q, int n
                      float scale, bool pack_group, bool allow_split, void* out, long long out_row_stride_bytes,
                      const int32_t* dst_rows, float* lse, DeviceStatus* status, void* scratch, size_t scratch_bytes,
                      cudaStream_t stream, bool after_kernel = false, const int32_t* q_pos = nullptr);
+// Steps 2 and 3 of a layer from one list of work items (one attention launch and one merge launch).
+struct JointPlan {
+    int nq;                                   // query tiles per CTA, both stages
+    int n_tb_i, n_units_i, chunk, n_slots, items_i;                       // important-token stage
+    int Gp_q, Tt_q, n_tb_q, n_units_q, head_blocks_q, n_splits_q, tiles_per_split_q, items_q;   // question stage
+    size_t part_bytes_q, part_bytes_i;        // partial results of each stage
+};
+JointPlan plan_joint(int k, int L_q, int L_d, int Hq, int G);
+size_t joint_partial_bytes(const JointPlan& jp);
+int launch_attention_joint(const void* q_imp, const void* k_imp, const void* v_imp, int k, void* out_imp,
+                           const int32_t* dst_rows_imp, const void* q_question, const void* kv_k, const void* kv_v,
+                           int L_q, int L_d, void* out_question, long long out_row_stride_bytes, int Hq, int Hkv,
+                           float scale, DeviceStatus* status, void* scratch, size_t scratch_bytes, cudaStream_t stream,
+                           bool after_kernel);
 
 // ---------------------------------------------------------------- device side
 #ifdef __CUDACC__

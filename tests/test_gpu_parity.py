@@ -345,7 +345,9 @@ def test_layer_smallest_configuration(fuse_mode):
         _assert_close(hidden[rows], ref["hidden"][rows], "fused hidden rows (scatter)")
         others = np.setdiff1d(np.arange(w.N), rows)
         assert torch.all(hidden[others] == -9.0), "a row that is neither important nor a question row was written"
-    # fused epilogues and the stand-alone fusion pass agree bit for bit
+    # fused epilogues and the stand-alone stages + fusion pass agree up to the last bf16 bit or two: the
+    # layer cuts the key axis into different ranges than the stand-alone stages, so the fp32 sums are
+    # associated differently before the final rounding
     p = api.make_params(w.L_d, w.L_q, w.r, w.n_q_heads, w.n_kv_heads, fuse_mode=fuse_mode)
     ws = api.alloc_workspace(p)
     k = len(idx)
@@ -360,7 +362,8 @@ def test_layer_smallest_configuration(fuse_mode):
     h2 = torch.full(hidden.shape, -9.0, dtype=torch.bfloat16, device=dev)
     api.check(api.daf_fuse(p, k, idx_d, o_imp, o_q, h2, None), "daf_fuse")
     torch.cuda.synchronize()
-    assert torch.equal(h2.cpu(), hidden)
+    assert torch.allclose(h2.cpu().float(), hidden.float(), rtol=2.0 ** -6, atol=2e-3)
+    assert torch.equal(h2.cpu() == -9.0, hidden == -9.0)
 
 
 def test_layer_with_selection_and_three_signal_rows():
