@@ -102,6 +102,8 @@ struct AttnArgs {
 #ifdef DAF_TRACE
 // Debug build only (-DDAF_TRACE): per-CTA time stamps for latency studies.
 __device__ unsigned long long g_trace[8 * 65536];
+DAF_KT_TABLE;
+DAF_KT_READER(daf_dbg_kt_attn)
 #define DAF_STAMP(slot)                                                                         \
     do {                                                                                        \
         const unsigned cta_ = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);   \
@@ -111,49 +113,122 @@ __device__ unsigned long long g_trace[8 * 65536];
 #define DAF_STAMP(slot) do {} while (0)
 #endif
 
+// One online-softmax step of one query row (one thread) over NCH * 32 keys starting at `key0`: reads the
+// row's logits from tensor memory, writes P = exp(s - m) as bf16 over the first half of the same columns,
+// keeps the running maximum m and sum l.  Returns the factor the row of O has to be multiplied by (1
+// unless the maximum grew past the lazy threshold).  `limit` is the last key the row may see;
+// c = softmax scale * log2(e).
+template <int NCH>
+__device__ __forceinline__ float softmax_core(uint32_t s_addr, int key0, int limit, float c, float& m, float& l) {
+    constexpr int H = NCH / 2;
+    // the logits are fetched in two halves so that the row maximum of the first half is computed
+    // while the second half is still on its way from tensor memory
+    uint32_t sr[NCH][32];
+#pragma unroll
+    for (int i = 0; i < H; ++i) tmem_ld32(s_addr + (uint32_t)(32 * i), sr[i]);
+    tc_wait_ld();
+#pragma unroll
+    for (int i = H; i < NCH; ++i) tmem_ld32(s_addr + (uint32_t)(32 * i), sr[i]);
+    const bool need_mask = key0 + NCH * 32 - 1 > limit;
+    float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+        if (half == 1) tc_wait_ld();
+        if (need_mask) {
+#pragma unroll
+            for (int cchunk = H * half; cchunk < H * half + H; ++cchunk)
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                    if (key0 + cchunk * 32 + i > limit) sr[cchunk][i] = 0xFF800000u;  // -inf
+        }
+#pragma unroll
+        for (int cchunk = H * half; cchunk < H * half + H; ++cchunk)
+#pragma unroll
+            for (int i = 0; i < 32; i += 8) {
+                // four independent chains of 3-input maxima
+                mx[0] = fmax3(mx[0], __uint_as_float(sr[cchunk][i + 0]), __uint_as_float(sr[cchunk][i + 1]));
+                mx[1] = fmax3(mx[1], __uint_as_float(sr[cchunk][i + 2]), __uint_as_float(sr[cchunk][i + 3]));
+                mx[2] = fmax3(mx[2], __uint_as_float(sr[cchunk][i + 4]), __uint_as_float(sr[cchunk][i + 5]));
+                mx[3] = fmax3(mx[3], __uint_as_float(sr[cchunk][i + 6]), __uint_as_float(sr[cchunk][i + 7]));
+            }
+    }
+    const float tmax = fmax3(mx[0], mx[1], fmaxf(mx[2], mx[3]));
+    float m_new = fmaxf(m, tmax);
+    // keep a slightly stale maximum: rescaling O is skipped while the growth stays below 2^8
+    if (m != -INFINITY && (m_new - m) * c <= kRescaleThreshold) m_new = m;
+    const float m_used = (m_new == -INFINITY) ? 0.f : m_new;
+    const float alpha = (m == -INFINITY) ? 1.f : fast_exp2((m - m_new) * c);
+    const float mc = m_used * c;
+    // p = 2^(s*c - m*c): packed two-wide FMA and adds, exponentials on the special-function unit
+    const uint64_t c2 = pack_f32x2(c, c), nmc2 = pack_f32x2(-mc, -mc);
+    uint64_t acc2[4] = {0ull, 0ull, 0ull, 0ull};
+    uint32_t pr[H][32];
+#pragma unroll
+    for (int cchunk = 0; cchunk < NCH; ++cchunk)
+#pragma unroll
+        for (int i = 0; i < 32; i += 2) {
+            const uint64_t x2 = ffma2(pack_f32x2(__uint_as_float(sr[cchunk][i]), __uint_as_float(sr[cchunk][i + 1])), c2, nmc2);
+            const float p0 = fast_exp2(f32x2_lo(x2));
+            const float p1 = fast_exp2(f32x2_hi(x2));
+            acc2[(i >> 1) & 3] = fadd2(acc2[(i >> 1) & 3], pack_f32x2(p0, p1));
+            pr[cchunk >> 1][(cchunk & 1) * 16 + (i >> 1)] = pack_bf16(p0, p1);
+        }
+    const uint64_t acc01 = fadd2(fadd2(acc2[0], acc2[1]), fadd2(acc2[2], acc2[3]));
+    const float rowsum = f32x2_lo(acc01) + f32x2_hi(acc01);
+    l = l * alpha + rowsum;
+    m = m_new;
+    // P (bf16, two keys per 32-bit column) overlays the first half of the columns of S
+#pragma unroll
+    for (int i = 0; i < H; ++i) tmem_st32(s_addr + (uint32_t)(32 * i), pr[i]);
+    return alpha;
+}
+
+// Multiplies this thread's row of O (128 fp32 columns in tensor memory) by alpha.  O must be quiescent.
+__device__ __forceinline__ void rescale_o(uint32_t o_addr, float alpha) {
+#pragma unroll
+    for (int cchunk = 0; cchunk < 4; ++cchunk) {
+        uint32_t orr[32];
+        tmem_ld32(o_addr + (uint32_t)(cchunk * 32), orr);
+        tc_wait_ld();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * alpha);
+        tmem_st32(o_addr + (uint32_t)(cchunk * 32), orr);
+    }
+}
+
+// A whole 128-key step: the commit that released S_j also covers the previous P V product, so O is
+// quiescent when the row has to be rescaled.
+__device__ __forceinline__ void softmax_step(uint32_t s_addr, uint32_t o_addr, int key0, int limit, float c, bool first,
+                                             float& m, float& l) {
+    const float alpha = softmax_core<4>(s_addr, key0, limit, c, m, l);
+    if (!first && __any_sync(0xFFFFFFFFu, alpha != 1.f)) rescale_o(o_addr, alpha);
+    tc_wait_st();
+    tc_fence_before();
+}
+
+// Picks a field of the problem a CTA works on (seg_id is uniform across the CTA).
+#define DAF_SEG(field) (seg_id ? args.seg[1].field : args.seg[0].field)
+
+// What one CTA works on: the problem's geometry and the CTA's item (a unit of NQ token blocks of one
+// head block, and a range of key tiles).
+struct CtaWork {
+    int n_q, n_kv, G, Gp, Tt, n_tb, causal_off;
+    const int32_t* q_pos;
+    float scale_log2;
+    int seg_id, hb, unit, j_begin, j_end, item_splits, tok_base;
+    long long part_row0;      // the item's first row in the partial-result arrays, in tokens
+};
+
 template <int NQ>
-__global__ void __launch_bounds__(AttnCfg<NQ>::kThreads, AttnCfg<NQ>::kCtasPerSM)
-attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_constant__ CUtensorMap tmap_k0,
-                const __grid_constant__ CUtensorMap tmap_v0, const __grid_constant__ CUtensorMap tmap_q1,
-                const __grid_constant__ CUtensorMap tmap_k1, const __grid_constant__ CUtensorMap tmap_v1,
-                const AttnArgs args) {
-    constexpr int kNQ = NQ;
-    constexpr int kStages = AttnCfg<NQ>::kStages;
-    constexpr int kTmaWarp = AttnCfg<NQ>::kTmaWarp;
-    constexpr int kMmaWarp = AttnCfg<NQ>::kMmaWarp;
-    constexpr int kTmemCols = AttnCfg<NQ>::kTmemCols;
-    extern __shared__ unsigned char attn_smem_raw[];
-    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(attn_smem_raw) + 1023) & ~(uintptr_t)1023);
-    unsigned char* q_smem = smem;                                   // kNQ tiles
-    unsigned char* kv_smem = smem + (size_t)kNQ * kTileBytes;       // kStages tiles
-    AttnSmem<NQ>* sm = reinterpret_cast<AttnSmem<NQ>*>(kv_smem + (size_t)kStages * kTileBytes);
-
-    pdl_wait();                // inputs may come from the kernel launched just before (gather / hybrid-cache update)
-    pdl_launch_dependents();   // a dependent kernel (the split merge) may start launching; it waits for this grid
-
-    // a CTA of this grid (or an earlier kernel sharing the workspace) has already given up: do nothing
-    __shared__ int skip_cta;
-    if (threadIdx.x == 0) skip_cta = (args.status != nullptr && *reinterpret_cast<volatile int*>(&args.status->code) != 0) ? 1 : 0;
-    __syncthreads();
-    if (skip_cta) return;
-
-    if (threadIdx.x == 0) DAF_STAMP(0);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-
+__device__ __forceinline__ void decode_work(const AttnArgs& args, CtaWork& a) {
     // ---- which item is this CTA's (uniform across the CTA)
     int seg_id = 0, item = (int)blockIdx.x;
     if (args.joint) {
         if (item < args.seg[1].n_items) seg_id = 1;
         else item -= args.seg[1].n_items;
     }
-#define DAF_SEG(field) (seg_id ? args.seg[1].field : args.seg[0].field)
-    struct { int n_q, n_kv, G, Gp, Tt, n_tb, causal_off; const int32_t* q_pos; float scale_log2; } a;
     a.n_q = DAF_SEG(n_q); a.n_kv = DAF_SEG(n_kv); a.G = DAF_SEG(G); a.Gp = DAF_SEG(Gp); a.Tt = DAF_SEG(Tt);
     a.n_tb = DAF_SEG(n_tb); a.causal_off = DAF_SEG(causal_off); a.q_pos = DAF_SEG(q_pos); a.scale_log2 = DAF_SEG(scale_log2);
-    const CUtensorMap* tmap_q = seg_id ? &tmap_q1 : &tmap_q0;
-    const CUtensorMap* tmap_k = seg_id ? &tmap_k1 : &tmap_k0;
-    const CUtensorMap* tmap_v = seg_id ? &tmap_v1 : &tmap_v0;
-    DeviceStatus* const status = args.status;
 
     int hb, unit, j_begin, j_end, item_splits, tok_base;
     long long part_row0;      // this item's first row in the partial-result arrays, in tokens
@@ -187,13 +262,159 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
         const int rem = slot - chunk * g * (g + 1) / 2;
         unit = g * chunk + rem / (g + 1);
         const int range = rem % (g + 1);
-        const int n_tiles = min(kNQ * (unit + 1), a.n_tb);
+        const int n_tiles = min(NQ * (unit + 1), a.n_tb);
         j_begin = range * n_tiles / (g + 1);
         j_end = (range + 1) * n_tiles / (g + 1);
         item_splits = g + 1;
-        part_row0 = (long long)slot * (kNQ * kBlockM);
-        tok_base = unit * (kNQ * kBlockM);
+        part_row0 = (long long)slot * (NQ * kBlockM);
+        tok_base = unit * (NQ * kBlockM);
     }
+    a.seg_id = seg_id; a.hb = hb; a.unit = unit; a.j_begin = j_begin; a.j_end = j_end;
+    a.item_splits = item_splits; a.tok_base = tok_base; a.part_row0 = part_row0;
+}
+
+// Final step of a tile: the warp's 32 rows of O (fp32 in tensor memory at o_addr, this thread's row
+// unnormalised with running maximum m and sum l) leave as bf16 output rows, or -- for an item that
+// covers only part of the keys -- as fp32 partial rows with their log-sum-exp.
+__device__ __forceinline__ void write_rows(const AttnArgs& args, const CtaWork& a, int t0, bool has_keys, bool row_valid,
+                                           bool row_valid_tile, int tok, int head, int h0, unsigned char* stage,
+                                           uint32_t o_addr, int quad, int lane, float m, float l) {
+    const int seg_id = a.seg_id;
+    // the fields only the epilogue needs are picked here, not held in registers through the loop
+    struct { int n_q, Gp, Tt, Hq; __nv_bfloat16* out; long long out_row_stride; const int32_t* dst_rows;
+             float* lse; float* part_o; float* part_lse; } e;
+    e.n_q = a.n_q; e.Gp = a.Gp; e.Tt = a.Tt; e.Hq = DAF_SEG(Hq);
+    e.out = DAF_SEG(out); e.out_row_stride = DAF_SEG(out_row_stride); e.dst_rows = DAF_SEG(dst_rows);
+    e.lse = DAF_SEG(lse); e.part_o = DAF_SEG(part_o); e.part_lse = DAF_SEG(part_lse);
+    const float inv_l = l > 0.f ? 1.f / l : 0.f;
+    const float lse_val = l > 0.f ? m * DAF_SEG(scale) + logf(l) : -INFINITY;
+    // Rows leave through shared memory so that global stores are whole 256-byte runs: each
+    // thread parks its own row (16-byte chunks, XOR-swizzled against bank conflicts) in the
+    // part of the Q tile that belongs to its warp (Q is dead once the last MMA has completed),
+    // then the warp writes its 32 rows out, 16 lanes per row.
+    auto park = [&](int chunk, uint4 w) {
+        *reinterpret_cast<uint4*>(stage + lane * 256 + ((chunk ^ (lane & 7)) << 4)) = w;
+    };
+    // copy phase: lanes 0-15 take row rr, lanes 16-31 row rr+1, rr advancing by 2; the row's
+    // (token, head) pair is tracked incrementally instead of dividing in the loop
+    const int sub = lane >> 4, cidx = lane & 15;
+    const int r_first = quad * 32 + sub;
+    const int step_t = 2 / e.Gp, step_h = 2 % e.Gp;
+    const int n_rows_tile = e.Gp * e.Tt;
+    if (a.item_splits == 1) {
+        if (row_valid && e.lse != nullptr) e.lse[(size_t)head * e.n_q + tok] = lse_val;
+        if (has_keys) {
+#pragma unroll
+            for (int cchunk = 0; cchunk < 4; ++cchunk) {
+                uint32_t orr[32];
+                tmem_ld32(o_addr + (uint32_t)(cchunk * 32), orr);
+                tc_wait_ld();
+#pragma unroll
+                for (int v = 0; v < 4; ++v) {
+                    uint4 w;
+                    w.x = pack_bf16(__uint_as_float(orr[v * 8 + 0]) * inv_l, __uint_as_float(orr[v * 8 + 1]) * inv_l);
+                    w.y = pack_bf16(__uint_as_float(orr[v * 8 + 2]) * inv_l, __uint_as_float(orr[v * 8 + 3]) * inv_l);
+                    w.z = pack_bf16(__uint_as_float(orr[v * 8 + 4]) * inv_l, __uint_as_float(orr[v * 8 + 5]) * inv_l);
+                    w.w = pack_bf16(__uint_as_float(orr[v * 8 + 6]) * inv_l, __uint_as_float(orr[v * 8 + 7]) * inv_l);
+                    park(cchunk * 4 + v, w);
+                }
+            }
+            __syncwarp();
+            int tok_r = t0 + r_first / e.Gp, head_off = r_first % e.Gp;
+#pragma unroll 4
+            for (int i = 0; i < 16; ++i) {
+                const int rr = 2 * i + sub;
+                if (quad * 32 + rr < n_rows_tile && tok_r < e.n_q) {
+                    const long long drow = e.dst_rows ? (long long)e.dst_rows[tok_r] : (long long)tok_r;
+                    const uint4 w = *reinterpret_cast<const uint4*>(stage + rr * 256 + ((cidx ^ (rr & 7)) << 4));
+                    reinterpret_cast<uint4*>(e.out + drow * e.out_row_stride + (long long)(h0 + head_off) * kD)[cidx] = w;
+                }
+                head_off += step_h; tok_r += step_t;
+                if (head_off >= e.Gp) { head_off -= e.Gp; ++tok_r; }
+            }
+        }
+    } else {
+        const long long prow0 = a.part_row0 - a.tok_base;
+        if (row_valid) e.part_lse[(prow0 + tok) * e.Hq + head] = lse_val;
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {   // 64 fp32 columns (256 bytes per row) at a time
+            if (has_keys) {
+#pragma unroll
+                for (int cc = 0; cc < 2; ++cc) {
+                    uint32_t orr[32];
+                    tmem_ld32(o_addr + (uint32_t)((half * 2 + cc) * 32), orr);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int v = 0; v < 8; ++v) {
+                        uint4 w;
+                        w.x = __float_as_uint(__uint_as_float(orr[v * 4 + 0]) * inv_l);
+                        w.y = __float_as_uint(__uint_as_float(orr[v * 4 + 1]) * inv_l);
+                        w.z = __float_as_uint(__uint_as_float(orr[v * 4 + 2]) * inv_l);
+                        w.w = __float_as_uint(__uint_as_float(orr[v * 4 + 3]) * inv_l);
+                        park(cc * 8 + v, w);
+                    }
+                }
+            } else {
+#pragma unroll
+                for (int v = 0; v < 16; ++v) park(v, make_uint4(0u, 0u, 0u, 0u));
+            }
+            __syncwarp();
+            int tok_r = t0 + r_first / e.Gp, head_off = r_first % e.Gp;
+#pragma unroll 4
+            for (int i = 0; i < 16; ++i) {
+                const int rr = 2 * i + sub;
+                if (row_valid_tile && quad * 32 + rr < n_rows_tile && tok_r < e.n_q) {
+                    const uint4 w = *reinterpret_cast<const uint4*>(stage + rr * 256 + ((cidx ^ (rr & 7)) << 4));
+                    float* prow = e.part_o + ((prow0 + tok_r) * e.Hq + (h0 + head_off)) * kD + half * 64;
+                    reinterpret_cast<uint4*>(prow)[cidx] = w;
+                }
+                head_off += step_h; tok_r += step_t;
+                if (head_off >= e.Gp) { head_off -= e.Gp; ++tok_r; }
+            }
+            __syncwarp();
+        }
+    }
+}
+
+template <int NQ>
+__global__ void __launch_bounds__(AttnCfg<NQ>::kThreads, AttnCfg<NQ>::kCtasPerSM)
+attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_constant__ CUtensorMap tmap_k0,
+                const __grid_constant__ CUtensorMap tmap_v0, const __grid_constant__ CUtensorMap tmap_q1,
+                const __grid_constant__ CUtensorMap tmap_k1, const __grid_constant__ CUtensorMap tmap_v1,
+                const AttnArgs args) {
+    constexpr int kNQ = NQ;
+    constexpr int kStages = AttnCfg<NQ>::kStages;
+    constexpr int kTmaWarp = AttnCfg<NQ>::kTmaWarp;
+    constexpr int kMmaWarp = AttnCfg<NQ>::kMmaWarp;
+    constexpr int kTmemCols = AttnCfg<NQ>::kTmemCols;
+    extern __shared__ unsigned char attn_smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(attn_smem_raw) + 1023) & ~(uintptr_t)1023);
+    unsigned char* q_smem = smem;                                   // kNQ tiles
+    unsigned char* kv_smem = smem + (size_t)kNQ * kTileBytes;       // kStages tiles
+    AttnSmem<NQ>* sm = reinterpret_cast<AttnSmem<NQ>*>(kv_smem + (size_t)kStages * kTileBytes);
+
+    pdl_wait();                // inputs may come from the kernel launched just before (gather / hybrid-cache update)
+    pdl_launch_dependents();   // a dependent kernel (the split merge) may start launching; it waits for this grid
+
+    // a CTA of this grid (or an earlier kernel sharing the workspace) has already given up: do nothing
+    __shared__ int skip_cta;
+    if (threadIdx.x == 0) skip_cta = (args.status != nullptr && *reinterpret_cast<volatile int*>(&args.status->code) != 0) ? 1 : 0;
+    __syncthreads();
+    if (skip_cta) return;
+
+    if (threadIdx.x == 0) DAF_STAMP(0);
+    DAF_KT_BEGIN(0);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    // ---- which item is this CTA's (uniform across the CTA)
+    CtaWork a;
+    decode_work<NQ>(args, a);
+    const int seg_id = a.seg_id, hb = a.hb, unit = a.unit, j_begin = a.j_begin, j_end = a.j_end;
+    const int item_splits = a.item_splits;
+    const CUtensorMap* tmap_q = seg_id ? &tmap_q1 : &tmap_q0;
+    const CUtensorMap* tmap_k = seg_id ? &tmap_k1 : &tmap_k0;
+    const CUtensorMap* tmap_v = seg_id ? &tmap_v1 : &tmap_v0;
+    DeviceStatus* const status = args.status;
     const int h0 = hb * a.Gp;
     const int g_kv = h0 / a.G;
 
@@ -364,80 +585,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
             if (!ok) break;
             tc_fence_after();
             if (threadIdx.x == 0 && j == 0) DAF_STAMP(2);
-            // logits of this row: 128 fp32 values, fetched in two halves so that the row maximum of the
-            // first half is computed while the second half is still on its way from tensor memory
-            uint32_t sr[4][32];
-            tmem_ld32(s_addr, sr[0]);
-            tmem_ld32(s_addr + 32u, sr[1]);
-            tc_wait_ld();
-            tmem_ld32(s_addr + 64u, sr[2]);
-            tmem_ld32(s_addr + 96u, sr[3]);
-            const int key0 = (j_begin + j) * kBlockN;
-            const bool need_mask = key0 + kBlockN - 1 > limit;
-            float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                if (half == 1) tc_wait_ld();
-                if (need_mask) {
-#pragma unroll
-                    for (int cchunk = 2 * half; cchunk < 2 * half + 2; ++cchunk)
-#pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            if (key0 + cchunk * 32 + i > limit) sr[cchunk][i] = 0xFF800000u;  // -inf
-                }
-#pragma unroll
-                for (int cchunk = 2 * half; cchunk < 2 * half + 2; ++cchunk)
-#pragma unroll
-                    for (int i = 0; i < 32; i += 8) {
-                        // four independent chains of 3-input maxima
-                        mx[0] = fmax3(mx[0], __uint_as_float(sr[cchunk][i + 0]), __uint_as_float(sr[cchunk][i + 1]));
-                        mx[1] = fmax3(mx[1], __uint_as_float(sr[cchunk][i + 2]), __uint_as_float(sr[cchunk][i + 3]));
-                        mx[2] = fmax3(mx[2], __uint_as_float(sr[cchunk][i + 4]), __uint_as_float(sr[cchunk][i + 5]));
-                        mx[3] = fmax3(mx[3], __uint_as_float(sr[cchunk][i + 6]), __uint_as_float(sr[cchunk][i + 7]));
-                    }
-            }
-            const float tmax = fmax3(mx[0], mx[1], fmaxf(mx[2], mx[3]));
-            float m_new = fmaxf(m, tmax);
-            // keep a slightly stale maximum: rescaling O is skipped while the growth stays below 2^8
-            if (m != -INFINITY && (m_new - m) * c <= kRescaleThreshold) m_new = m;
-            const float m_used = (m_new == -INFINITY) ? 0.f : m_new;
-            const float alpha = (m == -INFINITY) ? 1.f : fast_exp2((m - m_new) * c);
-            const float mc = m_used * c;
-            // p = 2^(s*c - m*c): packed two-wide FMA and adds, exponentials on the special-function unit
-            const uint64_t c2 = pack_f32x2(c, c), nmc2 = pack_f32x2(-mc, -mc);
-            uint64_t acc2[4] = {0ull, 0ull, 0ull, 0ull};
-            uint32_t pr[2][32];
-#pragma unroll
-            for (int cchunk = 0; cchunk < 4; ++cchunk)
-#pragma unroll
-                for (int i = 0; i < 32; i += 2) {
-                    const uint64_t x2 = ffma2(pack_f32x2(__uint_as_float(sr[cchunk][i]), __uint_as_float(sr[cchunk][i + 1])), c2, nmc2);
-                    const float p0 = fast_exp2(f32x2_lo(x2));
-                    const float p1 = fast_exp2(f32x2_hi(x2));
-                    acc2[(i >> 1) & 3] = fadd2(acc2[(i >> 1) & 3], pack_f32x2(p0, p1));
-                    pr[cchunk >> 1][(cchunk & 1) * 16 + (i >> 1)] = pack_bf16(p0, p1);
-                }
-            const uint64_t acc01 = fadd2(fadd2(acc2[0], acc2[1]), fadd2(acc2[2], acc2[3]));
-            const float rowsum = f32x2_lo(acc01) + f32x2_hi(acc01);
-            l = l * alpha + rowsum;
-            m = m_new;
-            // P (bf16, two keys per 32-bit column) overlays the first 64 columns of S
-            tmem_st32(s_addr, pr[0]);
-            tmem_st32(s_addr + 32u, pr[1]);
-            if (j > 0 && __any_sync(0xFFFFFFFFu, alpha != 1.f)) {
-                // the commit that released S_j also covers the previous P V product, so O is quiescent here
-#pragma unroll
-                for (int cchunk = 0; cchunk < 4; ++cchunk) {
-                    uint32_t orr[32];
-                    tmem_ld32(o_addr + (uint32_t)(cchunk * 32), orr);
-                    tc_wait_ld();
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * alpha);
-                    tmem_st32(o_addr + (uint32_t)(cchunk * 32), orr);
-                }
-            }
-            tc_wait_st();
-            tc_fence_before();
+            softmax_step(s_addr, o_addr, (j_begin + j) * kBlockN, limit, c, j == 0, m, l);
             mbar_arrive(&sm->p_full[q]);
         }
         if (threadIdx.x == 0) DAF_STAMP(3);
@@ -448,101 +596,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
         }
         if (ok) {
             tc_fence_after();
-            // the fields only the epilogue needs are picked here, not held in registers through the loop
-            struct { int n_q, Gp, Tt, Hq; __nv_bfloat16* out; long long out_row_stride; const int32_t* dst_rows;
-                     float* lse; float* part_o; float* part_lse; } e;
-            e.n_q = a.n_q; e.Gp = a.Gp; e.Tt = a.Tt; e.Hq = DAF_SEG(Hq);
-            e.out = DAF_SEG(out); e.out_row_stride = DAF_SEG(out_row_stride); e.dst_rows = DAF_SEG(dst_rows);
-            e.lse = DAF_SEG(lse); e.part_o = DAF_SEG(part_o); e.part_lse = DAF_SEG(part_lse);
-            const float inv_l = l > 0.f ? 1.f / l : 0.f;
-            const float lse_val = l > 0.f ? m * DAF_SEG(scale) + logf(l) : -INFINITY;
-            // Rows leave through shared memory so that global stores are whole 256-byte runs: each
-            // thread parks its own row (16-byte chunks, XOR-swizzled against bank conflicts) in the
-            // part of the Q tile that belongs to its warp (Q is dead once the last MMA has completed),
-            // then the warp writes its 32 rows out, 16 lanes per row.
-            unsigned char* stage = q_smem + (size_t)q * kTileBytes + (size_t)quad * 32 * 256;
-            auto park = [&](int chunk, uint4 w) {
-                *reinterpret_cast<uint4*>(stage + lane * 256 + ((chunk ^ (lane & 7)) << 4)) = w;
-            };
-            // copy phase: lanes 0-15 take row rr, lanes 16-31 row rr+1, rr advancing by 2; the row's
-            // (token, head) pair is tracked incrementally instead of dividing in the loop
-            const int sub = lane >> 4, cidx = lane & 15;
-            const int r_first = quad * 32 + sub;
-            const int step_t = 2 / e.Gp, step_h = 2 % e.Gp;
-            const int n_rows_tile = e.Gp * e.Tt;
-            if (item_splits == 1) {
-                if (row_valid && e.lse != nullptr) e.lse[(size_t)head * e.n_q + tok] = lse_val;
-                if (n_j[q] > 0) {
-#pragma unroll
-                    for (int cchunk = 0; cchunk < 4; ++cchunk) {
-                        uint32_t orr[32];
-                        tmem_ld32(o_addr + (uint32_t)(cchunk * 32), orr);
-                        tc_wait_ld();
-#pragma unroll
-                        for (int v = 0; v < 4; ++v) {
-                            uint4 w;
-                            w.x = pack_bf16(__uint_as_float(orr[v * 8 + 0]) * inv_l, __uint_as_float(orr[v * 8 + 1]) * inv_l);
-                            w.y = pack_bf16(__uint_as_float(orr[v * 8 + 2]) * inv_l, __uint_as_float(orr[v * 8 + 3]) * inv_l);
-                            w.z = pack_bf16(__uint_as_float(orr[v * 8 + 4]) * inv_l, __uint_as_float(orr[v * 8 + 5]) * inv_l);
-                            w.w = pack_bf16(__uint_as_float(orr[v * 8 + 6]) * inv_l, __uint_as_float(orr[v * 8 + 7]) * inv_l);
-                            park(cchunk * 4 + v, w);
-                        }
-                    }
-                    __syncwarp();
-                    int tok_r = t0[q] + r_first / e.Gp, head_off = r_first % e.Gp;
-#pragma unroll 4
-                    for (int i = 0; i < 16; ++i) {
-                        const int rr = 2 * i + sub;
-                        if (quad * 32 + rr < n_rows_tile && tok_r < e.n_q) {
-                            const long long drow = e.dst_rows ? (long long)e.dst_rows[tok_r] : (long long)tok_r;
-                            const uint4 w = *reinterpret_cast<const uint4*>(stage + rr * 256 + ((cidx ^ (rr & 7)) << 4));
-                            reinterpret_cast<uint4*>(e.out + drow * e.out_row_stride + (long long)(h0 + head_off) * kD)[cidx] = w;
-                        }
-                        head_off += step_h; tok_r += step_t;
-                        if (head_off >= e.Gp) { head_off -= e.Gp; ++tok_r; }
-                    }
-                }
-            } else {
-                const long long prow0 = part_row0 - tok_base;
-                if (row_valid) e.part_lse[(prow0 + tok) * e.Hq + head] = lse_val;
-#pragma unroll
-                for (int half = 0; half < 2; ++half) {   // 64 fp32 columns (256 bytes per row) at a time
-                    if (n_j[q] > 0) {
-#pragma unroll
-                        for (int cc = 0; cc < 2; ++cc) {
-                            uint32_t orr[32];
-                            tmem_ld32(o_addr + (uint32_t)((half * 2 + cc) * 32), orr);
-                            tc_wait_ld();
-#pragma unroll
-                            for (int v = 0; v < 8; ++v) {
-                                uint4 w;
-                                w.x = __float_as_uint(__uint_as_float(orr[v * 4 + 0]) * inv_l);
-                                w.y = __float_as_uint(__uint_as_float(orr[v * 4 + 1]) * inv_l);
-                                w.z = __float_as_uint(__uint_as_float(orr[v * 4 + 2]) * inv_l);
-                                w.w = __float_as_uint(__uint_as_float(orr[v * 4 + 3]) * inv_l);
-                                park(cc * 8 + v, w);
-                            }
-                        }
-                    } else {
-#pragma unroll
-                        for (int v = 0; v < 16; ++v) park(v, make_uint4(0u, 0u, 0u, 0u));
-                    }
-                    __syncwarp();
-                    int tok_r = t0[q] + r_first / e.Gp, head_off = r_first % e.Gp;
-#pragma unroll 4
-                    for (int i = 0; i < 16; ++i) {
-                        const int rr = 2 * i + sub;
-                        if (row_valid_tile && quad * 32 + rr < n_rows_tile && tok_r < e.n_q) {
-                            const uint4 w = *reinterpret_cast<const uint4*>(stage + rr * 256 + ((cidx ^ (rr & 7)) << 4));
-                            float* prow = e.part_o + ((prow0 + tok_r) * e.Hq + (h0 + head_off)) * kD + half * 64;
-                            reinterpret_cast<uint4*>(prow)[cidx] = w;
-                        }
-                        head_off += step_h; tok_r += step_t;
-                        if (head_off >= e.Gp) { head_off -= e.Gp; ++tok_r; }
-                    }
-                    __syncwarp();
-                }
-            }
+            write_rows(args, a, t0[q], n_j[q] > 0, row_valid, row_valid_tile, tok, head, h0,
+                       q_smem + (size_t)q * kTileBytes + (size_t)quad * 32 * 256, o_addr, quad, lane, m, l);
         }
     }
 
@@ -553,7 +608,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
         tc_fence_after();
         tmem_dealloc(tmem, kTmemCols);
     }
-#undef DAF_SEG
+    DAF_KT_END(0);
 #ifdef DAF_TRACE
     if (threadIdx.x == 0) {
         DAF_STAMP(5);
@@ -568,6 +623,256 @@ extern "C" int daf_dbg_read_trace(void* host, size_t bytes) {
     return (int)cudaMemcpyFromSymbol(host, g_trace, bytes < sizeof(g_trace) ? bytes : sizeof(g_trace));
 }
 #endif
+
+// ------------------------------------------------------------------------------------------------
+// One query tile per CTA, two CTAs per SM, for problems with few tiles.
+//
+// With a single tile a CTA has nothing to overlap a key tile's softmax with, and the chain
+// S = Q K^T -> softmax -> O += P V -> next S runs at the sum of its latencies.  Here the keys go
+// through in sub-steps of 64 and S is double-buffered (two 64-column halves of the same 128 tensor-
+// memory columns): the logits of sub-step t + 1 are computed while the softmax of sub-step t
+// runs, so the softmax warps find their next input ready.  The products O += P_t V_t are issued
+// as each P_t arrives; a row may only be rescaled, and P_{t+1} only be handed over, once the
+// product before it has completed (pv_done).
+constexpr int kSubN = 64;                               // keys per sub-step
+constexpr int kSubBytes = kSubN * kD * 2;               // 16 KB: K or V of one sub-step, two 64-column halves
+constexpr int kSubHalfBytes = kSubBytes / 2;
+constexpr int kSmallThreads = 192;                      // warps 0-3 softmax, warp 4 TMA, warp 5 MMA
+constexpr int kSmallTmemCols = 256;                     // S (two halves of 64) and O (128)
+
+struct SmallSmem {
+    uint64_t q_full;
+    uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2];
+    uint64_t s_full[2], p_full[2];
+    uint64_t pv_done;
+    uint32_t tmem_base;
+    int abort_flag;
+};
+constexpr size_t kSmallSmemBytes = 1024 + 3 * (size_t)kTileBytes + sizeof(SmallSmem);
+
+__global__ void __launch_bounds__(kSmallThreads, 2)
+attn_small_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_constant__ CUtensorMap tmap_k0,
+                  const __grid_constant__ CUtensorMap tmap_v0, const __grid_constant__ CUtensorMap tmap_q1,
+                  const __grid_constant__ CUtensorMap tmap_k1, const __grid_constant__ CUtensorMap tmap_v1,
+                  const AttnArgs args) {
+    extern __shared__ unsigned char attn_smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(attn_smem_raw) + 1023) & ~(uintptr_t)1023);
+    unsigned char* q_smem = smem;                                 // 32 KB
+    unsigned char* k_smem = smem + kTileBytes;                    // two sub-step slots
+    unsigned char* v_smem = smem + 2 * (size_t)kTileBytes;        // two sub-step slots
+    SmallSmem* sm = reinterpret_cast<SmallSmem*>(smem + 3 * (size_t)kTileBytes);
+
+    pdl_wait();                // inputs may come from the kernel launched just before (gather / hybrid-cache update)
+    pdl_launch_dependents();   // a dependent kernel (the split merge) may start launching; it waits for this grid
+
+    // a CTA of this grid (or an earlier kernel sharing the workspace) has already given up: do nothing
+    __shared__ int skip_cta;
+    if (threadIdx.x == 0) skip_cta = (args.status != nullptr && *reinterpret_cast<volatile int*>(&args.status->code) != 0) ? 1 : 0;
+    __syncthreads();
+    if (skip_cta) return;
+
+    if (threadIdx.x == 0) DAF_STAMP(0);
+    DAF_KT_BEGIN(0);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    CtaWork a;
+    decode_work<1>(args, a);
+    const int seg_id = a.seg_id;
+    const CUtensorMap* tmap_q = seg_id ? &tmap_q1 : &tmap_q0;
+    const CUtensorMap* tmap_k = seg_id ? &tmap_k1 : &tmap_k0;
+    const CUtensorMap* tmap_v = seg_id ? &tmap_v1 : &tmap_v0;
+    DeviceStatus* const status = args.status;
+    const int h0 = a.hb * a.Gp;
+    const int g_kv = h0 / a.G;
+    const int t0 = a.unit * a.Tt;
+    // sub-steps of this item: the keys of its range that the tile's last token may see
+    const int key_begin = a.j_begin * kBlockN;
+    int n_t = 0;
+    if (a.unit < a.n_tb) {
+        const int max_tok = min(a.n_q, t0 + a.Tt) - 1;
+        const long long last_key = a.q_pos ? (long long)__ldg(a.q_pos + max_tok) : (long long)max_tok + a.causal_off;
+        long long hi = min((long long)a.n_kv, last_key + 1);
+        hi = min(hi, (long long)a.j_end * kBlockN);
+        if (hi > key_begin) n_t = (int)((hi - key_begin + kSubN - 1) / kSubN);
+    }
+
+    if (threadIdx.x == 0) {
+        mbar_init(&sm->q_full, 1);
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(&sm->k_full[s], 1); mbar_init(&sm->k_empty[s], 1);
+            mbar_init(&sm->v_full[s], 1); mbar_init(&sm->v_empty[s], 1);
+            mbar_init(&sm->s_full[s], 1); mbar_init(&sm->p_full[s], 128);
+        }
+        mbar_init(&sm->pv_done, 1);
+        sm->abort_flag = 0;
+        mbar_fence_init();
+    }
+    if (warp == 5) {
+        tmem_alloc(&sm->tmem_base, kSmallTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = sm->tmem_base;
+    volatile int* abort_flag = &sm->abort_flag;
+    if (threadIdx.x == 0) DAF_STAMP(1);
+
+    if (warp == 4) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0 && n_t > 0) {
+            tma_prefetch_desc(tmap_q);
+            tma_prefetch_desc(tmap_k);
+            tma_prefetch_desc(tmap_v);
+            mbar_arrive_expect_tx(&sm->q_full, 2u * 128u * (uint32_t)(a.Gp * a.Tt));
+            tma_load_3d(q_smem, tmap_q, &sm->q_full, 0, h0, t0);
+            tma_load_3d(q_smem + kHalfBytes, tmap_q, &sm->q_full, 64, h0, t0);
+            bool ok = true;
+            for (int t = 0; t < n_t && ok; ++t) {
+                const int slot = t & 1;
+                const uint32_t round = (uint32_t)(t >> 1);
+                const int key0 = key_begin + t * kSubN;
+                for (int kv = 0; kv < 2 && ok; ++kv) {
+                    uint64_t* empty = kv == 0 ? &sm->k_empty[slot] : &sm->v_empty[slot];
+                    uint64_t* full = kv == 0 ? &sm->k_full[slot] : &sm->v_full[slot];
+                    if (round > 0) ok = mbar_wait(empty, (round - 1) & 1u, abort_flag, status, 10 + 2 * kv + slot);
+                    if (!ok) break;
+                    unsigned char* dst = (kv == 0 ? k_smem : v_smem) + (size_t)slot * kSubBytes;
+                    const CUtensorMap* tm = kv == 0 ? tmap_k : tmap_v;
+                    mbar_arrive_expect_tx(full, (uint32_t)kSubBytes);
+                    tma_load_3d(dst, tm, full, 0, g_kv, key0);
+                    tma_load_3d(dst + kSubHalfBytes, tm, full, 64, g_kv, key0);
+                }
+            }
+            if (!ok) {
+                // give loads already in flight a bounded chance to land before the CTA retires
+                for (int s = 0; s < 2; ++s) {
+                    for (int i = 0; i < 4096 && !mbar_try_wait(&sm->k_full[s], 0) && !mbar_try_wait(&sm->k_full[s], 1); ++i) {}
+                    for (int i = 0; i < 4096 && !mbar_try_wait(&sm->v_full[s], 0) && !mbar_try_wait(&sm->v_full[s], 1); ++i) {}
+                }
+            }
+        }
+    } else if (warp == 5) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0 && n_t > 0) {
+            constexpr uint32_t idesc_qk = make_idesc_bf16(kBlockM, kSubN, 0);
+            constexpr uint32_t idesc_pv = make_idesc_bf16(kBlockM, kD, 1);
+            const uint32_t qa = smem_u32(q_smem);
+            // S_b = Q K_t^T for the 64 keys in K slot b (= t & 1)
+            auto issue_qk = [&](int b) {
+                const uint32_t ka = smem_u32(k_smem + (size_t)b * kSubBytes);
+#pragma unroll
+                for (int kk = 0; kk < kD / 16; ++kk) {
+                    const uint32_t qoff = (uint32_t)((kk & 3) * 32 + (kk >> 2) * kHalfBytes);
+                    const uint32_t koff = (uint32_t)((kk & 3) * 32 + (kk >> 2) * kSubHalfBytes);
+                    tc_mma_ss(tmem + (uint32_t)(b * kSubN), make_smem_desc(qa + qoff, 16, 1024), make_smem_desc(ka + koff, 16, 1024),
+                              idesc_qk, kk > 0 ? 1u : 0u);
+                }
+            };
+            // O (+)= P_b V_t for the 64 keys in V slot b; P (bf16) sits in the first 32 columns of S_b
+            auto issue_pv = [&](int b, bool first) {
+                const uint32_t va = smem_u32(v_smem + (size_t)b * kSubBytes);
+#pragma unroll
+                for (int kk = 0; kk < kSubN / 16; ++kk)
+                    tc_mma_ts(tmem + (uint32_t)kBlockN, tmem + (uint32_t)(b * kSubN + kk * 8),
+                              make_smem_desc(va + (uint32_t)kk * 2048u, kSubHalfBytes, 1024), idesc_pv, (first && kk == 0) ? 0u : 1u);
+            };
+            bool ok = mbar_wait(&sm->q_full, 0, abort_flag, status, 20);
+            for (int t = 0; t < 2 && t < n_t && ok; ++t) {   // the first two S tiles
+                ok = mbar_wait(&sm->k_full[t], 0, abort_flag, status, 30 + t);
+                if (!ok) break;
+                tc_fence_after();
+                issue_qk(t);
+                tc_commit(&sm->s_full[t]);
+                tc_commit(&sm->k_empty[t]);
+            }
+            for (int t = 0; t < n_t && ok; ++t) {
+                const int b = t & 1;
+                const uint32_t par = (uint32_t)((t >> 1) & 1);
+                ok = mbar_wait(&sm->v_full[b], par, abort_flag, status, 32 + b);
+                if (ok) ok = mbar_wait(&sm->p_full[b], par, abort_flag, status, 40 + b);
+                if (!ok) break;
+                tc_fence_after();
+                issue_pv(b, t == 0);
+                tc_commit(&sm->v_empty[b]);
+                tc_commit(&sm->pv_done);
+                if (t + 2 < n_t) {
+                    ok = mbar_wait(&sm->k_full[b], (uint32_t)(((t + 2) >> 1) & 1), abort_flag, status, 34 + b);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_qk(b);
+                    tc_commit(&sm->s_full[b]);
+                    tc_commit(&sm->k_empty[b]);
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ softmax + epilogue, one row per thread
+        const int quad = warp;
+        const int r = quad * 32 + lane;
+        const int tok = t0 + r / a.Gp;
+        const int head = h0 + r % a.Gp;
+        const bool row_valid_tile = (n_t > 0 || a.item_splits > 1) && (a.unit < a.n_tb);
+        const bool row_valid = (r < a.Gp * a.Tt) && (tok < a.n_q) && row_valid_tile;
+        const long long lim_ll = (a.q_pos && tok < a.n_q) ? (long long)__ldg(a.q_pos + tok) : (long long)tok + a.causal_off;
+        const int limit = row_valid ? (int)min(lim_ll, (long long)a.n_kv - 1) : -1;   // last visible key
+        const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+        const uint32_t s_addr = tmem + lane_addr;
+        const uint32_t o_addr = tmem + lane_addr + (uint32_t)kBlockN;
+        const float c = a.scale_log2;
+
+        float m = -INFINITY, l = 0.f;
+        bool ok = true;
+        for (int t = 0; t < n_t; ++t) {
+            const int b = t & 1;
+            ok = mbar_wait(&sm->s_full[b], (uint32_t)((t >> 1) & 1), abort_flag, status, 50 + b);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            if (threadIdx.x == 0 && t == 0) DAF_STAMP(2);
+            const float alpha = softmax_core<2>(s_addr + (uint32_t)(b * kSubN), key_begin + t * kSubN, limit, c, m, l);
+            if (t > 0) {
+                // O may be touched, and the next product be issued, only once the previous product has completed
+                ok = mbar_wait(&sm->pv_done, (uint32_t)((t - 1) & 1), abort_flag, status, 60);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) break;
+                tc_fence_after();
+                if (__any_sync(0xFFFFFFFFu, alpha != 1.f)) rescale_o(o_addr, alpha);
+            }
+            tc_wait_st();
+            tc_fence_before();
+            mbar_arrive(&sm->p_full[b]);
+        }
+        if (threadIdx.x == 0) DAF_STAMP(3);
+        // ---- epilogue
+        if (ok && n_t > 0) {
+            ok = mbar_wait(&sm->pv_done, (uint32_t)((n_t - 1) & 1), abort_flag, status, 61);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+        }
+        if (ok) {
+            tc_fence_after();
+            write_rows(args, a, t0, n_t > 0, row_valid, row_valid_tile, tok, head, h0, q_smem + (size_t)quad * 32 * 256, o_addr,
+                       quad, lane, m, l);
+        }
+    }
+
+    if (threadIdx.x == 0) DAF_STAMP(4);
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 5) {
+        tc_fence_after();
+        tmem_dealloc(tmem, kSmallTmemCols);
+    }
+    DAF_KT_END(0);
+#ifdef DAF_TRACE
+    if (threadIdx.x == 0) {
+        DAF_STAMP(5);
+        const unsigned cta = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
+        if (cta < 65536u) g_trace[8 * cta + 6] = (unsigned long long)n_t;
+    }
+#endif
+}
+
+#undef DAF_SEG
 
 // Merge of partial results: one warp per (token, head) row.  A launch merges the rows of up to two
 // problems (those of s0 first).  A row's partials sit `stride` rows apart; how many there are is the
@@ -584,7 +889,9 @@ struct CombineSeg {
 
 __global__ void __launch_bounds__(256)
 attn_combine_kernel(const CombineSeg s0, const CombineSeg s1) {
+    DAF_KT_BEGIN(2);
     pdl_wait();                // partial results come from the attention kernel launched just before
+    DAF_KT_BEGIN(3);
     int row = blockIdx.x * 8 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     const bool second = row >= s0.n_rows;
@@ -644,6 +951,7 @@ attn_combine_kernel(const CombineSeg s0, const CombineSeg s1) {
     reinterpret_cast<uint2*>(DAF_CS(out) + drow * DAF_CS(out_row_stride) + (long long)head * kD)[lane] = w2;
     float* lse = DAF_CS(lse);
     if (lse != nullptr && lane == 0) lse[(size_t)head * n_q + tok] = wsum > 0.f ? mx + logf(wsum) : -INFINITY;
+    DAF_KT_END(2);
 #undef DAF_CS
 }
 
@@ -691,6 +999,8 @@ static int set_kernel_attributes() {
         cudaError_t e = cudaFuncSetAttribute(attn_fwd_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem_bytes<1>());
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(attn_fwd_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem_bytes<2>());
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(attn_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmallSmemBytes);
         if (e != cudaSuccess) { set_cuda_error(e); return DAF_ERR_CUDA; }
         attr_done[dev] = true;
     }
@@ -700,6 +1010,7 @@ static int set_kernel_attributes() {
 // How a single problem is cut into CTAs.  Splitting the KV axis is only used for the
 // question rows, where there are few query tiles and a long KV axis.
 static int g_force_nq = 0;        // 0: choose by problem size (the tuning builds can pin a shape)
+static int g_small = 1;            // one-tile launches use the kernel with 64-key sub-steps
 static float g_joint_factor = 1.0f;   // longest item of a joint launch, as a fraction of the mean load of a CTA slot
 
 AttnPlan plan_attention(int n_q, int n_kv, int Hq, int G, int causal_off, bool pack_group, bool allow_split) {
@@ -799,6 +1110,7 @@ JointPlan plan_joint(int k, int L_q, int L_d, int Hq, int G) {
 #ifdef DAF_TRACE
 extern "C" void daf_dbg_force_nq(int nq) { g_force_nq = nq; }
 extern "C" void daf_dbg_joint_factor(float f) { g_joint_factor = f; }
+extern "C" void daf_dbg_small(int on) { g_small = on; }
 #endif
 
 static void fill_problem(SegArgs* s, int n_q, int n_kv, int Hq, int G, int Gp, int causal_off, const int32_t* q_pos,
@@ -849,8 +1161,10 @@ int launch_attention(const void* q, const void* k, const void* v, int n_q, int n
 
     CUtensorMap tq, tk, tv;
     if (int rc = make_tmap(&tq, q, n_q, Hq, pl.Gp, pl.Tt)) return rc;
-    if (int rc = make_tmap(&tk, k, n_kv, Hkv, 1, kBlockN)) return rc;
-    if (int rc = make_tmap(&tv, v, n_kv, Hkv, 1, kBlockN)) return rc;
+    const bool small = pl.nq == 1 && g_small;      // one tile per CTA: keys go through in sub-steps of 64
+    const int kv_box = small ? kSubN : kBlockN;
+    if (int rc = make_tmap(&tk, k, n_kv, Hkv, 1, kv_box)) return rc;
+    if (int rc = make_tmap(&tv, v, n_kv, Hkv, 1, kv_box)) return rc;
     if (int rc = set_kernel_attributes()) return rc;
 
     AttnArgs a;
@@ -870,6 +1184,7 @@ int launch_attention(const void* q, const void* k, const void* v, int n_q, int n
     dim3 grid((unsigned)pl.head_blocks, (unsigned)pl.pairs, (unsigned)pl.n_splits);
     cudaError_t e;
     if (pl.nq == 2) e = launch_kernel(attn_fwd_kernel<2>, grid, dim3(AttnCfg<2>::kThreads), attn_smem_bytes<2>(), stream, after_kernel, tq, tk, tv, tq, tk, tv, a);
+    else if (small) e = launch_kernel(attn_small_kernel, grid, dim3(kSmallThreads), kSmallSmemBytes, stream, after_kernel, tq, tk, tv, tq, tk, tv, a);
     else e = launch_kernel(attn_fwd_kernel<1>, grid, dim3(AttnCfg<1>::kThreads), attn_smem_bytes<1>(), stream, after_kernel, tq, tk, tv, tq, tk, tv, a);
     count_launch();
     if (e != cudaSuccess) { set_cuda_error(e); return DAF_ERR_CUDA; }
@@ -896,11 +1211,13 @@ int launch_attention_joint(const void* q_imp, const void* k_imp, const void* v_i
 
     CUtensorMap tq0, tk0, tv0, tq1, tk1, tv1;
     if (int rc = make_tmap(&tq0, q_imp, k, Hq, 1, kBlockM)) return rc;
-    if (int rc = make_tmap(&tk0, k_imp, k, Hkv, 1, kBlockN)) return rc;
-    if (int rc = make_tmap(&tv0, v_imp, k, Hkv, 1, kBlockN)) return rc;
+    const bool small = jp.nq == 1 && g_small;
+    const int kv_box = small ? kSubN : kBlockN;
+    if (int rc = make_tmap(&tk0, k_imp, k, Hkv, 1, kv_box)) return rc;
+    if (int rc = make_tmap(&tv0, v_imp, k, Hkv, 1, kv_box)) return rc;
     if (int rc = make_tmap(&tq1, q_question, L_q, Hq, jp.Gp_q, jp.Tt_q)) return rc;
-    if (int rc = make_tmap(&tk1, kv_k, N, Hkv, 1, kBlockN)) return rc;
-    if (int rc = make_tmap(&tv1, kv_v, N, Hkv, 1, kBlockN)) return rc;
+    if (int rc = make_tmap(&tk1, kv_k, N, Hkv, 1, kv_box)) return rc;
+    if (int rc = make_tmap(&tv1, kv_v, N, Hkv, 1, kv_box)) return rc;
     if (int rc = set_kernel_attributes()) return rc;
 
     AttnArgs a;
@@ -928,10 +1245,18 @@ int launch_attention_joint(const void* q_imp, const void* k_imp, const void* v_i
     a.joint = 1;
     a.status = status;
 
-    dim3 grid((unsigned)(jp.items_q + jp.items_i), 1, 1);
+    const int items = jp.items_q + jp.items_i;
     cudaError_t e;
-    if (jp.nq == 2) e = launch_kernel(attn_fwd_kernel<2>, grid, dim3(AttnCfg<2>::kThreads), attn_smem_bytes<2>(), stream, after_kernel, tq0, tk0, tv0, tq1, tk1, tv1, a);
-    else e = launch_kernel(attn_fwd_kernel<1>, grid, dim3(AttnCfg<1>::kThreads), attn_smem_bytes<1>(), stream, after_kernel, tq0, tk0, tv0, tq1, tk1, tv1, a);
+    if (jp.nq == 2) {
+        e = launch_kernel(attn_fwd_kernel<2>, dim3((unsigned)items), dim3(AttnCfg<2>::kThreads), attn_smem_bytes<2>(), stream,
+                          after_kernel, tq0, tk0, tv0, tq1, tk1, tv1, a);
+    } else if (small) {
+        e = launch_kernel(attn_small_kernel, dim3((unsigned)items), dim3(kSmallThreads), kSmallSmemBytes, stream,
+                          after_kernel, tq0, tk0, tv0, tq1, tk1, tv1, a);
+    } else {
+        e = launch_kernel(attn_fwd_kernel<1>, dim3((unsigned)items), dim3(AttnCfg<1>::kThreads), attn_smem_bytes<1>(), stream,
+                          after_kernel, tq0, tk0, tv0, tq1, tk1, tv1, a);
+    }
     count_launch();
     if (e != cudaSuccess) { set_cuda_error(e); return DAF_ERR_CUDA; }
     if (int rc = check_launch()) return rc;

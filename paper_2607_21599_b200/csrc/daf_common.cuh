@@ -140,6 +140,24 @@ __device__ __forceinline__ unsigned long long global_ns() {
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
+#ifdef DAF_TRACE
+// Debug build only (-DDAF_TRACE): first-start / last-end time of each kernel, one table per source file.
+#define DAF_KT_TABLE static __device__ unsigned long long g_kt[32]
+#define DAF_KT_BEGIN(id) do { if (threadIdx.x == 0) atomicMin(&g_kt[2 * (id)], global_ns()); } while (0)
+#define DAF_KT_END(id) do { if (threadIdx.x == 0) atomicMax(&g_kt[2 * (id) + 1], global_ns()); } while (0)
+#define DAF_KT_READER(name)                                                                   \
+    extern "C" int name(void* host, int reset) {                                              \
+        if (reset) {                                                                          \
+            unsigned long long init[32];                                                      \
+            for (int i = 0; i < 32; ++i) init[i] = (i & 1) ? 0ull : ~0ull;                    \
+            return (int)cudaMemcpyToSymbol(g_kt, init, sizeof(init));                         \
+        }                                                                                     \
+        return (int)cudaMemcpyFromSymbol(host, g_kt, 32 * sizeof(unsigned long long));        \
+    }
+#else
+#define DAF_KT_BEGIN(id) do {} while (0)
+#define DAF_KT_END(id) do {} while (0)
+#endif
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
                                           DeviceStatus* st, int where) {
     if (mbar_try_wait(bar, parity)) return true;

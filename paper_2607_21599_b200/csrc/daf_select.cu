@@ -10,6 +10,11 @@
 
 namespace daf {
 
+#ifdef DAF_TRACE
+DAF_KT_TABLE;
+DAF_KT_READER(daf_dbg_kt_select)
+#endif
+
 // ------------------------------------------------------------------ selection
 // A cluster of 8 CTAs ranks all L_d aggregated scores.  Each CTA keeps a
 // contiguous slice of the keys in its shared memory.  Four passes of an
@@ -46,6 +51,7 @@ select_topk_kernel(const float* __restrict__ scores, int n_sig, int L_d, int k,
                    uint32_t* __restrict__ gkeys, int32_t* __restrict__ idx_out) {
     namespace cg = cooperative_groups;
     cg::cluster_group cluster = cg::this_cluster();
+    DAF_KT_BEGIN(0);
     pdl_launch_dependents();   // the gather kernel may start launching; it waits for this grid before reading idx
     extern __shared__ __align__(16) unsigned char sel_smem[];
     SelShared* sh = reinterpret_cast<SelShared*>(sel_smem);
@@ -178,6 +184,7 @@ select_topk_kernel(const float* __restrict__ scores, int n_sig, int L_d, int k,
         }
     }
     cluster.sync();   // no CTA may retire while a peer can still read its shared memory
+    DAF_KT_END(0);
 }
 
 // ------------------------------------------------ selection, one CTA (small L_d)
@@ -358,7 +365,9 @@ struct GatherArgs {
 
 __global__ void __launch_bounds__(kRowThreads)
 gather_update_kernel(const GatherArgs a) {
+    DAF_KT_BEGIN(1);
     pdl_wait();                // idx comes from the selection kernel launched just before
+    DAF_KT_BEGIN(2);
     pdl_launch_dependents();   // the attention kernel may start launching; it waits for this grid
     const int row = blockIdx.x;
     const int per_row = a.cq + 2 * a.ckv;
@@ -393,6 +402,7 @@ gather_update_kernel(const GatherArgs a) {
             else a.kv_v[off + c - a.ckv] = __ldg(a.v_fresh + off + c - a.ckv);
         }
     }
+    DAF_KT_END(1);
 }
 
 // ------------------------------------------------------------- state fusion
