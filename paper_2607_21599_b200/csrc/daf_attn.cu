@@ -2,20 +2,11 @@
 // softmax attention with a causal limit (Methods, items 1 and 2; complexity
 // analysis: the r^2 L_d^2 and L_q (L_d + L_q) terms).
 //
-// One kernel serves all three.  A CTA owns up to two 128-row query tiles that
-// share one KV head and walks the key/value tiles they can see:
-//   - one thread issues TMA loads of K and V tiles into a shared-memory ring,
-//   - one thread issues tcgen05 MMAs: S = Q K^T into tensor memory, then
-//     O += P V with P read back from tensor memory,
-//   - one warpgroup per query tile runs the online softmax, one thread per row,
-//     straight out of tensor memory, and writes the final rows.
-// The two query tiles alternate on the tensor pipe so that the softmax of one
-// overlaps the MMAs of the other.
-//
-// A query tile's 128 rows are (token, head) pairs: `Gp` query heads of one KV
-// group times 128/Gp consecutive tokens.  Gp = 1 for the packed causal
-// attention; Gp = group size for the question rows, so that one pass over the
-// KV cache serves every query head of the group.
+// One kernel (attn_fwd_kernel, described where it is defined) serves all of them;
+// a second one merges the partial results of launches that cut the key axis into
+// ranges.  A launch runs one attention problem, or -- for a DAF layer -- the
+// important-token stage and the question stage together from one list of work
+// items.
 #include <math.h>
 #include <string.h>
 
@@ -26,43 +17,11 @@ namespace daf {
 constexpr int kBlockM = 128;            // rows per query tile
 constexpr int kBlockN = 128;            // keys per KV tile
 constexpr int kD = 128;                 // head_dim
-constexpr int kTileBytes = kBlockN * kD * 2;      // 32 KB: one Q, K or V tile
+constexpr int kTileBytes = kBlockN * kD * 2;      // 32 KB: one Q tile, or K (or V) of 128 keys
 constexpr int kHalfBytes = kTileBytes / 2;        // one 64-column half (128-byte rows)
 constexpr int kMaxSplits = 32;
 constexpr int kNumSMs = 148;
 constexpr float kRescaleThreshold = 8.0f;   // in log2 units: keep a stale row maximum up to 2^8
-
-// Two shapes of the same kernel:
-//   NQ = 2: two query tiles per CTA share every K/V tile (half the shared-memory fill traffic), one CTA
-//           per SM with all 512 tensor-memory columns and a 4-slot ring: for large problems;
-//   NQ = 1: one query tile per CTA, 256 tensor-memory columns and a 2-slot ring, so that two CTAs live on
-//           an SM and cover each other's softmax, prologue and output stores: for problems with few tiles.
-template <int NQ>
-struct AttnCfg {
-    static constexpr int kStages = NQ == 2 ? 4 : 2;        // KV ring slots (K and V tiles alternate through it)
-    static constexpr int kSoftmaxWarps = 4 * NQ;
-    static constexpr int kTmaWarp = kSoftmaxWarps;
-    static constexpr int kMmaWarp = kSoftmaxWarps + 1;
-    static constexpr int kThreads = 32 * (kSoftmaxWarps + 2);
-    static constexpr int kTmemCols = 256 * NQ;             // per tile: S (128 fp32 columns) and O (128)
-    static constexpr int kCtasPerSM = NQ == 2 ? 1 : 2;
-};
-
-template <int NQ>
-struct AttnSmem {
-    uint64_t q_full[NQ];
-    uint64_t kv_full[AttnCfg<NQ>::kStages];
-    uint64_t kv_empty[AttnCfg<NQ>::kStages];
-    uint64_t s_full[NQ];
-    uint64_t p_full[NQ];
-    uint64_t o_done[NQ];
-    uint32_t tmem_base;
-    int abort_flag;
-};
-template <int NQ>
-constexpr size_t attn_smem_bytes() {
-    return 1024 /*alignment slack*/ + (size_t)(NQ + AttnCfg<NQ>::kStages) * kTileBytes + sizeof(AttnSmem<NQ>);
-}
 
 // One attention problem and how it is cut into work items.
 struct SegArgs {
@@ -74,10 +33,10 @@ struct SegArgs {
     int n_tb;           // token blocks = ceil(n_q / Tt)
     int causal_off;     // token t sees keys <= t + causal_off ...
     const int32_t* q_pos; // ... or, when given, keys <= q_pos[t] (ascending positions of the query tokens)
-    // Work items.  A unit is NQ adjacent token blocks (the tiles one CTA owns).  Either every unit is cut
-    // into the same n_splits KV ranges of tiles_per_split tiles (chunk == 0), or -- packed causal attention
-    // only, where unit u sees min(NQ (u + 1), n_tb) tiles -- units [g chunk, (g + 1) chunk) are cut into
-    // g + 1 balanced ranges each, so that no item walks more than about NQ * chunk tiles.
+    // Work items.  A CTA owns one token block (a unit).  Either every unit is cut into the same n_splits
+    // KV ranges of tiles_per_split tiles (chunk == 0), or -- packed causal attention only, where unit u
+    // sees min(u + 1, n_tb) tiles -- units [g chunk, (g + 1) chunk) are cut into g + 1 balanced ranges
+    // each, so that no item walks more than about `chunk` tiles.
     int head_blocks, n_units;
     int n_splits, tiles_per_split;
     int chunk, n_slots;    // n_slots: number of (unit, range) pairs = partial-result slots
@@ -209,8 +168,8 @@ __device__ __forceinline__ void softmax_step(uint32_t s_addr, uint32_t o_addr, i
 // Picks a field of the problem a CTA works on (seg_id is uniform across the CTA).
 #define DAF_SEG(field) (seg_id ? args.seg[1].field : args.seg[0].field)
 
-// What one CTA works on: the problem's geometry and the CTA's item (a unit of NQ token blocks of one
-// head block, and a range of key tiles).
+// What one CTA works on: the problem's geometry and the CTA's item (one token block of one head
+// block, and a range of key tiles).
 struct CtaWork {
     int n_q, n_kv, G, Gp, Tt, n_tb, causal_off;
     const int32_t* q_pos;
@@ -219,7 +178,6 @@ struct CtaWork {
     long long part_row0;      // the item's first row in the partial-result arrays, in tokens
 };
 
-template <int NQ>
 __device__ __forceinline__ void decode_work(const AttnArgs& args, CtaWork& a) {
     // ---- which item is this CTA's (uniform across the CTA)
     int seg_id = 0, item = (int)blockIdx.x;
@@ -262,12 +220,12 @@ __device__ __forceinline__ void decode_work(const AttnArgs& args, CtaWork& a) {
         const int rem = slot - chunk * g * (g + 1) / 2;
         unit = g * chunk + rem / (g + 1);
         const int range = rem % (g + 1);
-        const int n_tiles = min(NQ * (unit + 1), a.n_tb);
+        const int n_tiles = min(unit + 1, a.n_tb);
         j_begin = range * n_tiles / (g + 1);
         j_end = (range + 1) * n_tiles / (g + 1);
         item_splits = g + 1;
-        part_row0 = (long long)slot * (NQ * kBlockM);
-        tok_base = unit * (NQ * kBlockM);
+        part_row0 = (long long)slot * kBlockM;
+        tok_base = unit * kBlockM;
     }
     a.seg_id = seg_id; a.hb = hb; a.unit = unit; a.j_begin = j_begin; a.j_end = j_end;
     a.item_splits = item_splits; a.tok_base = tok_base; a.part_row0 = part_row0;
@@ -376,248 +334,6 @@ __device__ __forceinline__ void write_rows(const AttnArgs& args, const CtaWork& 
     }
 }
 
-template <int NQ>
-__global__ void __launch_bounds__(AttnCfg<NQ>::kThreads, AttnCfg<NQ>::kCtasPerSM)
-attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_constant__ CUtensorMap tmap_k0,
-                const __grid_constant__ CUtensorMap tmap_v0, const __grid_constant__ CUtensorMap tmap_q1,
-                const __grid_constant__ CUtensorMap tmap_k1, const __grid_constant__ CUtensorMap tmap_v1,
-                const AttnArgs args) {
-    constexpr int kNQ = NQ;
-    constexpr int kStages = AttnCfg<NQ>::kStages;
-    constexpr int kTmaWarp = AttnCfg<NQ>::kTmaWarp;
-    constexpr int kMmaWarp = AttnCfg<NQ>::kMmaWarp;
-    constexpr int kTmemCols = AttnCfg<NQ>::kTmemCols;
-    extern __shared__ unsigned char attn_smem_raw[];
-    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(attn_smem_raw) + 1023) & ~(uintptr_t)1023);
-    unsigned char* q_smem = smem;                                   // kNQ tiles
-    unsigned char* kv_smem = smem + (size_t)kNQ * kTileBytes;       // kStages tiles
-    AttnSmem<NQ>* sm = reinterpret_cast<AttnSmem<NQ>*>(kv_smem + (size_t)kStages * kTileBytes);
-
-    pdl_wait();                // inputs may come from the kernel launched just before (gather / hybrid-cache update)
-    pdl_launch_dependents();   // a dependent kernel (the split merge) may start launching; it waits for this grid
-
-    // a CTA of this grid (or an earlier kernel sharing the workspace) has already given up: do nothing
-    __shared__ int skip_cta;
-    if (threadIdx.x == 0) skip_cta = (args.status != nullptr && *reinterpret_cast<volatile int*>(&args.status->code) != 0) ? 1 : 0;
-    __syncthreads();
-    if (skip_cta) return;
-
-    if (threadIdx.x == 0) DAF_STAMP(0);
-    DAF_KT_BEGIN(0);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-
-    // ---- which item is this CTA's (uniform across the CTA)
-    CtaWork a;
-    decode_work<NQ>(args, a);
-    const int seg_id = a.seg_id, hb = a.hb, unit = a.unit, j_begin = a.j_begin, j_end = a.j_end;
-    const int item_splits = a.item_splits;
-    const CUtensorMap* tmap_q = seg_id ? &tmap_q1 : &tmap_q0;
-    const CUtensorMap* tmap_k = seg_id ? &tmap_k1 : &tmap_k0;
-    const CUtensorMap* tmap_v = seg_id ? &tmap_v1 : &tmap_v0;
-    DeviceStatus* const status = args.status;
-    const int h0 = hb * a.Gp;
-    const int g_kv = h0 / a.G;
-
-    // per-tile geometry (uniform across the CTA)
-    int t0[kNQ], n_j[kNQ];
-    int n_j_max = 0;
-#pragma unroll
-    for (int q = 0; q < kNQ; ++q) {
-        const int tb = unit * kNQ + q;
-        t0[q] = tb * a.Tt;
-        int nj = 0;
-        if (tb < a.n_tb) {
-            const int max_tok = min(a.n_q, t0[q] + a.Tt) - 1;
-            const long long last_key = a.q_pos ? (long long)__ldg(a.q_pos + max_tok) : (long long)max_tok + a.causal_off;
-            const long long kv_hi = min((long long)a.n_kv, last_key + 1);
-            const int tiles_total = kv_hi > 0 ? (int)((kv_hi + kBlockN - 1) / kBlockN) : 0;
-            nj = max(0, min(tiles_total, j_end) - j_begin);
-        }
-        n_j[q] = nj;
-        n_j_max = max(n_j_max, nj);
-    }
-
-    if (threadIdx.x == 0) {
-        for (int q = 0; q < kNQ; ++q) {
-            mbar_init(&sm->q_full[q], 1);
-            mbar_init(&sm->s_full[q], 1);
-            mbar_init(&sm->p_full[q], 128);
-            mbar_init(&sm->o_done[q], 1);
-        }
-        for (int s = 0; s < kStages; ++s) { mbar_init(&sm->kv_full[s], 1); mbar_init(&sm->kv_empty[s], 1); }
-        sm->abort_flag = 0;
-        mbar_fence_init();
-    }
-    if (warp == kMmaWarp) {
-        tmem_alloc(&sm->tmem_base, kTmemCols);
-        tmem_relinquish();
-    }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem = sm->tmem_base;
-    volatile int* abort_flag = &sm->abort_flag;
-    if (threadIdx.x == 0) DAF_STAMP(1);
-
-    if (warp == kTmaWarp) {
-        // ------------------------------------------------------------ TMA producer
-        if (lane == 0) {
-            tma_prefetch_desc(tmap_q);
-            tma_prefetch_desc(tmap_k);
-            tma_prefetch_desc(tmap_v);
-            const uint32_t q_tx = 2u * 128u * (uint32_t)(a.Gp * a.Tt);
-            for (int q = 0; q < kNQ; ++q) {
-                if (n_j[q] > 0) {
-                    unsigned char* dst = q_smem + (size_t)q * kTileBytes;
-                    mbar_arrive_expect_tx(&sm->q_full[q], q_tx);
-                    tma_load_3d(dst, tmap_q, &sm->q_full[q], 0, h0, t0[q]);
-                    tma_load_3d(dst + kHalfBytes, tmap_q, &sm->q_full[q], 64, h0, t0[q]);
-                }
-            }
-            bool ok = true;
-            int seq = 0;
-            for (int j = 0; j < n_j_max && ok; ++j) {
-                const int key0 = (j_begin + j) * kBlockN;
-                for (int kv = 0; kv < 2 && ok; ++kv, ++seq) {
-                    const int slot = seq % kStages;
-                    const uint32_t round = (uint32_t)(seq / kStages);
-                    if (round > 0) ok = mbar_wait(&sm->kv_empty[slot], (round - 1) & 1u, abort_flag, status, 10 + slot);
-                    if (!ok) break;
-                    unsigned char* dst = kv_smem + (size_t)slot * kTileBytes;
-                    const CUtensorMap* tm = kv == 0 ? tmap_k : tmap_v;
-                    mbar_arrive_expect_tx(&sm->kv_full[slot], (uint32_t)kTileBytes);
-                    tma_load_3d(dst, tm, &sm->kv_full[slot], 0, g_kv, key0);
-                    tma_load_3d(dst + kHalfBytes, tm, &sm->kv_full[slot], 64, g_kv, key0);
-                }
-            }
-            if (!ok) {
-                // give loads already in flight a bounded chance to land before the CTA retires
-                for (int s = 0; s < kStages; ++s)
-                    for (int it = 0; it < 4096 && !mbar_try_wait(&sm->kv_full[s], 0) && !mbar_try_wait(&sm->kv_full[s], 1); ++it) {}
-            }
-        }
-    } else if (warp == kMmaWarp) {
-        // ------------------------------------------------------------ MMA issuer
-        if (lane == 0 && n_j_max > 0) {
-            constexpr uint32_t idesc_qk = make_idesc_bf16(kBlockM, kBlockN, 0);
-            constexpr uint32_t idesc_pv = make_idesc_bf16(kBlockM, kD, 1);
-            bool ok = true;
-            for (int q = 0; q < kNQ && ok; ++q)
-                if (n_j[q] > 0) ok = mbar_wait(&sm->q_full[q], 0, abort_flag, status, 20 + q);
-            auto slot_of = [](int seq) { return seq % kStages; };
-            auto parity_of = [](int seq) { return (uint32_t)((seq / kStages) & 1); };
-            auto issue_qk = [&](int q, int slot) {
-                const uint32_t qa = smem_u32(q_smem + (size_t)q * kTileBytes);
-                const uint32_t ka = smem_u32(kv_smem + (size_t)slot * kTileBytes);
-#pragma unroll
-                for (int kk = 0; kk < kD / 16; ++kk) {
-                    const uint32_t off = (uint32_t)((kk & 3) * 32 + (kk >> 2) * kHalfBytes);
-                    tc_mma_ss(tmem + (uint32_t)(q * kBlockN), make_smem_desc(qa + off, 16, 1024),
-                              make_smem_desc(ka + off, 16, 1024), idesc_qk, kk > 0 ? 1u : 0u);
-                }
-            };
-            auto issue_pv = [&](int q, int slot, bool first) {
-                const uint32_t va = smem_u32(kv_smem + (size_t)slot * kTileBytes);
-#pragma unroll
-                for (int kk = 0; kk < kBlockN / 16; ++kk) {
-                    // 16 keys per MMA: two 8-key groups of 1024 bytes; the two 64-column halves are kHalfBytes apart
-                    tc_mma_ts(tmem + (uint32_t)(kNQ * kBlockN + q * kD), tmem + (uint32_t)(q * kBlockN + kk * 8),
-                              make_smem_desc(va + (uint32_t)kk * 2048u, kHalfBytes, 1024), idesc_pv,
-                              (first && kk == 0) ? 0u : 1u);
-                }
-            };
-            if (ok) ok = mbar_wait(&sm->kv_full[slot_of(0)], parity_of(0), abort_flag, status, 30);
-            if (ok) {
-                tc_fence_after();
-                for (int q = 0; q < kNQ; ++q)
-                    if (n_j[q] > 0) { issue_qk(q, slot_of(0)); tc_commit(&sm->s_full[q]); }
-                tc_commit(&sm->kv_empty[slot_of(0)]);
-            }
-            for (int j = 0; j < n_j_max && ok; ++j) {
-                const int seq_v = 2 * j + 1, seq_k = 2 * j + 2;
-                const bool more = j + 1 < n_j_max;
-                ok = mbar_wait(&sm->kv_full[slot_of(seq_v)], parity_of(seq_v), abort_flag, status, 31);
-                if (ok && more) ok = mbar_wait(&sm->kv_full[slot_of(seq_k)], parity_of(seq_k), abort_flag, status, 32);
-                if (!ok) break;
-                tc_fence_after();
-                bool last_tile[kNQ];
-                for (int q = 0; q < kNQ && ok; ++q) {
-                    last_tile[q] = false;
-                    if (j >= n_j[q]) continue;
-                    ok = mbar_wait(&sm->p_full[q], (uint32_t)(j & 1), abort_flag, status, 40 + q);
-                    if (!ok) break;
-                    tc_fence_after();
-                    issue_pv(q, slot_of(seq_v), j == 0);
-                    if (j + 1 < n_j[q]) { issue_qk(q, slot_of(seq_k)); tc_commit(&sm->s_full[q]); }
-                    else if (more) tc_commit(&sm->o_done[q]);   // this tile is done early: release its epilogue now
-                    else last_tile[q] = true;
-                }
-                if (!ok) break;
-                tc_commit(&sm->kv_empty[slot_of(seq_v)]);
-                if (more) tc_commit(&sm->kv_empty[slot_of(seq_k)]);
-                // the "output ready" arrival goes last, so that no arrival of this CTA is still
-                // outstanding once its softmax warps have seen it
-                for (int q = 0; q < kNQ; ++q)
-                    if (last_tile[q]) tc_commit(&sm->o_done[q]);
-            }
-        }
-    } else {
-        // ------------------------------------------------------------ softmax + epilogue, one row per thread
-        const int q = warp >> 2;
-        const int quad = warp & 3;
-        const int r = quad * 32 + lane;
-        const int tok = t0[q] + r / a.Gp;
-        const int head = h0 + r % a.Gp;
-        const bool row_valid_tile = (n_j[q] > 0 || item_splits > 1) && (unit * kNQ + q < a.n_tb);
-        const bool row_valid = (r < a.Gp * a.Tt) && (tok < a.n_q) && row_valid_tile;
-        const long long lim_ll = (a.q_pos && tok < a.n_q) ? (long long)__ldg(a.q_pos + tok) : (long long)tok + a.causal_off;
-        const int limit = row_valid ? (int)min(lim_ll, (long long)a.n_kv - 1) : -1;   // last visible key
-        const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
-        const uint32_t s_addr = tmem + lane_addr + (uint32_t)(q * kBlockN);
-        const uint32_t o_addr = tmem + lane_addr + (uint32_t)(kNQ * kBlockN + q * kD);
-        const float c = a.scale_log2;
-
-        float m = -INFINITY, l = 0.f;
-        bool ok = true;
-        for (int j = 0; j < n_j[q]; ++j) {
-            ok = mbar_wait(&sm->s_full[q], (uint32_t)(j & 1), abort_flag, status, 50 + q);
-            ok = __all_sync(0xFFFFFFFFu, ok);
-            if (!ok) break;
-            tc_fence_after();
-            if (threadIdx.x == 0 && j == 0) DAF_STAMP(2);
-            softmax_step(s_addr, o_addr, (j_begin + j) * kBlockN, limit, c, j == 0, m, l);
-            mbar_arrive(&sm->p_full[q]);
-        }
-        if (threadIdx.x == 0) DAF_STAMP(3);
-        // ---- epilogue
-        if (ok && n_j[q] > 0) {
-            ok = mbar_wait(&sm->o_done[q], 0, abort_flag, status, 60 + q);
-            ok = __all_sync(0xFFFFFFFFu, ok);
-        }
-        if (ok) {
-            tc_fence_after();
-            write_rows(args, a, t0[q], n_j[q] > 0, row_valid, row_valid_tile, tok, head, h0,
-                       q_smem + (size_t)q * kTileBytes + (size_t)quad * 32 * 256, o_addr, quad, lane, m, l);
-        }
-    }
-
-    if (threadIdx.x == 0) DAF_STAMP(4);
-    tc_fence_before();
-    __syncthreads();
-    if (warp == kMmaWarp) {
-        tc_fence_after();
-        tmem_dealloc(tmem, kTmemCols);
-    }
-    DAF_KT_END(0);
-#ifdef DAF_TRACE
-    if (threadIdx.x == 0) {
-        DAF_STAMP(5);
-        const unsigned cta = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
-        if (cta < 65536u) g_trace[8 * cta + 6] = (unsigned long long)n_j_max;
-    }
-#endif
-}
-
 #ifdef DAF_TRACE
 extern "C" int daf_dbg_read_trace(void* host, size_t bytes) {
     return (int)cudaMemcpyFromSymbol(host, g_trace, bytes < sizeof(g_trace) ? bytes : sizeof(g_trace));
@@ -625,22 +341,30 @@ extern "C" int daf_dbg_read_trace(void* host, size_t bytes) {
 #endif
 
 // ------------------------------------------------------------------------------------------------
-// One query tile per CTA, two CTAs per SM, for problems with few tiles.
+// The attention kernel: one 128-row query tile per CTA, two CTAs per SM.
 //
-// With a single tile a CTA has nothing to overlap a key tile's softmax with, and the chain
-// S = Q K^T -> softmax -> O += P V -> next S runs at the sum of its latencies.  Here the keys go
-// through in sub-steps of 64 and S is double-buffered (two 64-column halves of the same 128 tensor-
-// memory columns): the logits of sub-step t + 1 are computed while the softmax of sub-step t
-// runs, so the softmax warps find their next input ready.  The products O += P_t V_t are issued
-// as each P_t arrives; a row may only be rescaled, and P_{t+1} only be handed over, once the
-// product before it has completed (pv_done).
+// A tile's rows are (token, head) pairs: `Gp` query heads of one KV group times 128/Gp consecutive
+// tokens.  Gp = 1 for the packed causal attention; Gp = group size for the question rows, so that
+// one pass over the KV cache serves every query head of the group.
+//   - one thread issues TMA loads of Q and of K/V sub-tiles of 64 keys into shared-memory rings,
+//   - one thread issues tcgen05 MMAs: S = Q K^T into tensor memory, then O += P V with P read back
+//     from tensor memory,
+//   - four warps run the online softmax, one thread per row, straight out of tensor memory, and
+//     write the final rows.
+// The keys go through in sub-steps of 64 and S is double-buffered (two 64-column halves of the
+// same 128 tensor-memory columns): the logits of sub-step t + 1 are computed while the softmax of
+// sub-step t runs, so the softmax warps find their next input ready.  The products O += P_t V_t are
+// issued as each P_t arrives; a row may only be rescaled, and P_{t+1} only be handed over, once the
+// product before it has completed (pv_done).  The second CTA of the SM fills what gaps remain.
+// Two tiles per CTA sharing every K/V tile (half the shared-memory fill traffic, one CTA per SM)
+// measured slower at every size from 1k to 136k tokens and was removed.
 constexpr int kSubN = 64;                               // keys per sub-step
 constexpr int kSubBytes = kSubN * kD * 2;               // 16 KB: K or V of one sub-step, two 64-column halves
 constexpr int kSubHalfBytes = kSubBytes / 2;
-constexpr int kSmallThreads = 192;                      // warps 0-3 softmax, warp 4 TMA, warp 5 MMA
-constexpr int kSmallTmemCols = 256;                     // S (two halves of 64) and O (128)
+constexpr int kAttnThreads = 192;                      // warps 0-3 softmax, warp 4 TMA, warp 5 MMA
+constexpr int kAttnTmemCols = 256;                     // S (two halves of 64) and O (128)
 
-struct SmallSmem {
+struct AttnSmem {
     uint64_t q_full;
     uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2];
     uint64_t s_full[2], p_full[2];
@@ -648,10 +372,10 @@ struct SmallSmem {
     uint32_t tmem_base;
     int abort_flag;
 };
-constexpr size_t kSmallSmemBytes = 1024 + 3 * (size_t)kTileBytes + sizeof(SmallSmem);
+constexpr size_t kAttnSmemBytes = 1024 + 3 * (size_t)kTileBytes + sizeof(AttnSmem);
 
-__global__ void __launch_bounds__(kSmallThreads, 2)
-attn_small_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_constant__ CUtensorMap tmap_k0,
+__global__ void __launch_bounds__(kAttnThreads, 2)
+attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_constant__ CUtensorMap tmap_k0,
                   const __grid_constant__ CUtensorMap tmap_v0, const __grid_constant__ CUtensorMap tmap_q1,
                   const __grid_constant__ CUtensorMap tmap_k1, const __grid_constant__ CUtensorMap tmap_v1,
                   const AttnArgs args) {
@@ -660,7 +384,7 @@ attn_small_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_cons
     unsigned char* q_smem = smem;                                 // 32 KB
     unsigned char* k_smem = smem + kTileBytes;                    // two sub-step slots
     unsigned char* v_smem = smem + 2 * (size_t)kTileBytes;        // two sub-step slots
-    SmallSmem* sm = reinterpret_cast<SmallSmem*>(smem + 3 * (size_t)kTileBytes);
+    AttnSmem* sm = reinterpret_cast<AttnSmem*>(smem + 3 * (size_t)kTileBytes);
 
     pdl_wait();                // inputs may come from the kernel launched just before (gather / hybrid-cache update)
     pdl_launch_dependents();   // a dependent kernel (the split merge) may start launching; it waits for this grid
@@ -675,7 +399,7 @@ attn_small_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_cons
     DAF_KT_BEGIN(0);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     CtaWork a;
-    decode_work<1>(args, a);
+    decode_work(args, a);
     const int seg_id = a.seg_id;
     const CUtensorMap* tmap_q = seg_id ? &tmap_q1 : &tmap_q0;
     const CUtensorMap* tmap_k = seg_id ? &tmap_k1 : &tmap_k0;
@@ -707,7 +431,7 @@ attn_small_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_cons
         mbar_fence_init();
     }
     if (warp == 5) {
-        tmem_alloc(&sm->tmem_base, kSmallTmemCols);
+        tmem_alloc(&sm->tmem_base, kAttnTmemCols);
         tmem_relinquish();
     }
     tc_fence_before();
@@ -860,7 +584,7 @@ attn_small_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_cons
     __syncthreads();
     if (warp == 5) {
         tc_fence_after();
-        tmem_dealloc(tmem, kSmallTmemCols);
+        tmem_dealloc(tmem, kAttnTmemCols);
     }
     DAF_KT_END(0);
 #ifdef DAF_TRACE
@@ -996,21 +720,15 @@ static int set_kernel_attributes() {
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !attr_done[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(attn_fwd_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem_bytes<1>());
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(attn_fwd_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem_bytes<2>());
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(attn_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmallSmemBytes);
+        cudaError_t e = cudaFuncSetAttribute(attn_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttnSmemBytes);
         if (e != cudaSuccess) { set_cuda_error(e); return DAF_ERR_CUDA; }
         attr_done[dev] = true;
     }
     return DAF_OK;
 }
 
-// How a single problem is cut into CTAs.  Splitting the KV axis is only used for the
-// question rows, where there are few query tiles and a long KV axis.
-static int g_force_nq = 0;        // 0: choose by problem size (the tuning builds can pin a shape)
-static int g_small = 1;            // one-tile launches use the kernel with 64-key sub-steps
+// How a single problem is cut into CTAs: one per (head block, token block), and for the question rows,
+// where there are few query tiles and a long KV axis, also per range of the KV axis.
 static float g_joint_factor = 1.0f;   // longest item of a joint launch, as a fraction of the mean load of a CTA slot
 
 AttnPlan plan_attention(int n_q, int n_kv, int Hq, int G, int causal_off, bool pack_group, bool allow_split) {
@@ -1020,22 +738,14 @@ AttnPlan plan_attention(int n_q, int n_kv, int Hq, int G, int causal_off, bool p
     pl.Tt = kBlockM / pl.Gp;
     pl.n_tb = (n_q + pl.Tt - 1) / pl.Tt;
     pl.head_blocks = Hq / pl.Gp;
-    // two tiles per CTA once that alone fills every SM twice over; otherwise one tile per CTA, two CTAs per SM
-    const int ctas_two = ((pl.n_tb + 1) / 2) * pl.head_blocks;
-    pl.nq = ctas_two >= 2 * kNumSMs ? 2 : 1;
-    // The question stage streams a long KV axis through few query tiles: there two tiles per CTA that share
-    // every K/V tile measured faster (at 32k context: 96 us with one tile per CTA, about 70 us with two).
-    if (allow_split && pl.n_tb >= 2) pl.nq = 2;
-    if (g_force_nq == 1 || g_force_nq == 2) pl.nq = g_force_nq;
-    pl.pairs = (pl.n_tb + pl.nq - 1) / pl.nq;
     long long kv_hi = (long long)n_q - 1 + causal_off + 1;
     if (kv_hi > n_kv) kv_hi = n_kv;
     const int total_tiles = kv_hi > 0 ? (int)((kv_hi + kBlockN - 1) / kBlockN) : 0;
     pl.n_splits = 1;
     pl.tiles_per_split = total_tiles > 0 ? total_tiles : 1;
     if (allow_split && total_tiles > 1) {
-        const int ctas = pl.pairs * pl.head_blocks;
-        const int slots = kNumSMs * (pl.nq == 2 ? 1 : 2);
+        const int ctas = pl.n_tb * pl.head_blocks;
+        const int slots = kNumSMs * 2;
         int want = ctas > 0 ? slots / ctas : 1;
         if (want > kMaxSplits) want = kMaxSplits;
         if (want > total_tiles) want = total_tiles;
@@ -1067,50 +777,43 @@ JointPlan plan_joint(int k, int L_q, int L_d, int Hq, int G) {
     JointPlan jp;
     const int N = L_d + L_q;
     jp.n_tb_i = (k + kBlockM - 1) / kBlockM;
-    jp.nq = ((jp.n_tb_i + 1) / 2) * Hq >= 2 * kNumSMs ? 2 : 1;
-    if (g_force_nq == 1 || g_force_nq == 2) jp.nq = g_force_nq;
-    jp.n_units_i = (jp.n_tb_i + jp.nq - 1) / jp.nq;
     jp.Gp_q = G > 128 ? 1 : G;
     jp.Tt_q = kBlockM / jp.Gp_q;
     jp.n_tb_q = (L_q + jp.Tt_q - 1) / jp.Tt_q;
     jp.head_blocks_q = Hq / jp.Gp_q;
-    jp.n_units_q = (jp.n_tb_q + jp.nq - 1) / jp.nq;
     const int tiles_q = (N + kBlockN - 1) / kBlockN;
-    long long work = 0;   // in CTA steps (one K/V tile through the CTA's tiles)
-    for (int u = 0; u < jp.n_units_i; ++u) work += (long long)Hq * (jp.nq * (u + 1) < jp.n_tb_i ? jp.nq * (u + 1) : jp.n_tb_i);
-    work += (long long)jp.head_blocks_q * jp.n_units_q * tiles_q;
-    const int slots = kNumSMs * (jp.nq == 2 ? 1 : 2);
+    // work in CTA steps (one 128-key tile through one query tile)
+    long long work = (long long)Hq * jp.n_tb_i * (jp.n_tb_i + 1) / 2 + (long long)jp.head_blocks_q * jp.n_tb_q * tiles_q;
+    const int slots = kNumSMs * 2;
     int longest = (int)ceilf(g_joint_factor * (float)work / (float)slots);
     if (longest < 2) longest = 2;
     auto set_chunk = [&](int chunk) {
         if (chunk < 1) chunk = 1;
-        if (chunk < (jp.n_units_i + 31) / 32) chunk = (jp.n_units_i + 31) / 32;   // at most 32 ranges per unit
-        if (chunk > jp.n_units_i) chunk = jp.n_units_i;
+        if (chunk < (jp.n_tb_i + 31) / 32) chunk = (jp.n_tb_i + 31) / 32;   // at most 32 ranges per token block
+        if (chunk > jp.n_tb_i) chunk = jp.n_tb_i;
         jp.chunk = chunk;
-        jp.n_slots = slots_before(jp.n_units_i, chunk);
+        jp.n_slots = slots_before(jp.n_tb_i, chunk);
         jp.part_bytes_i = 0;
-        if (chunk < jp.n_units_i) {
-            const size_t rows = (size_t)jp.n_slots * jp.nq * kBlockM * Hq;
+        if (chunk < jp.n_tb_i) {
+            const size_t rows = (size_t)jp.n_slots * kBlockM * Hq;
             jp.part_bytes_i = rows * kD * sizeof(float) + (rows * sizeof(float) + 255) / 256 * 256;
         }
     };
-    set_chunk(longest / jp.nq);
-    if (jp.part_bytes_i > ((size_t)256 << 20)) set_chunk(jp.n_units_i);   // partials of a large problem: not worth their traffic
+    set_chunk(longest);
+    if (jp.part_bytes_i > ((size_t)256 << 20)) set_chunk(jp.n_tb_i);   // partials of a large problem: not worth their traffic
     jp.items_i = Hq * jp.n_slots;
     int want = (tiles_q + longest - 1) / longest;
     if (want > kMaxSplits) want = kMaxSplits;
     if (want < 1) want = 1;
     jp.tiles_per_split_q = (tiles_q + want - 1) / want;
     jp.n_splits_q = (tiles_q + jp.tiles_per_split_q - 1) / jp.tiles_per_split_q;
-    jp.items_q = jp.head_blocks_q * jp.n_units_q * jp.n_splits_q;
+    jp.items_q = jp.head_blocks_q * jp.n_tb_q * jp.n_splits_q;
     jp.part_bytes_q = attn_partial_bytes(L_q, Hq, jp.n_splits_q);
     return jp;
 }
 
 #ifdef DAF_TRACE
-extern "C" void daf_dbg_force_nq(int nq) { g_force_nq = nq; }
 extern "C" void daf_dbg_joint_factor(float f) { g_joint_factor = f; }
-extern "C" void daf_dbg_small(int on) { g_small = on; }
 #endif
 
 static void fill_problem(SegArgs* s, int n_q, int n_kv, int Hq, int G, int Gp, int causal_off, const int32_t* q_pos,
@@ -1127,7 +830,8 @@ static void fill_problem(SegArgs* s, int n_q, int n_kv, int Hq, int G, int Gp, i
     s->lse = lse;
 }
 
-static void fill_combine(CombineSeg* c, const SegArgs& s, int unit_tokens) {
+static void fill_combine(CombineSeg* c, const SegArgs& s) {
+    const int unit_tokens = kBlockM;   // packed causal attention has one head per tile: a unit is 128 tokens
     c->part_o = s.part_o; c->part_lse = s.part_lse;
     c->n_q = s.n_q; c->Hq = s.Hq;
     c->n_splits = s.chunk == 0 ? s.n_splits : 0;
@@ -1161,37 +865,32 @@ int launch_attention(const void* q, const void* k, const void* v, int n_q, int n
 
     CUtensorMap tq, tk, tv;
     if (int rc = make_tmap(&tq, q, n_q, Hq, pl.Gp, pl.Tt)) return rc;
-    const bool small = pl.nq == 1 && g_small;      // one tile per CTA: keys go through in sub-steps of 64
-    const int kv_box = small ? kSubN : kBlockN;
-    if (int rc = make_tmap(&tk, k, n_kv, Hkv, 1, kv_box)) return rc;
-    if (int rc = make_tmap(&tv, v, n_kv, Hkv, 1, kv_box)) return rc;
+    if (int rc = make_tmap(&tk, k, n_kv, Hkv, 1, kSubN)) return rc;
+    if (int rc = make_tmap(&tv, v, n_kv, Hkv, 1, kSubN)) return rc;
     if (int rc = set_kernel_attributes()) return rc;
 
     AttnArgs a;
     memset(&a, 0, sizeof(a));
     SegArgs& s = a.seg[0];
     fill_problem(&s, n_q, n_kv, Hq, G, pl.Gp, causal_off, q_pos, scale, out, out_row_stride_bytes, dst_rows, lse);
-    s.n_units = pl.pairs;
+    s.n_units = pl.n_tb;
     s.n_splits = pl.n_splits; s.tiles_per_split = pl.tiles_per_split;
     s.chunk = 0; s.n_slots = 0;
-    s.n_items = pl.head_blocks * pl.pairs * pl.n_splits;
+    s.n_items = pl.head_blocks * pl.n_tb * pl.n_splits;
     s.part_o = reinterpret_cast<float*>(scratch);
     s.part_lse = pl.n_splits > 1 ? reinterpret_cast<float*>(reinterpret_cast<char*>(scratch) +
                                                             (size_t)pl.n_splits * n_q * Hq * kD * sizeof(float))
                                  : nullptr;
     a.joint = 0;
     a.status = status;
-    dim3 grid((unsigned)pl.head_blocks, (unsigned)pl.pairs, (unsigned)pl.n_splits);
-    cudaError_t e;
-    if (pl.nq == 2) e = launch_kernel(attn_fwd_kernel<2>, grid, dim3(AttnCfg<2>::kThreads), attn_smem_bytes<2>(), stream, after_kernel, tq, tk, tv, tq, tk, tv, a);
-    else if (small) e = launch_kernel(attn_small_kernel, grid, dim3(kSmallThreads), kSmallSmemBytes, stream, after_kernel, tq, tk, tv, tq, tk, tv, a);
-    else e = launch_kernel(attn_fwd_kernel<1>, grid, dim3(AttnCfg<1>::kThreads), attn_smem_bytes<1>(), stream, after_kernel, tq, tk, tv, tq, tk, tv, a);
+    dim3 grid((unsigned)pl.head_blocks, (unsigned)pl.n_tb, (unsigned)pl.n_splits);
+    cudaError_t e = launch_kernel(attn_fwd_kernel, grid, dim3(kAttnThreads), kAttnSmemBytes, stream, after_kernel, tq, tk, tv, tq, tk, tv, a);
     count_launch();
     if (e != cudaSuccess) { set_cuda_error(e); return DAF_ERR_CUDA; }
     if (int rc = check_launch()) return rc;
     if (pl.n_splits > 1) {
         CombineSeg c0, c1;
-        fill_combine(&c0, s, pl.nq * kBlockM);
+        fill_combine(&c0, s);
         memset(&c1, 0, sizeof(c1));
         return launch_combine(c0, c1, stream);
     }
@@ -1211,13 +910,11 @@ int launch_attention_joint(const void* q_imp, const void* k_imp, const void* v_i
 
     CUtensorMap tq0, tk0, tv0, tq1, tk1, tv1;
     if (int rc = make_tmap(&tq0, q_imp, k, Hq, 1, kBlockM)) return rc;
-    const bool small = jp.nq == 1 && g_small;
-    const int kv_box = small ? kSubN : kBlockN;
-    if (int rc = make_tmap(&tk0, k_imp, k, Hkv, 1, kv_box)) return rc;
-    if (int rc = make_tmap(&tv0, v_imp, k, Hkv, 1, kv_box)) return rc;
+    if (int rc = make_tmap(&tk0, k_imp, k, Hkv, 1, kSubN)) return rc;
+    if (int rc = make_tmap(&tv0, v_imp, k, Hkv, 1, kSubN)) return rc;
     if (int rc = make_tmap(&tq1, q_question, L_q, Hq, jp.Gp_q, jp.Tt_q)) return rc;
-    if (int rc = make_tmap(&tk1, kv_k, N, Hkv, 1, kv_box)) return rc;
-    if (int rc = make_tmap(&tv1, kv_v, N, Hkv, 1, kv_box)) return rc;
+    if (int rc = make_tmap(&tk1, kv_k, N, Hkv, 1, kSubN)) return rc;
+    if (int rc = make_tmap(&tv1, kv_v, N, Hkv, 1, kSubN)) return rc;
     if (int rc = set_kernel_attributes()) return rc;
 
     AttnArgs a;
@@ -1226,7 +923,7 @@ int launch_attention_joint(const void* q_imp, const void* k_imp, const void* v_i
     // question rows: every unit cut into the same KV splits
     SegArgs& sq = a.seg[1];
     fill_problem(&sq, L_q, N, Hq, G, jp.Gp_q, L_d, nullptr, scale, out_question, out_row_stride_bytes, nullptr, nullptr);
-    sq.n_units = jp.n_units_q;
+    sq.n_units = jp.n_tb_q;
     sq.n_splits = jp.n_splits_q; sq.tiles_per_split = jp.tiles_per_split_q;
     sq.chunk = 0; sq.n_slots = 0;
     sq.n_items = jp.items_q;
@@ -1235,34 +932,25 @@ int launch_attention_joint(const void* q_imp, const void* k_imp, const void* v_i
     // important tokens: packed causal attention, long chains cut into balanced ranges
     SegArgs& si = a.seg[0];
     fill_problem(&si, k, k, Hq, G, 1, 0, nullptr, scale, out_imp, out_row_stride_bytes, dst_rows_imp, nullptr);
-    si.n_units = jp.n_units_i;
+    si.n_units = jp.n_tb_i;
     si.n_splits = 1; si.tiles_per_split = jp.n_tb_i;
     si.chunk = jp.chunk; si.n_slots = jp.n_slots;
     si.n_items = jp.items_i;
-    const size_t rows_i = (size_t)jp.n_slots * jp.nq * kBlockM * Hq;
+    const size_t rows_i = (size_t)jp.n_slots * kBlockM * Hq;
     si.part_o = reinterpret_cast<float*>(sc + jp.part_bytes_q);
     si.part_lse = reinterpret_cast<float*>(sc + jp.part_bytes_q + rows_i * kD * sizeof(float));
     a.joint = 1;
     a.status = status;
 
     const int items = jp.items_q + jp.items_i;
-    cudaError_t e;
-    if (jp.nq == 2) {
-        e = launch_kernel(attn_fwd_kernel<2>, dim3((unsigned)items), dim3(AttnCfg<2>::kThreads), attn_smem_bytes<2>(), stream,
-                          after_kernel, tq0, tk0, tv0, tq1, tk1, tv1, a);
-    } else if (small) {
-        e = launch_kernel(attn_small_kernel, dim3((unsigned)items), dim3(kSmallThreads), kSmallSmemBytes, stream,
-                          after_kernel, tq0, tk0, tv0, tq1, tk1, tv1, a);
-    } else {
-        e = launch_kernel(attn_fwd_kernel<1>, dim3((unsigned)items), dim3(AttnCfg<1>::kThreads), attn_smem_bytes<1>(), stream,
-                          after_kernel, tq0, tk0, tv0, tq1, tk1, tv1, a);
-    }
+    const cudaError_t e = launch_kernel(attn_fwd_kernel, dim3((unsigned)items), dim3(kAttnThreads), kAttnSmemBytes, stream,
+                                        after_kernel, tq0, tk0, tv0, tq1, tk1, tv1, a);
     count_launch();
     if (e != cudaSuccess) { set_cuda_error(e); return DAF_ERR_CUDA; }
     if (int rc = check_launch()) return rc;
     CombineSeg ci, cq;
-    fill_combine(&ci, si, jp.nq * kBlockM);
-    fill_combine(&cq, sq, jp.nq * kBlockM);
+    fill_combine(&ci, si);
+    fill_combine(&cq, sq);
     return launch_combine(ci, cq, stream);
 }
 

@@ -45,7 +45,7 @@ int launch_fuse(const ResolvedParams& rp, const int32_t* idx, const void* o_imp,
                 int32_t* row_pos_out, cudaStream_t stream);
 int launch_deviation_scores(const ResolvedParams& rp, const void* k_fresh, const void* v_fresh, const void* k_cached,
                             const void* v_cached, float* scores, cudaStream_t stream);
-struct AttnPlan { int Gp, Tt, n_tb, nq, pairs, head_blocks, n_splits, tiles_per_split; };
+struct AttnPlan { int Gp, Tt, n_tb, head_blocks, n_splits, tiles_per_split; };
 AttnPlan plan_attention(int n_q, int n_kv, int Hq, int G, int causal_off, bool pack_group, bool allow_split);
 size_t attn_partial_bytes(int n_q, int Hq, int n_splits);
 int launch_attention(const void* q, const void* k, const void* v, int n_q, int n_kv, int Hq, int Hkv, int causal_off,
@@ -54,9 +54,8 @@ int launch_attention(const void* q, const void* k, const void* v, int n_q, int n
                      cudaStream_t stream, bool after_kernel = false, const int32_t* q_pos = nullptr);
 // Steps 2 and 3 of a layer from one list of work items (one attention launch and one merge launch).
 struct JointPlan {
-    int nq;                                   // query tiles per CTA, both stages
-    int n_tb_i, n_units_i, chunk, n_slots, items_i;                       // important-token stage
-    int Gp_q, Tt_q, n_tb_q, n_units_q, head_blocks_q, n_splits_q, tiles_per_split_q, items_q;   // question stage
+    int n_tb_i, chunk, n_slots, items_i;                                  // important-token stage
+    int Gp_q, Tt_q, n_tb_q, head_blocks_q, n_splits_q, tiles_per_split_q, items_q;   // question stage
     size_t part_bytes_q, part_bytes_i;        // partial results of each stage
 };
 JointPlan plan_joint(int k, int L_q, int L_d, int Hq, int G);
