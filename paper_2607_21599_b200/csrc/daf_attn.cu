@@ -63,6 +63,13 @@ struct AttnArgs {
 __device__ unsigned long long g_trace[8 * 65536];
 DAF_KT_TABLE;
 DAF_KT_READER(daf_dbg_kt_attn)
+// per-CTA clock totals of the first softmax thread: total, wait S, softmax, wait P V + rescale, epilogue, sub-steps
+__device__ long long g_laps[8 * 65536];
+extern "C" int daf_dbg_read_laps(void* host, size_t bytes) {
+    return (int)cudaMemcpyFromSymbol(host, g_laps, bytes < sizeof(g_laps) ? bytes : sizeof(g_laps));
+}
+#define DAF_LAP_DECL long long lap_s = 0, lap_soft = 0, lap_pv = 0, lap_t = clock64(); const long long lap_begin = lap_t
+#define DAF_LAP(acc) do { const long long now_ = clock64(); acc += now_ - lap_t; lap_t = now_; } while (0)
 #define DAF_STAMP(slot)                                                                         \
     do {                                                                                        \
         const unsigned cta_ = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);   \
@@ -70,6 +77,8 @@ DAF_KT_READER(daf_dbg_kt_attn)
     } while (0)
 #else
 #define DAF_STAMP(slot) do {} while (0)
+#define DAF_LAP_DECL do {} while (0)
+#define DAF_LAP(acc) do {} while (0)
 #endif
 
 // One online-softmax step of one query row (one thread) over NCH * 32 keys starting at `key0`: reads the
@@ -389,12 +398,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
     pdl_wait();                // inputs may come from the kernel launched just before (gather / hybrid-cache update)
     pdl_launch_dependents();   // a dependent kernel (the split merge) may start launching; it waits for this grid
 
-    // a CTA of this grid (or an earlier kernel sharing the workspace) has already given up: do nothing
-    __shared__ int skip_cta;
-    if (threadIdx.x == 0) skip_cta = (args.status != nullptr && *reinterpret_cast<volatile int*>(&args.status->code) != 0) ? 1 : 0;
-    __syncthreads();
-    if (skip_cta) return;
-
     if (threadIdx.x == 0) DAF_STAMP(0);
     DAF_KT_BEGIN(0);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -419,7 +422,22 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
         if (hi > key_begin) n_t = (int)((hi - key_begin + kSubN - 1) / kSubN);
     }
 
-    if (threadIdx.x == 0) {
+    // Loads K (kv = 0) or V (kv = 1) of sub-step t into its ring slot (the slot must be free).
+    auto issue_kv = [&](int t, int kv) {
+        const int slot = t & 1;
+        uint64_t* full = kv == 0 ? &sm->k_full[slot] : &sm->v_full[slot];
+        unsigned char* dst = (kv == 0 ? k_smem : v_smem) + (size_t)slot * kSubBytes;
+        const CUtensorMap* tm = kv == 0 ? tmap_k : tmap_v;
+        const int key0 = key_begin + t * kSubN;
+        mbar_arrive_expect_tx(full, (uint32_t)kSubBytes);
+        tma_load_3d(dst, tm, full, 0, g_kv, key0);
+        tma_load_3d(dst + kSubHalfBytes, tm, full, 64, g_kv, key0);
+    };
+    // Set-up.  The producer thread prepares the barriers and at once starts the loads that need no free
+    // slot (Q and the first two sub-steps), so that their latency overlaps the rest of the set-up: the
+    // status check (a global read) and the tensor-memory allocation.
+    __shared__ int skip_cta;
+    if (warp == 4 && lane == 0) {
         mbar_init(&sm->q_full, 1);
         for (int s = 0; s < 2; ++s) {
             mbar_init(&sm->k_full[s], 1); mbar_init(&sm->k_empty[s], 1);
@@ -429,7 +447,18 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
         mbar_init(&sm->pv_done, 1);
         sm->abort_flag = 0;
         mbar_fence_init();
+        if (n_t > 0) {
+            tma_prefetch_desc(tmap_q);
+            tma_prefetch_desc(tmap_k);
+            tma_prefetch_desc(tmap_v);
+            mbar_arrive_expect_tx(&sm->q_full, 2u * 128u * (uint32_t)(a.Gp * a.Tt));
+            tma_load_3d(q_smem, tmap_q, &sm->q_full, 0, h0, t0);
+            tma_load_3d(q_smem + kHalfBytes, tmap_q, &sm->q_full, 64, h0, t0);
+            for (int t = 0; t < 2 && t < n_t; ++t) { issue_kv(t, 0); issue_kv(t, 1); }
+        }
     }
+    // a CTA of this grid (or an earlier kernel sharing the workspace) has already given up: do nothing
+    if (threadIdx.x == 0) skip_cta = (status != nullptr && *reinterpret_cast<volatile int*>(&status->code) != 0) ? 1 : 0;
     if (warp == 5) {
         tmem_alloc(&sm->tmem_base, kAttnTmemCols);
         tmem_relinquish();
@@ -439,32 +468,29 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
     tc_fence_after();
     const uint32_t tmem = sm->tmem_base;
     volatile int* abort_flag = &sm->abort_flag;
+    const bool skip = skip_cta != 0;
     if (threadIdx.x == 0) DAF_STAMP(1);
 
-    if (warp == 4) {
-        // ------------------------------------------------------------ TMA producer
-        if (lane == 0 && n_t > 0) {
-            tma_prefetch_desc(tmap_q);
-            tma_prefetch_desc(tmap_k);
-            tma_prefetch_desc(tmap_v);
-            mbar_arrive_expect_tx(&sm->q_full, 2u * 128u * (uint32_t)(a.Gp * a.Tt));
-            tma_load_3d(q_smem, tmap_q, &sm->q_full, 0, h0, t0);
-            tma_load_3d(q_smem + kHalfBytes, tmap_q, &sm->q_full, 64, h0, t0);
+    if (skip) {
+        // nothing is computed; the loads already under way get a bounded chance to land before the CTA retires
+        if (warp == 4 && lane == 0 && n_t > 0) {
+            for (int i = 0; i < 4096 && !mbar_try_wait(&sm->q_full, 0); ++i) {}
+            for (int s = 0; s < 2 && s < n_t; ++s) {
+                for (int i = 0; i < 4096 && !mbar_try_wait(&sm->k_full[s], 0); ++i) {}
+                for (int i = 0; i < 4096 && !mbar_try_wait(&sm->v_full[s], 0); ++i) {}
+            }
+        }
+    } else if (warp == 4) {
+        // ------------------------------------------------------------ TMA producer (the rest of the sub-steps)
+        if (lane == 0 && n_t > 2) {
             bool ok = true;
-            for (int t = 0; t < n_t && ok; ++t) {
+            for (int t = 2; t < n_t && ok; ++t) {
                 const int slot = t & 1;
                 const uint32_t round = (uint32_t)(t >> 1);
-                const int key0 = key_begin + t * kSubN;
                 for (int kv = 0; kv < 2 && ok; ++kv) {
                     uint64_t* empty = kv == 0 ? &sm->k_empty[slot] : &sm->v_empty[slot];
-                    uint64_t* full = kv == 0 ? &sm->k_full[slot] : &sm->v_full[slot];
-                    if (round > 0) ok = mbar_wait(empty, (round - 1) & 1u, abort_flag, status, 10 + 2 * kv + slot);
-                    if (!ok) break;
-                    unsigned char* dst = (kv == 0 ? k_smem : v_smem) + (size_t)slot * kSubBytes;
-                    const CUtensorMap* tm = kv == 0 ? tmap_k : tmap_v;
-                    mbar_arrive_expect_tx(full, (uint32_t)kSubBytes);
-                    tma_load_3d(dst, tm, full, 0, g_kv, key0);
-                    tma_load_3d(dst + kSubHalfBytes, tm, full, 64, g_kv, key0);
+                    ok = mbar_wait(empty, (round - 1) & 1u, abort_flag, status, 10 + 2 * kv + slot);
+                    if (ok) issue_kv(t, kv);
                 }
             }
             if (!ok) {
@@ -546,6 +572,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
 
         float m = -INFINITY, l = 0.f;
         bool ok = true;
+        DAF_LAP_DECL;
         for (int t = 0; t < n_t; ++t) {
             const int b = t & 1;
             ok = mbar_wait(&sm->s_full[b], (uint32_t)((t >> 1) & 1), abort_flag, status, 50 + b);
@@ -553,7 +580,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
             if (!ok) break;
             tc_fence_after();
             if (threadIdx.x == 0 && t == 0) DAF_STAMP(2);
+            DAF_LAP(lap_s);
             const float alpha = softmax_core<2>(s_addr + (uint32_t)(b * kSubN), key_begin + t * kSubN, limit, c, m, l);
+            DAF_LAP(lap_soft);
             if (t > 0) {
                 // O may be touched, and the next product be issued, only once the previous product has completed
                 ok = mbar_wait(&sm->pv_done, (uint32_t)((t - 1) & 1), abort_flag, status, 60);
@@ -565,6 +594,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
             tc_wait_st();
             tc_fence_before();
             mbar_arrive(&sm->p_full[b]);
+            DAF_LAP(lap_pv);
         }
         if (threadIdx.x == 0) DAF_STAMP(3);
         // ---- epilogue
@@ -577,6 +607,16 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
             write_rows(args, a, t0, n_t > 0, row_valid, row_valid_tile, tok, head, h0, q_smem + (size_t)quad * 32 * 256, o_addr,
                        quad, lane, m, l);
         }
+#ifdef DAF_TRACE
+        if (threadIdx.x == 0) {
+            const unsigned cta = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
+            if (cta < 65536u) {
+                long long* t = g_laps + 8 * cta;
+                const long long now = clock64();
+                t[0] = now - lap_begin; t[1] = lap_s; t[2] = lap_soft; t[3] = lap_pv; t[4] = now - lap_t; t[5] = n_t;
+            }
+        }
+#endif
     }
 
     if (threadIdx.x == 0) DAF_STAMP(4);
