@@ -7,6 +7,7 @@
  *                       sequence, hybrid KV-cache update              (items 1, 2)
  *   daf_important_attn  self-attention among the condensed tokens     (item 1)
  *   daf_qd_attn         question rows over the hybrid cache           (item 2)
+ *   daf_imp_qd_attn     the two attention stages from one list of work items (items 1, 2)
  *   daf_fuse            state fusion into the final hidden-state rows (item 3)
  *   daf_full_causal_attn  full recomputation, the comparison path (section
  *                       "Preliminary Results", the full-recompute baseline)
@@ -137,6 +138,23 @@ int daf_important_attn(const daf_params* p, int32_t k,
 int daf_qd_attn(const daf_params* p, const void* q_question, const void* kv_k, const void* kv_v,
                 void* out, int64_t out_row_stride_bytes, const int32_t* dst_rows, float* lse,
                 void* workspace, size_t workspace_bytes, void* stream);
+
+/* Steps 2 and 3 together, the way daf_layer runs them: one attention launch over the work
+ * items of both stages (long causal chains of step 2 and the KV axis of step 3 are cut into
+ * ranges) and one launch that merges the ranges' partial results.  Results equal those of
+ * daf_important_attn + daf_qd_attn up to fp32 summation order.  State fusion (Methods item 3)
+ * is done by the epilogues as in daf_layer:
+ *   q_pack, k_pack, v_pack   the k packed rows left by daf_select
+ *   q_question, kv_k, kv_v   as in daf_qd_attn
+ *   idx      int32 [k] positions of the packed rows; read iff p->fuse_mode == 1
+ *   hidden   bf16, row stride n_q_heads * 256 bytes.  fuse_mode 0: rows 0..k-1 are the
+ *            important rows in position order, rows k..k+L_q-1 the question rows;
+ *            fuse_mode 1: [N rows], important row j at row idx[j], question row i at row L_d + i,
+ *            other rows untouched.
+ * Both k and L_q must be positive (use the single-stage calls otherwise). */
+int daf_imp_qd_attn(const daf_params* p, const void* q_pack, const void* k_pack, const void* v_pack,
+                    const void* q_question, const void* kv_k, const void* kv_v, const int32_t* idx,
+                    void* hidden, void* workspace, size_t workspace_bytes, void* stream);
 
 /* daf_qd_attn for callers that cannot provide a workspace.  (The paper has no
  * counterpart of this entry point; it exists for integration only.)

@@ -178,6 +178,28 @@ int daf_qd_attn(const daf_params* p, const void* q_question, const void* kv_k, c
                             (cudaStream_t)stream);
 }
 
+int daf_imp_qd_attn(const daf_params* p, const void* q_pack, const void* k_pack, const void* v_pack,
+                    const void* q_question, const void* kv_k, const void* kv_v, const int32_t* idx,
+                    void* hidden, void* workspace, size_t workspace_bytes_, void* stream) {
+    ResolvedParams rp;
+    if (int rc = resolve_params(p, &rp)) return rc;
+    Workspace ws;
+    if (int rc = carve_workspace(rp, workspace, workspace_bytes_, &ws)) return rc;
+    if (rp.k <= 0 || rp.L_q <= 0) return DAF_ERR_INVALID_ARG;
+    if (!q_pack || !k_pack || !v_pack || !q_question || !kv_k || !kv_v) return DAF_ERR_INVALID_ARG;
+    if (rp.fuse_mode == 1 && idx == nullptr) return DAF_ERR_INVALID_ARG;
+    const void* ptrs[] = {q_pack, k_pack, v_pack, q_question, kv_k, kv_v, idx};
+    for (const void* ptr : ptrs)
+        if (ptr != nullptr && !aligned16(ptr)) return DAF_ERR_ALIGNMENT;
+    const int64_t row_bytes = (int64_t)rp.Hq * 256;
+    if (int rc = check_out(hidden, row_bytes, rp.Hq)) return rc;
+    char* h = reinterpret_cast<char*>(hidden);
+    const int64_t first_row = rp.fuse_mode == 1 ? rp.L_d : rp.k;
+    return launch_attention_joint(q_pack, k_pack, v_pack, rp.k, h, rp.fuse_mode == 1 ? idx : nullptr, q_question, kv_k, kv_v,
+                                  rp.L_q, rp.L_d, h + first_row * row_bytes, row_bytes, rp.Hq, rp.Hkv, rp.scale, ws.status,
+                                  ws.attn_scratch, ws.attn_bytes, (cudaStream_t)stream, /*after_kernel=*/false);
+}
+
 int daf_blend_attn(const daf_params* p, int32_t n_rows, const void* q_rows, const void* kv_k, const void* kv_v,
                    const int32_t* row_pos, void* out, int64_t out_row_stride_bytes, float* lse,
                    void* workspace, size_t workspace_bytes_, void* stream) {

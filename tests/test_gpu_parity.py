@@ -471,3 +471,37 @@ def test_layer_edge_shapes(L_d, L_q, r, Hq, Hkv, n_sig):
         assert np.array_equal(_f(kv_k), ref["kv_k"]) and np.array_equal(_f(kv_v), ref["kv_v"])
         rows = np.arange(len(ref["row_pos"])) if fuse_mode == 0 else ref["row_pos"]
         _assert_close(hidden[rows], ref["hidden"][rows], f"edge shape L_d={L_d} L_q={L_q} mode={fuse_mode}")
+
+
+@pytest.mark.parametrize("k,L_d,L_q,Hq,Hkv,fuse_mode", [(700, 2000, 70, 8, 2, 0), (922, 3000, 64, 28, 4, 1),
+                                                        (129, 400, 1, 4, 4, 0), (1300, 1300, 260, 4, 1, 1)])
+def test_both_attention_stages_from_one_work_list(k, L_d, L_q, Hq, Hkv, fuse_mode):
+    """daf_imp_qd_attn (the two stages as one launch, ranges merged afterwards) against the oracle of
+    each stage, element by element: ragged last tiles, causal chains long enough to be cut into ranges,
+    several token blocks of question rows, compact and scattered output rows."""
+    dev = "cuda"
+    N = L_d + L_q
+    r = k / L_d
+    p = api.make_params(L_d, L_q, r, Hq, Hkv, fuse_mode=fuse_mode)
+    assert api.daf_num_important(L_d, r) == k
+    ws = api.alloc_workspace(p)
+    qp, kp, vp = _normal((k, Hq, 128), 11), _normal((k, Hkv, 128), 12), _normal((k, Hkv, 128), 13)
+    qq = _normal((L_q, Hq, 128), 14)
+    kv_k, kv_v = _normal((N, Hkv, 128), 15), _normal((N, Hkv, 128), 16)
+    idx = torch.from_numpy(np.sort(np.random.default_rng(5).choice(L_d, k, replace=False)).astype(np.int32))
+    rows = k + L_q if fuse_mode == 0 else N
+    hidden = torch.full((rows, Hq, 128), -9.0, dtype=torch.bfloat16, device=dev)
+    _ok(api.daf_imp_qd_attn(p, qp.to(dev), kp.to(dev), vp.to(dev), qq.to(dev), kv_k.to(dev), kv_v.to(dev), idx.to(dev),
+                            hidden, ws), ws, "daf_imp_qd_attn")
+    scale = 1.0 / math.sqrt(128)
+    ref_i = oracle.important_attn(_f(qp), _f(kp), _f(vp), scale)
+    ref_q = oracle.qd_attn(_f(qq), _f(kv_k), _f(kv_v), L_d, scale)
+    h = hidden.cpu()
+    if fuse_mode == 0:
+        _assert_close(h[:k], ref_i, "important rows")
+        _assert_close(h[k:], ref_q, "question rows")
+    else:
+        _assert_close(h[idx.long()], ref_i, "important rows (scattered)")
+        _assert_close(h[L_d:], ref_q, "question rows")
+        others = np.setdiff1d(np.arange(L_d), idx.numpy())
+        assert torch.all(h[others] == -9.0), "a row that is neither important nor a question row was written"
