@@ -35,7 +35,7 @@ UNIT = "us/layer"
 
 # DRAM bytes per launch of the dominant kernel from the ncu capture summarised under profiles/
 # (dram__bytes_read.sum + dram__bytes_write.sum); None where no capture exists for the workload.
-NCU_TRAFFIC_BYTES = {"c1": 8678400, "c3": 73693440}   # important-token stage, profiles/attn_fwd_kernel_c1_c3.md
+NCU_TRAFFIC_BYTES = {"c1": 21736704, "c3": 147695616}   # joint attention launch, profiles/attn_fwd_kernel_c1_c3.md
 
 
 def _peaks():
