@@ -35,6 +35,7 @@ UNIT = "us/layer"
 
 # DRAM bytes per launch of the dominant kernel from the ncu capture summarised under profiles/
 # (dram__bytes_read.sum + dram__bytes_write.sum); None where no capture exists for the workload.
+Q_IN_PLACE_MIN_K = 4096     # from this many important tokens on, the layer is called without a packed-Q buffer
 NCU_TRAFFIC_BYTES = {"c1": 21736704, "c3": 147695616}   # joint attention launch, profiles/attn_fwd_kernel_c1_c3.md
 
 
@@ -221,15 +222,23 @@ def run_ours(args, w: W.Workload):
     row_bytes = Hq * 256
 
     # All launches below go to torch's current stream (the capture stream while a graph is recorded).
+    # With both stages present the layer needs no packed copy of the Q rows: step 2 can read them in place.
+    # That saves most of the gather traffic but costs each work item a scattered fetch of its Q rows, which
+    # pays off once the items are long (measured: c3, k = 6554: 428 -> 416 us/layer; c1, k = 922: 43 -> 47.5).
+    both = w.k > 0 and w.L_q > 0
+    q_in_place = both and w.k >= Q_IN_PLACE_MIN_K
+
     def layer_call(b: LayerBuffers):
         L = b.L
         api.check(api.daf_layer(p, L["scores"], b.n_sig, L["idx_in"], L["q_fresh"], L["k_fresh"], L["v_fresh"], b.kv_k,
-                                b.kv_v, b.idx_out, b.q_pack, b.k_pack, b.v_pack, b.hidden, None, ws), "daf_layer")
+                                b.kv_v, b.idx_out, None if q_in_place else b.q_pack, b.k_pack, b.v_pack, b.hidden, None, ws),
+                  "daf_layer")
 
-    def st_select(b):
+    def st_select(b, pack_q=False):
         L = b.L
         api.check(api.daf_select(p, L["scores"], b.n_sig, L["idx_in"], L["q_fresh"], L["k_fresh"], L["v_fresh"],
-                                 b.kv_k, b.kv_v, b.idx_out, b.q_pack, b.k_pack, b.v_pack, ws), "daf_select")
+                                 b.kv_k, b.kv_v, b.idx_out, b.q_pack if (pack_q or not q_in_place) else None, b.k_pack, b.v_pack,
+                                 ws), "daf_select")
 
     def st_imp(b):
         api.check(api.daf_important_attn(p, b.k, b.q_pack, b.k_pack, b.v_pack, b.hidden, row_bytes, None, None, ws),
@@ -240,8 +249,8 @@ def run_ours(args, w: W.Workload):
                                   out_offset_bytes=b.k * row_bytes), "daf_qd_attn")
 
     def st_both(b):
-        api.check(api.daf_imp_qd_attn(p, b.q_pack, b.k_pack, b.v_pack, b.L["q_fresh"][w.L_d:], b.kv_k, b.kv_v, b.idx_out,
-                                      b.hidden, ws), "daf_imp_qd_attn")
+        api.check(api.daf_imp_qd_attn(p, None if q_in_place else b.q_pack, b.L["q_fresh"], b.k_pack, b.v_pack,
+                                      b.L["q_fresh"][w.L_d:], b.kv_k, b.kv_v, b.idx_out, b.hidden, ws), "daf_imp_qd_attn")
 
     n_full = min(len(bufs), 4)
     pf = api.make_params(w.N, 0, 1.0, w.n_q_heads, w.n_kv_heads)
@@ -344,12 +353,13 @@ def run_ours(args, w: W.Workload):
         api.check(api.daf_deviation_scores(p, b.L["k_fresh"], b.L["v_fresh"], b.L["k_cached"], b.L["v_cached"],
                                            dev_scores), "daf_deviation_scores")
 
+    for b in bufs:                       # the stand-alone important-token stage below reads packed Q rows
+        st_select(b, pack_q=True)
     us_dev = time_stage(st_dev, bufs)
     us_select = time_stage(st_select, bufs)
     us_imp = time_stage(st_imp, bufs) if w.k > 0 else 0.0
     us_qd = time_stage(st_qd, bufs) if w.L_q > 0 else 0.0
     # the two attention stages the way the layer runs them: one launch over both stages' work items, one merge launch
-    both = w.k > 0 and w.L_q > 0
     us_both = time_stage(st_both, bufs) if both else (us_imp + us_qd)
     # full recompute on the same kernel (comparison path), bounded number of layers
     us_full = time_stage(st_full, bufs[:n_full], reps=3)
@@ -375,7 +385,8 @@ def run_ours(args, w: W.Workload):
     imp_tflops = flops["important"] / (us_imp * 1e-6) / 1e12 if us_imp else 0.0
     qd_tflops = flops["question"] / (us_qd * 1e-6) / 1e12 if us_qd else 0.0
     full_tflops = flops["full"] / (us_full * 1e-6) / 1e12
-    gather_bytes = 2 * w.k * (w.n_q_heads + 2 * w.n_kv_heads) * 256 + (w.k + 2 * w.L_q) * 2 * w.n_kv_heads * 256
+    packed_heads = 2 * w.n_kv_heads + (0 if q_in_place else w.n_q_heads)     # heads of a packed row
+    gather_bytes = 2 * w.k * packed_heads * 256 + (w.k + 2 * w.L_q) * 2 * w.n_kv_heads * 256
     dev_bytes = 4 * w.L_d * w.n_kv_heads * 256 + 4 * w.L_d
 
     both_tflops = daf_flops / (us_both * 1e-6) / 1e12 if us_both else 0.0

@@ -109,7 +109,9 @@ int daf_deviation_scores(const daf_params* p, const void* k_fresh, const void* v
  *            cache on entry.  On exit rows idx hold fresh K/V (if overwrite_doc_kv)
  *            and rows L_d..N-1 hold the fresh question K/V.  Must not alias k_fresh/v_fresh.
  *   idx_out  int32 [k] selected positions, ascending (also written when idx_in is given)
- *   q_pack   [k, n_q_heads, 128]; k_pack, v_pack [k, n_kv_heads, 128]: rows idx of the fresh tensors
+ *   q_pack   [k, n_q_heads, 128]; k_pack, v_pack [k, n_kv_heads, 128]: rows idx of the fresh tensors.
+ *            q_pack may be NULL when no packed copy of the Q rows is wanted (daf_layer and
+ *            daf_imp_qd_attn can read them in place).
  */
 int daf_select(const daf_params* p, const float* scores, int32_t n_sig, const int32_t* idx_in,
                const void* q_fresh, const void* k_fresh, const void* v_fresh,
@@ -144,15 +146,19 @@ int daf_qd_attn(const daf_params* p, const void* q_question, const void* kv_k, c
  * ranges) and one launch that merges the ranges' partial results.  Results equal those of
  * daf_important_attn + daf_qd_attn up to fp32 summation order.  State fusion (Methods item 3)
  * is done by the epilogues as in daf_layer:
- *   q_pack, k_pack, v_pack   the k packed rows left by daf_select
+ *   q_pack, k_pack, v_pack   the k packed rows left by daf_select.  q_pack may be NULL: the Q row of
+ *            packed row j is then read in place, row idx[j] of q_fresh ([>= L_d, n_q_heads, 128]),
+ *            which saves writing and re-reading the largest of the packed tensors but costs every
+ *            work item a scattered fetch; measured on B200 it pays off for k in the thousands
+ *            (k = 6554: -3 % layer time) and not for small k (k = 922: +10 %).
  *   q_question, kv_k, kv_v   as in daf_qd_attn
- *   idx      int32 [k] positions of the packed rows; read iff p->fuse_mode == 1
+ *   idx      int32 [k] positions of the packed rows; read iff p->fuse_mode == 1 or q_pack == NULL
  *   hidden   bf16, row stride n_q_heads * 256 bytes.  fuse_mode 0: rows 0..k-1 are the
  *            important rows in position order, rows k..k+L_q-1 the question rows;
  *            fuse_mode 1: [N rows], important row j at row idx[j], question row i at row L_d + i,
  *            other rows untouched.
  * Both k and L_q must be positive (use the single-stage calls otherwise). */
-int daf_imp_qd_attn(const daf_params* p, const void* q_pack, const void* k_pack, const void* v_pack,
+int daf_imp_qd_attn(const daf_params* p, const void* q_pack, const void* q_fresh, const void* k_pack, const void* v_pack,
                     const void* q_question, const void* kv_k, const void* kv_v, const int32_t* idx,
                     void* hidden, void* workspace, size_t workspace_bytes, void* stream);
 
@@ -201,6 +207,7 @@ int daf_full_causal_attn(const daf_params* p, int32_t n_tokens, const void* q, c
  * epilogues (device pointers; arguments as in daf_select, plus)
  *   hidden       compact: [k+L_q, n_q_heads*128]; scatter: [N, n_q_heads*128]
  *   row_pos_out  optional int32 [k+L_q]
+ *   q_pack       may be NULL when L_q > 0: step 2 then reads its Q rows in place (see daf_imp_qd_attn)
  */
 int daf_layer(const daf_params* p, const float* scores, int32_t n_sig, const int32_t* idx_in,
               const void* q_fresh, const void* k_fresh, const void* v_fresh, void* kv_k, void* kv_v,

@@ -91,7 +91,7 @@ def lib() -> ctypes.CDLL:
         L.daf_qd_attn_static_max_bytes.restype = sz
         L.daf_qd_attn_static_max_bytes.argtypes = []
         L.daf_imp_qd_attn.restype = ctypes.c_int
-        L.daf_imp_qd_attn.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.daf_imp_qd_attn.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.daf_blend_attn.restype = ctypes.c_int
         L.daf_blend_attn.argtypes = [pp, i32, vp, vp, vp, vp, vp, i64, vp, vp, sz, vp]
         L.daf_deviation_scores.restype = ctypes.c_int
@@ -207,9 +207,10 @@ def daf_qd_attn_static_max_bytes() -> int:
     return int(lib().daf_qd_attn_static_max_bytes())
 
 
-def daf_imp_qd_attn(p, q_pack, k_pack, v_pack, q_question, kv_k, kv_v, idx, hidden, workspace, stream=None) -> int:
-    return lib().daf_imp_qd_attn(ctypes.byref(p), _ptr(q_pack), _ptr(k_pack), _ptr(v_pack), _ptr(q_question), _ptr(kv_k),
-                                 _ptr(kv_v), _ptr(idx), _ptr(hidden), _ptr(workspace), _nbytes(workspace), _stream(stream))
+def daf_imp_qd_attn(p, q_pack, q_fresh, k_pack, v_pack, q_question, kv_k, kv_v, idx, hidden, workspace, stream=None) -> int:
+    return lib().daf_imp_qd_attn(ctypes.byref(p), _ptr(q_pack), _ptr(q_fresh), _ptr(k_pack), _ptr(v_pack), _ptr(q_question),
+                                 _ptr(kv_k), _ptr(kv_v), _ptr(idx), _ptr(hidden), _ptr(workspace), _nbytes(workspace),
+                                 _stream(stream))
 
 
 def daf_blend_attn(p, n_rows, q_rows, kv_k, kv_v, row_pos, out, out_row_stride_bytes, lse, workspace, stream=None) -> int:

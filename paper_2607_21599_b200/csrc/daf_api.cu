@@ -94,7 +94,7 @@ static int do_select(const ResolvedParams& rp, const float* scores, int32_t n_si
     if (rp.k > 0) {
         if (scores == nullptr && idx_in == nullptr) return DAF_ERR_INVALID_ARG;
         if (scores != nullptr && idx_out == nullptr) return DAF_ERR_INVALID_ARG;
-        if (!q_fresh || !k_fresh || !v_fresh || !q_pack || !k_pack || !v_pack) return DAF_ERR_INVALID_ARG;
+        if (!q_fresh || !k_fresh || !v_fresh || !k_pack || !v_pack) return DAF_ERR_INVALID_ARG;   // q_pack is optional
         if (rp.overwrite && (!kv_k || !kv_v)) return DAF_ERR_INVALID_ARG;
     }
     if (rp.L_q > 0 && (!k_fresh || !v_fresh || !kv_k || !kv_v)) return DAF_ERR_INVALID_ARG;
@@ -178,7 +178,7 @@ int daf_qd_attn(const daf_params* p, const void* q_question, const void* kv_k, c
                             (cudaStream_t)stream);
 }
 
-int daf_imp_qd_attn(const daf_params* p, const void* q_pack, const void* k_pack, const void* v_pack,
+int daf_imp_qd_attn(const daf_params* p, const void* q_pack, const void* q_fresh, const void* k_pack, const void* v_pack,
                     const void* q_question, const void* kv_k, const void* kv_v, const int32_t* idx,
                     void* hidden, void* workspace, size_t workspace_bytes_, void* stream) {
     ResolvedParams rp;
@@ -186,16 +186,17 @@ int daf_imp_qd_attn(const daf_params* p, const void* q_pack, const void* k_pack,
     Workspace ws;
     if (int rc = carve_workspace(rp, workspace, workspace_bytes_, &ws)) return rc;
     if (rp.k <= 0 || rp.L_q <= 0) return DAF_ERR_INVALID_ARG;
-    if (!q_pack || !k_pack || !v_pack || !q_question || !kv_k || !kv_v) return DAF_ERR_INVALID_ARG;
+    if (!k_pack || !v_pack || !q_question || !kv_k || !kv_v) return DAF_ERR_INVALID_ARG;
+    if (q_pack == nullptr && (q_fresh == nullptr || idx == nullptr)) return DAF_ERR_INVALID_ARG;
     if (rp.fuse_mode == 1 && idx == nullptr) return DAF_ERR_INVALID_ARG;
-    const void* ptrs[] = {q_pack, k_pack, v_pack, q_question, kv_k, kv_v, idx};
+    const void* ptrs[] = {q_pack, q_fresh, k_pack, v_pack, q_question, kv_k, kv_v, idx};
     for (const void* ptr : ptrs)
         if (ptr != nullptr && !aligned16(ptr)) return DAF_ERR_ALIGNMENT;
     const int64_t row_bytes = (int64_t)rp.Hq * 256;
     if (int rc = check_out(hidden, row_bytes, rp.Hq)) return rc;
     char* h = reinterpret_cast<char*>(hidden);
     const int64_t first_row = rp.fuse_mode == 1 ? rp.L_d : rp.k;
-    return launch_attention_joint(q_pack, k_pack, v_pack, rp.k, h, rp.fuse_mode == 1 ? idx : nullptr, q_question, kv_k, kv_v,
+    return launch_attention_joint(q_pack, q_fresh, idx, k_pack, v_pack, rp.k, h, rp.fuse_mode == 1 ? idx : nullptr, q_question, kv_k, kv_v,
                                   rp.L_q, rp.L_d, h + first_row * row_bytes, row_bytes, rp.Hq, rp.Hkv, rp.scale, ws.status,
                                   ws.attn_scratch, ws.attn_bytes, (cudaStream_t)stream, /*after_kernel=*/false);
 }
@@ -270,6 +271,7 @@ int daf_layer(const daf_params* p, const float* scores, int32_t n_sig, const int
     cudaStream_t st = (cudaStream_t)stream;
     if (rp.k + rp.L_q == 0) return DAF_OK;
     if (rp.k > 0 && idx_out == nullptr) return DAF_ERR_INVALID_ARG;
+    if (rp.k > 0 && rp.L_q == 0 && q_pack == nullptr) return DAF_ERR_INVALID_ARG;   // only the joint launch reads Q in place
     const int64_t row_bytes = (int64_t)rp.Hq * 256;
     if (int rc = check_out(hidden, row_bytes, rp.Hq)) return rc;
     if (int rc = do_select(rp, scores, n_sig, idx_in, q_fresh, k_fresh, v_fresh, kv_k, kv_v, idx_out, q_pack, k_pack,
@@ -282,7 +284,7 @@ int daf_layer(const daf_params* p, const float* scores, int32_t n_sig, const int
     const char* qq = reinterpret_cast<const char*>(q_fresh) + (int64_t)rp.L_d * row_bytes;
     const int32_t* dst = rp.fuse_mode == 1 ? idx_out : nullptr;
     if (rp.k > 0 && rp.L_q > 0) {
-        if (int rc = launch_attention_joint(q_pack, k_pack, v_pack, rp.k, h, dst, qq, kv_k, kv_v, rp.L_q, rp.L_d,
+        if (int rc = launch_attention_joint(q_pack, q_fresh, idx_out, k_pack, v_pack, rp.k, h, dst, qq, kv_k, kv_v, rp.L_q, rp.L_d,
                                             h + first_row * row_bytes, row_bytes, rp.Hq, rp.Hkv, rp.scale, ws.status,
                                             ws.attn_scratch, ws.attn_bytes, st, /*after_kernel=*/true)) return rc;
     } else if (rp.L_q > 0) {
@@ -330,6 +332,9 @@ void carve_arena(const ResolvedParams& rp, int n_sig, char* base, Arena* a) {
     a->total = off;
 }
 constexpr int kArenaSignalRows = 8;   // arena is sized for up to this many signal rows
+// From this many important tokens on the host-buffer layer skips the packed copy of the Q rows (step 2 reads
+// them in place): measured faster at k = 6554 (-3 % layer time), slower at k = 922 (+10 %).
+constexpr int kQInPlaceMinK = 4096;
 }  // namespace
 
 size_t daf_layer_host_arena_bytes(const daf_params* p) {
@@ -368,7 +373,8 @@ int daf_layer_host(const daf_params* p, const float* h_scores, int32_t n_sig, co
     DAF_CUDA_TRY(cudaMemcpyAsync(a.kv_k, h_kv_k, kvrow * rp.L_d, cudaMemcpyHostToDevice, st));
     DAF_CUDA_TRY(cudaMemcpyAsync(a.kv_v, h_kv_v, kvrow * rp.L_d, cudaMemcpyHostToDevice, st));
     if (int rc = daf_layer(p, h_scores ? a.scores : nullptr, n_sig, h_scores ? nullptr : a.idx_in, a.q_fresh, a.k_fresh,
-                           a.v_fresh, a.kv_k, a.kv_v, a.idx_out, a.q_pack, a.k_pack, a.v_pack, a.hidden, nullptr, a.ws,
+                           a.v_fresh, a.kv_k, a.kv_v, a.idx_out, (rp.k >= kQInPlaceMinK && rp.L_q > 0) ? nullptr : a.q_pack, a.k_pack,
+                           a.v_pack, a.hidden, nullptr, a.ws,
                            a.ws_bytes, stream)) return rc;
     const size_t hidden_rows = rp.fuse_mode == 1 ? rp.N : rp.k + rp.L_q;
     DAF_CUDA_TRY(cudaMemcpyAsync(h_hidden, a.hidden, qrow * hidden_rows, cudaMemcpyDeviceToHost, st));

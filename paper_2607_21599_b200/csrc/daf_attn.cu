@@ -33,6 +33,11 @@ struct SegArgs {
     int n_tb;           // token blocks = ceil(n_q / Tt)
     int causal_off;     // token t sees keys <= t + causal_off ...
     const int32_t* q_pos; // ... or, when given, keys <= q_pos[t] (ascending positions of the query tokens)
+    // Query rows read in place instead of from a packed copy (Gp == 1 only): query token t is row q_idx[t]
+    // of q_src, a [q_src_rows, Hq, 128] tensor.  q_idx == nullptr: the Q tensor map covers packed rows.
+    const __nv_bfloat16* q_src;
+    const int32_t* q_idx;
+    int q_src_rows;
     // Work items.  A CTA owns one token block (a unit).  Either every unit is cut into the same n_splits
     // KV ranges of tiles_per_split tiles (chunk == 0), or -- packed causal attention only, where unit u
     // sees min(u + 1, n_tb) tiles -- units [g chunk, (g + 1) chunk) are cut into g + 1 balanced ranges
@@ -437,8 +442,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
     // slot (Q and the first two sub-steps), so that their latency overlaps the rest of the set-up: the
     // status check (a global read) and the tensor-memory allocation.
     __shared__ int skip_cta;
+    const int32_t* const q_idx = DAF_SEG(q_idx);     // non-null: the softmax warps fetch the Q rows themselves
     if (warp == 4 && lane == 0) {
-        mbar_init(&sm->q_full, 1);
+        mbar_init(&sm->q_full, q_idx != nullptr ? 4 : 1);
         for (int s = 0; s < 2; ++s) {
             mbar_init(&sm->k_full[s], 1); mbar_init(&sm->k_empty[s], 1);
             mbar_init(&sm->v_full[s], 1); mbar_init(&sm->v_empty[s], 1);
@@ -448,14 +454,42 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
         sm->abort_flag = 0;
         mbar_fence_init();
         if (n_t > 0) {
-            tma_prefetch_desc(tmap_q);
             tma_prefetch_desc(tmap_k);
             tma_prefetch_desc(tmap_v);
-            mbar_arrive_expect_tx(&sm->q_full, 2u * 128u * (uint32_t)(a.Gp * a.Tt));
-            tma_load_3d(q_smem, tmap_q, &sm->q_full, 0, h0, t0);
-            tma_load_3d(q_smem + kHalfBytes, tmap_q, &sm->q_full, 64, h0, t0);
+            if (q_idx == nullptr) {
+                tma_prefetch_desc(tmap_q);
+                mbar_arrive_expect_tx(&sm->q_full, 2u * 128u * (uint32_t)(a.Gp * a.Tt));
+                tma_load_3d(q_smem, tmap_q, &sm->q_full, 0, h0, t0);
+                tma_load_3d(q_smem + kHalfBytes, tmap_q, &sm->q_full, 64, h0, t0);
+            }
             for (int t = 0; t < 2 && t < n_t; ++t) { issue_kv(t, 0); issue_kv(t, 1); }
         }
+    }
+    if (q_idx != nullptr && n_t > 0 && warp < 4) {
+        const int quad = warp;
+        // Q rows of the condensed sequence straight from the unpacked tensor: each warp fetches its 32
+        // rows (16 lanes per 256-byte row) into the layout the TMA load would have produced
+        // (two 64-column halves of 128-byte rows, 16-byte chunks XOR-ed with the row number mod 8).
+        const __nv_bfloat16* q_src = DAF_SEG(q_src);
+        const int q_src_rows = DAF_SEG(q_src_rows), Hq = DAF_SEG(Hq);
+        const int sub = lane >> 4, cidx = lane & 15;
+        uint4 w[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const int tokr = t0 + quad * 32 + 2 * i + sub;
+            w[i] = make_uint4(0u, 0u, 0u, 0u);
+            if (tokr < a.n_q) {
+                const int src = __ldg(q_idx + tokr);
+                if ((unsigned)src < (unsigned)q_src_rows)   // a bad position is reported by the gather kernel
+                    w[i] = __ldg(reinterpret_cast<const uint4*>(q_src + ((size_t)src * Hq + h0) * kD) + cidx);
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const int rr = quad * 32 + 2 * i + sub;
+            *reinterpret_cast<uint4*>(q_smem + (cidx >> 3) * kHalfBytes + rr * 128 + (((cidx & 7) ^ (rr & 7)) << 4)) = w[i];
+        }
+        fence_proxy_async();
     }
     // a CTA of this grid (or an earlier kernel sharing the workspace) has already given up: do nothing
     if (threadIdx.x == 0) skip_cta = (status != nullptr && *reinterpret_cast<volatile int*>(&status->code) != 0) ? 1 : 0;
@@ -570,6 +604,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
         const uint32_t o_addr = tmem + lane_addr + (uint32_t)kBlockN;
         const float c = a.scale_log2;
 
+        if (q_idx != nullptr && n_t > 0 && lane == 0) mbar_arrive(&sm->q_full);   // this warp's Q rows were stored before the set-up barrier
         float m = -INFINITY, l = 0.f;
         bool ok = true;
         DAF_LAP_DECL;
@@ -939,8 +974,9 @@ int launch_attention(const void* q, const void* k, const void* v, int n_q, int n
 
 size_t joint_partial_bytes(const JointPlan& jp) { return jp.part_bytes_q + jp.part_bytes_i; }
 
-int launch_attention_joint(const void* q_imp, const void* k_imp, const void* v_imp, int k, void* out_imp,
-                           const int32_t* dst_rows_imp, const void* q_question, const void* kv_k, const void* kv_v,
+int launch_attention_joint(const void* q_imp, const void* q_fresh, const int32_t* idx, const void* k_imp, const void* v_imp,
+                           int k, void* out_imp, const int32_t* dst_rows_imp, const void* q_question, const void* kv_k,
+                           const void* kv_v,
                            int L_q, int L_d, void* out_question, long long out_row_stride_bytes, int Hq, int Hkv,
                            float scale, DeviceStatus* status, void* scratch, size_t scratch_bytes, cudaStream_t stream,
                            bool after_kernel) {
@@ -949,7 +985,10 @@ int launch_attention_joint(const void* q_imp, const void* k_imp, const void* v_i
     if (joint_partial_bytes(jp) > scratch_bytes) return DAF_ERR_WORKSPACE;
 
     CUtensorMap tq0, tk0, tv0, tq1, tk1, tv1;
-    if (int rc = make_tmap(&tq0, q_imp, k, Hq, 1, kBlockM)) return rc;
+    // without packed Q rows the kernel reads them in place through idx (no tensor map needed for them)
+    const bool gather_q = q_imp == nullptr;
+    if (gather_q && (q_fresh == nullptr || idx == nullptr)) return DAF_ERR_INVALID_ARG;
+    if (int rc = make_tmap(&tq0, gather_q ? q_question : q_imp, gather_q ? L_q : k, Hq, 1, kBlockM)) return rc;
     if (int rc = make_tmap(&tk0, k_imp, k, Hkv, 1, kSubN)) return rc;
     if (int rc = make_tmap(&tv0, v_imp, k, Hkv, 1, kSubN)) return rc;
     if (int rc = make_tmap(&tq1, q_question, L_q, Hq, jp.Gp_q, jp.Tt_q)) return rc;
@@ -972,6 +1011,11 @@ int launch_attention_joint(const void* q_imp, const void* k_imp, const void* v_i
     // important tokens: packed causal attention, long chains cut into balanced ranges
     SegArgs& si = a.seg[0];
     fill_problem(&si, k, k, Hq, G, 1, 0, nullptr, scale, out_imp, out_row_stride_bytes, dst_rows_imp, nullptr);
+    if (gather_q) {
+        si.q_src = reinterpret_cast<const __nv_bfloat16*>(q_fresh);
+        si.q_idx = idx;
+        si.q_src_rows = L_d;
+    }
     si.n_units = jp.n_tb_i;
     si.n_splits = 1; si.tiles_per_split = jp.n_tb_i;
     si.chunk = jp.chunk; si.n_slots = jp.n_slots;

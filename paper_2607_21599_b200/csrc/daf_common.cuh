@@ -60,8 +60,10 @@ struct JointPlan {
 };
 JointPlan plan_joint(int k, int L_q, int L_d, int Hq, int G);
 size_t joint_partial_bytes(const JointPlan& jp);
-int launch_attention_joint(const void* q_imp, const void* k_imp, const void* v_imp, int k, void* out_imp,
-                           const int32_t* dst_rows_imp, const void* q_question, const void* kv_k, const void* kv_v,
+// q_imp == nullptr: the important rows' Q is read in place, row idx[j] of q_fresh
+int launch_attention_joint(const void* q_imp, const void* q_fresh, const int32_t* idx, const void* k_imp, const void* v_imp,
+                           int k, void* out_imp, const int32_t* dst_rows_imp, const void* q_question, const void* kv_k,
+                           const void* kv_v,
                            int L_q, int L_d, void* out_question, long long out_row_stride_bytes, int Hq, int Hkv,
                            float scale, DeviceStatus* status, void* scratch, size_t scratch_bytes, cudaStream_t stream,
                            bool after_kernel);
@@ -183,6 +185,9 @@ __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* m, uin
         ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
         : "memory");
 }
+
+// makes this thread's earlier shared-memory writes visible to the asynchronous proxy (TMA, tensor cores)
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // ---- tcgen05 (5th-generation tensor cores, accumulators in tensor memory)
 __device__ __forceinline__ void tmem_alloc(uint32_t* smem_dst, uint32_t ncols) {

@@ -380,7 +380,7 @@ gather_update_kernel(const GatherArgs a) {
         }
         const size_t qsrc = (size_t)p * a.cq, qdst = (size_t)row * a.cq;
         const size_t ksrc = (size_t)p * a.ckv, kdst = (size_t)row * a.ckv;
-        for (int c = threadIdx.x; c < per_row; c += kRowThreads) {
+        for (int c = (a.q_pack != nullptr ? 0 : a.cq) + threadIdx.x; c < per_row; c += kRowThreads) {   // no packed Q wanted: K, V only
             if (c < a.cq) {
                 a.q_pack[qdst + c] = __ldg(a.q_fresh + qsrc + c);
             } else if (c < a.cq + a.ckv) {

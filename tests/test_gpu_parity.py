@@ -491,8 +491,15 @@ def test_both_attention_stages_from_one_work_list(k, L_d, L_q, Hq, Hkv, fuse_mod
     idx = torch.from_numpy(np.sort(np.random.default_rng(5).choice(L_d, k, replace=False)).astype(np.int32))
     rows = k + L_q if fuse_mode == 0 else N
     hidden = torch.full((rows, Hq, 128), -9.0, dtype=torch.bfloat16, device=dev)
-    _ok(api.daf_imp_qd_attn(p, qp.to(dev), kp.to(dev), vp.to(dev), qq.to(dev), kv_k.to(dev), kv_v.to(dev), idx.to(dev),
-                            hidden, ws), ws, "daf_imp_qd_attn")
+    _ok(api.daf_imp_qd_attn(p, qp.to(dev), None, kp.to(dev), vp.to(dev), qq.to(dev), kv_k.to(dev), kv_v.to(dev),
+                            idx.to(dev), hidden, ws), ws, "daf_imp_qd_attn")
+    # the same with the Q rows read in place: q_fresh holds packed row j at position idx[j], noise elsewhere
+    q_fresh = _normal((L_d, Hq, 128), 17)
+    q_fresh[idx.long()] = qp
+    hidden2 = torch.full((rows, Hq, 128), -9.0, dtype=torch.bfloat16, device=dev)
+    _ok(api.daf_imp_qd_attn(p, None, q_fresh.to(dev), kp.to(dev), vp.to(dev), qq.to(dev), kv_k.to(dev), kv_v.to(dev),
+                            idx.to(dev), hidden2, ws), ws, "daf_imp_qd_attn (Q in place)")
+    assert torch.equal(hidden2, hidden), "reading Q in place must give the same bits as reading the packed copy"
     scale = 1.0 / math.sqrt(128)
     ref_i = oracle.important_attn(_f(qp), _f(kp), _f(vp), scale)
     ref_q = oracle.qd_attn(_f(qq), _f(kv_k), _f(kv_v), L_d, scale)
