@@ -187,21 +187,25 @@ select_topk_kernel(const float* __restrict__ scores, int n_sig, int L_d, int k,
     DAF_KT_END(0);
 }
 
-// ------------------------------------------------ selection, one CTA (small L_d)
-// Latency matters more than bandwidth here (at most 160 KB of keys), so the common sizes run in
-// one CTA with no cluster traffic.  One pass over all keys histograms their top 12 bits and finds
-// the bin that holds the k-th largest key; only the keys of that bin (typically a few per cent)
-// go on to two 10-bit passes that fix the remaining 20 bits; an ordered compaction then emits the
-// positions.
+// ------------------------------------------------ selection, one CTA (up to 16K tokens)
+// Latency matters more than bandwidth here (at most 64 KB of keys), so the common sizes run in one
+// CTA with no cluster traffic.  The keys are first reduced to their offset from the smallest key.  One
+// pass over all keys histograms the top 11 of the bits that offset needs (typically 24-27 of 32, fewer
+// when the scores are close together) with shared-memory atomics and finds the bin that holds the k-th
+// largest key; only the keys of that bin (typically well under one per cent) go on to passes of 9 bits
+// that fix the remaining bits.  Because the offsets of real scores spread over the whole histogram,
+// the atomics rarely collide; scores that are all (nearly) equal collide more, and all of them become
+// candidates, but the result stays correct.  An ordered compaction then emits the positions.
 constexpr int kSel1Threads = 1024;
 constexpr int kSel1Warps = kSel1Threads / 32;
-constexpr int kSel1MaxKeys = 4096;    // capacity of the one-CTA kernel (= candidate list size)
-constexpr int kSel1Bins = 4096;
-constexpr int kSel1CandMax = 4096;
+constexpr int kSel1MaxKeys = 16384;   // capacity of the one-CTA kernel (keys live in shared memory)
+constexpr int kSel1TopBits = 11;      // first pass, over all keys
+constexpr int kSel1TopBins = 1 << kSel1TopBits;
+constexpr int kSel1Bits = 9;          // later passes, over the candidates
+constexpr int kSel1Bins = 1 << kSel1Bits;
 
 struct Sel1Shared {
-    uint32_t hist[kSel1Bins];
-    uint32_t cand[kSel1CandMax];
+    uint32_t hist[kSel1TopBins];
     uint32_t warp_a[kSel1Warps];
     uint32_t warp_b[kSel1Warps];
     uint32_t pick[2];       // chosen digit, remaining rank
@@ -234,94 +238,114 @@ __device__ __forceinline__ void block_excl_scan2(uint32_t a, uint32_t b, uint32_
     __syncthreads();   // wa/wb may be reused by the next scan
 }
 
-// Adds one to hist[bin] for every thread with `in`; a warp whose keys share one bin adds once.
-__device__ __forceinline__ void hist_add(uint32_t* hist, bool in, uint32_t bin) {
-    const int lane = threadIdx.x & 31;
-    const uint32_t active = __ballot_sync(0xFFFFFFFFu, in);
-    if (active == 0u) return;
-    const int leader = __ffs(active) - 1;
-    const uint32_t lead_bin = __shfl_sync(0xFFFFFFFFu, bin, leader);
-    const uint32_t same = __ballot_sync(0xFFFFFFFFu, in && bin == lead_bin);
-    if (same == active) {
-        if (lane == leader) atomicAdd(&hist[lead_bin], (uint32_t)__popc(active));
-    } else if (in) {
-        atomicAdd(&hist[bin], 1u);
-    }
-}
-
 // Finds, from the top, the bin in which the k_rem-th element falls.  Thread t owns `per` consecutive
 // bins in descending order; the result goes to pick[0] (bin) and pick[1] (rank inside that bin).
 __device__ __forceinline__ void pick_bin(Sel1Shared* sh, int n_bins, int per) {
-    const int tid = threadIdx.x;
-    const int top = n_bins - 1 - tid * per;   // this thread's highest bin
-    uint32_t s = 0;
+    const int top = n_bins - 1 - (int)threadIdx.x * per;   // this thread's highest bin
+    uint32_t c = 0;
     if (top >= 0)
-        for (int b = 0; b < per; ++b) s += sh->hist[top - b];
+        for (int b = 0; b < per; ++b) c += sh->hist[top - b];
     uint32_t above, dummy, tot, tot2;
-    block_excl_scan2(s, 0u, sh->warp_a, sh->warp_b, above, dummy, tot, tot2);
+    block_excl_scan2(c, 0u, sh->warp_a, sh->warp_b, above, dummy, tot, tot2);
     const uint32_t k_rem = sh->pick[1];
-    if (top >= 0 && k_rem > above && k_rem <= above + s) {
-        uint32_t a = above;
+    if (top >= 0 && k_rem > above && k_rem <= above + c) {
+        uint32_t acc = above;
         for (int b = 0; b < per; ++b) {
-            const uint32_t c = sh->hist[top - b];
-            if (k_rem <= a + c) { sh->pick[0] = (uint32_t)(top - b); sh->pick[1] = k_rem - a; break; }
-            a += c;
+            const uint32_t cb = sh->hist[top - b];
+            if (k_rem <= acc + cb) { sh->pick[0] = (uint32_t)(top - b); sh->pick[1] = k_rem - acc; break; }
+            acc += cb;
         }
     }
     __syncthreads();
 }
+
+// Keys sit in shared memory with one word of padding per 32, so that both access patterns are free of bank
+// conflicts: consecutive threads reading consecutive keys, and each thread walking its own run of keys.
+__host__ __device__ __forceinline__ int padded(int i) { return i + (i >> 5); }
 
 __global__ void __launch_bounds__(kSel1Threads, 1)
 select_topk_cta_kernel(const float* __restrict__ scores, int n_sig, int L_d, int k, int32_t* __restrict__ idx_out) {
     extern __shared__ __align__(16) unsigned char sel_smem[];
     Sel1Shared* sh = reinterpret_cast<Sel1Shared*>(sel_smem);
     uint32_t* keys = reinterpret_cast<uint32_t*>(sel_smem + sizeof(Sel1Shared));
-    const int tid = threadIdx.x;
+    uint32_t* cand = keys + padded(L_d);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    DAF_KT_BEGIN(0);
     pdl_launch_dependents();   // the gather kernel may start launching; it waits for this grid before reading idx
 
-    for (int i = tid; i < kSel1Bins; i += kSel1Threads) sh->hist[i] = 0u;
+    // aggregate the signal rows in ascending row order (fp32 adds, no fusing), build keys, find their range
+    // (eight loads in flight per thread: one load per trip would serialise on memory latency)
+    uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
+    for (int base = tid; base < L_d; base += 8 * kSel1Threads) {
+        float acc[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int i = base + u * kSel1Threads;
+            acc[u] = i < L_d ? scores[i] : 0.f;
+        }
+        for (int l = 1; l < n_sig; ++l) {
+            float nxt[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int i = base + u * kSel1Threads;
+                nxt[u] = i < L_d ? scores[(size_t)l * L_d + i] : 0.f;
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) acc[u] = __fadd_rn(acc[u], nxt[u]);
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int i = base + u * kSel1Threads;
+            if (i < L_d) {
+                const uint32_t key = score_key(acc[u]);
+                keys[padded(i)] = key;
+                kmin = min(kmin, key);
+                kmax = max(kmax, key);
+            }
+        }
+    }
+    for (int i = tid; i < kSel1TopBins; i += kSel1Threads) sh->hist[i] = 0u;
     if (tid == 0) { sh->pick[0] = 0u; sh->pick[1] = (uint32_t)k; sh->n_cand = 0u; }
+    kmin = __reduce_min_sync(0xFFFFFFFFu, kmin);
+    kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
+    if (lane == 0) { sh->warp_a[warp] = kmin; sh->warp_b[warp] = kmax; }
     __syncthreads();
-    // pass 1 over all keys: aggregate the signal rows in ascending row order, build keys, histogram bits [31:20]
-    const int n_round = (L_d + 31) / 32 * 32;
-    for (int i = tid; i < n_round; i += kSel1Threads) {
-        uint32_t key = 0u;
-        if (i < L_d) {
-            float acc = scores[i];
-            for (int l = 1; l < n_sig; ++l) acc = __fadd_rn(acc, scores[(size_t)l * L_d + i]);
-            key = score_key(acc);
-            keys[i] = key;
-        }
-        hist_add(sh->hist, i < L_d, key >> 20);
-    }
+    kmin = __reduce_min_sync(0xFFFFFFFFu, sh->warp_a[lane]);
+    kmax = __reduce_max_sync(0xFFFFFFFFu, sh->warp_b[lane]);
+    __syncthreads();   // warp_a/warp_b are reused by the scans below
+    const uint32_t range = kmax - kmin;
+    const int bits = 32 - __clz((int)range);        // bits the offsets need (0 when all keys are equal)
+    const int low_bits = max(bits - kSel1TopBits, 0);   // bits left after the first pass
+
+    // first pass, all keys: the top bits of the offset
+    for (int i = tid; i < L_d; i += kSel1Threads) atomicAdd(&sh->hist[(keys[padded(i)] - kmin) >> low_bits], 1u);
     __syncthreads();
-    pick_bin(sh, kSel1Bins, kSel1Bins / kSel1Threads);
-    const uint32_t d1 = sh->pick[0];
-    // candidates: keys whose top 12 bits equal d1
+    pick_bin(sh, kSel1TopBins, kSel1TopBins / kSel1Threads);
+    const uint32_t top_digit = sh->pick[0];
+    // candidates: the low bits of the keys that fall in the chosen bin
     for (int i = tid; i < L_d; i += kSel1Threads) {
-        const uint32_t key = keys[i];
-        if ((key >> 20) == d1) {
-            sh->cand[atomicAdd(&sh->n_cand, 1u)] = key;
-        }
+        const uint32_t off = keys[padded(i)] - kmin;
+        if ((off >> low_bits) == top_digit) cand[atomicAdd(&sh->n_cand, 1u)] = low_bits > 0 ? off & ((1u << low_bits) - 1u) : 0u;
     }
-    for (int i = tid; i < 1024; i += kSel1Threads) sh->hist[i] = 0u;
+    if (tid < kSel1Bins) sh->hist[tid] = 0u;
     __syncthreads();
-    const int n_cand = (int)sh->n_cand;    // at most L_d <= kSel1CandMax, so the list never overflows
-    uint32_t prefix = d1 << 20, mask = 0xFFF00000u;
-    for (int shift = 10; shift >= 0; shift -= 10) {
-        const int n_c_round = (n_cand + 31) / 32 * 32;
-        for (int i = tid; i < n_c_round; i += kSel1Threads) {
-            const uint32_t key = i < n_cand ? sh->cand[i] : 0u;
-            hist_add(sh->hist, i < n_cand && (key & mask) == prefix, (key >> shift) & 0x3FFu);
+    const int n_cand = (int)sh->n_cand;    // at most L_d, the capacity of the list
+    const int passes = (low_bits + kSel1Bits - 1) / kSel1Bits;
+    uint32_t prefix = 0u;      // the low digits fixed so far
+    for (int p = 0; p < passes; ++p) {
+        const int shift = (passes - 1 - p) * kSel1Bits;
+        for (int i = tid; i < n_cand; i += kSel1Threads) {
+            const uint32_t low = cand[i];
+            if ((low >> (shift + kSel1Bits)) == prefix) atomicAdd(&sh->hist[(low >> shift) & (kSel1Bins - 1)], 1u);
         }
         __syncthreads();
-        pick_bin(sh, 1024, 1);
-        prefix |= sh->pick[0] << shift;
-        mask |= 0x3FFu << shift;
-        if (tid < 1024) sh->hist[tid] = 0u;
+        pick_bin(sh, kSel1Bins, 1);
+        prefix = (prefix << kSel1Bits) | sh->pick[0];
+        if (tid < kSel1Bins) sh->hist[tid] = 0u;
         __syncthreads();
     }
-    const uint32_t thr = prefix;           // key of the k-th largest score
+    prefix |= top_digit << low_bits;       // the whole offset of the threshold (passes == 0: the top digit alone)
+    const uint32_t thr = kmin + prefix;    // key of the k-th largest score (passes == 0: every key equals kmin)
     const uint32_t need_eq = sh->pick[1];  // how many keys equal to thr are taken (lowest positions first)
 
     // ordered compaction: thread t owns the contiguous positions [t*E, (t+1)*E)
@@ -329,7 +353,7 @@ select_topk_cta_kernel(const float* __restrict__ scores, int n_sig, int L_d, int
     const int lo = min(L_d, tid * E), hi = min(L_d, lo + E);
     uint32_t n_gt = 0, n_eq = 0;
     for (int i = lo; i < hi; ++i) {
-        const uint32_t key = keys[i];
+        const uint32_t key = keys[padded(i)];
         n_gt += key > thr;
         n_eq += key == thr;
     }
@@ -338,12 +362,13 @@ select_topk_cta_kernel(const float* __restrict__ scores, int n_sig, int L_d, int
     if (k > 0) {
         uint32_t pos = gt_before + min(eq_before, need_eq);
         for (int i = lo; i < hi; ++i) {
-            const uint32_t key = keys[i];
+            const uint32_t key = keys[padded(i)];
             bool take = key > thr;
             if (key == thr) { take = eq_before < need_eq; ++eq_before; }
             if (take) idx_out[pos++] = i;
         }
     }
+    DAF_KT_END(0);
 }
 
 // --------------------------------------------------- gather + hybrid KV update
@@ -466,9 +491,9 @@ deviation_scores_kernel(const int4* __restrict__ k_fresh, const int4* __restrict
 }
 
 // ----------------------------------------------------------------- host side
-// Measured on B200: one CTA is faster up to about 2K tokens (3.8 vs 6.5 us at 1K); from 6K on the cluster's eight
-// histogram engines win (7.8 vs 18 us at 16K).
-static int g_sel1_max_keys = 2048;   // sizes up to this run in one CTA, larger ones in the cluster kernel
+// Measured on B200 (selection alone): one CTA 5.1 / 6.9 / 6.8 / 9.9 us at 1K / 6K / 8K / 16K tokens, the cluster
+// of eight 7.6 / 8.4 / 8.4 / 9.0 us: one CTA up to 8K tokens, the cluster beyond.
+static int g_sel1_max_keys = 8192;
 #ifdef DAF_TRACE
 extern "C" void daf_dbg_sel1_max_keys(int n) { g_sel1_max_keys = n < kSel1MaxKeys ? n : kSel1MaxKeys; }
 #endif
@@ -497,12 +522,12 @@ int launch_select(const ResolvedParams& rp, const float* scores, int n_sig, cons
                                                  (int)(sizeof(SelShared) + (size_t)kSelSmemKeysPerCta * sizeof(uint32_t)));
             if (e == cudaSuccess)
                 e = cudaFuncSetAttribute(select_topk_cta_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)(sizeof(Sel1Shared) + (size_t)kSel1MaxKeys * sizeof(uint32_t)));
+                                         (int)(sizeof(Sel1Shared) + ((size_t)padded(kSel1MaxKeys) + kSel1MaxKeys) * sizeof(uint32_t)));
             if (e != cudaSuccess) { set_cuda_error(e); return DAF_ERR_CUDA; }
             attr_done[dev] = true;
         }
         if (rp.L_d <= g_sel1_max_keys) {
-            const size_t smem1 = sizeof(Sel1Shared) + (size_t)rp.L_d * sizeof(uint32_t);
+            const size_t smem1 = sizeof(Sel1Shared) + ((size_t)padded(rp.L_d) + rp.L_d) * sizeof(uint32_t);   // keys and candidate list
             select_topk_cta_kernel<<<1, kSel1Threads, smem1, stream>>>(scores, n_sig, rp.L_d, rp.k, idx_out);
         } else {
             const size_t smem = select_smem_bytes(rp.L_d);

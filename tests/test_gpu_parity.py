@@ -58,7 +58,8 @@ def _normal(shape, seed, scale=1.0):
     (32768, 0.20, 1, "pareto"), (1000, 0.1, 2, "ties"), (777, 1.0, 1, "lognormal"), (130, 0.5, 1, "special"),
     (50000, 0.07, 1, "lognormal"), (33, 0.03, 1, "ties"), (4096, 0.25, 1, "constant"),
     (16384, 0.10, 1, "constant"), (20000, 0.3, 2, "ties"), (40960, 0.2, 1, "lognormal"), (40961, 0.2, 1, "lognormal"),
-    (7, 0.5, 1, "lognormal"), (1, 1.0, 1, "lognormal"),
+    (7, 0.5, 1, "lognormal"), (1, 1.0, 1, "lognormal"), (12000, 0.2, 1, "special"), (16384, 0.5, 1, "ties"),
+    (16385, 0.5, 1, "ties"), (2048, 0.05, 1, "narrow"),
 ])
 def test_select_indices_bit_exact(L_d, r, n_sig, kind):
     if kind == "pareto":
@@ -71,6 +72,8 @@ def test_select_indices_bit_exact(L_d, r, n_sig, kind):
             S = torch.round(S * 2) / 2
         if kind == "constant":
             S = torch.full_like(S, 1.5)
+        if kind == "narrow":      # scores within a few ulps of each other: the key range needs only a few bits
+            S = 1.0 + torch.floor(S * 4) * 2.0 ** -22
         if kind == "special":
             S[0, 3] = float("nan"); S[0, 4] = float("inf"); S[0, 5] = -float("inf")
             S[0, 6] = 0.0; S[0, 7] = -0.0; S[0, 8] = float("nan"); S[0, 9:40] = -S[0, 9:40]
