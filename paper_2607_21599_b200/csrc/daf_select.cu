@@ -37,6 +37,10 @@ __device__ __forceinline__ uint32_t score_key(float s) {
     return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
 
+// Keys sit in shared memory with one word of padding per 32, so that both access patterns are free of bank
+// conflicts: consecutive threads reading consecutive keys, and each thread walking its own run of keys.
+__host__ __device__ __forceinline__ int padded(int i) { return i + (i >> 5); }
+
 struct SelShared {
     uint32_t hist[2][256];     // double-buffered so that a peer may still read pass p while pass p+1 is filled
     uint32_t total[256];
@@ -62,14 +66,16 @@ select_topk_kernel(const float* __restrict__ scores, int n_sig, int L_d, int k,
     const int per_cta = (L_d + kSelCluster - 1) / kSelCluster;
     const int lo_cta = min(L_d, rank * per_cta);
     const int n_loc = min(L_d, lo_cta + per_cta) - lo_cta;
-    uint32_t* keys = (per_cta <= kSelSmemKeysPerCta) ? skeys : (gkeys + lo_cta);
+    const bool in_smem = per_cta <= kSelSmemKeysPerCta;
+    uint32_t* keys = in_smem ? skeys : (gkeys + lo_cta);
+    auto at = [&](int i) { return in_smem ? padded(i) : i; };   // padded layout in shared memory only
 
     // aggregate the signal rows in ascending row order (fp32 adds, no fusing) and build keys
     for (int i = tid; i < n_loc; i += kSelThreads) {
         const int g = lo_cta + i;
         float acc = scores[g];
         for (int l = 1; l < n_sig; ++l) acc = __fadd_rn(acc, scores[(size_t)l * L_d + g]);
-        keys[i] = score_key(acc);
+        keys[at(i)] = score_key(acc);
     }
     if (tid < 256) { sh->hist[0][tid] = 0u; sh->hist[1][tid] = 0u; }
     if (tid == 0) { sh->pick[0] = 0u; sh->pick[1] = (uint32_t)k; }
@@ -84,7 +90,7 @@ select_topk_kernel(const float* __restrict__ scores, int n_sig, int L_d, int k,
             bool in = false;
             uint32_t bin = 0u;
             if (i < n_loc) {
-                const uint32_t key = keys[i];
+                const uint32_t key = keys[at(i)];
                 in = (key & mask) == prefix;
                 bin = (key >> shift) & 0xFFu;
             }
@@ -145,7 +151,7 @@ select_topk_kernel(const float* __restrict__ scores, int n_sig, int L_d, int k,
     const int lo = min(n_loc, tid * E), hi = min(n_loc, lo + E);
     uint32_t n_gt = 0, n_eq = 0;
     for (int i = lo; i < hi; ++i) {
-        const uint32_t key = keys[i];
+        const uint32_t key = keys[at(i)];
         n_gt += key > thr;
         n_eq += key == thr;
     }
@@ -177,7 +183,7 @@ select_topk_kernel(const float* __restrict__ scores, int n_sig, int L_d, int k,
     if (k > 0) {
         uint32_t pos = gt_before + min(eq_before, need_eq);
         for (int i = lo; i < hi; ++i) {
-            const uint32_t key = keys[i];
+            const uint32_t key = keys[at(i)];
             bool take = key > thr;
             if (key == thr) { take = eq_before < need_eq; ++eq_before; }
             if (take) idx_out[pos++] = lo_cta + i;
@@ -258,10 +264,6 @@ __device__ __forceinline__ void pick_bin(Sel1Shared* sh, int n_bins, int per) {
     }
     __syncthreads();
 }
-
-// Keys sit in shared memory with one word of padding per 32, so that both access patterns are free of bank
-// conflicts: consecutive threads reading consecutive keys, and each thread walking its own run of keys.
-__host__ __device__ __forceinline__ int padded(int i) { return i + (i >> 5); }
 
 __global__ void __launch_bounds__(kSel1Threads, 1)
 select_topk_cta_kernel(const float* __restrict__ scores, int n_sig, int L_d, int k, int32_t* __restrict__ idx_out) {
@@ -505,7 +507,7 @@ size_t select_scratch_bytes(int L_d) {
 
 static size_t select_smem_bytes(int L_d) {
     const int per_cta = (L_d + kSelCluster - 1) / kSelCluster;
-    return sizeof(SelShared) + (per_cta <= kSelSmemKeysPerCta ? (size_t)per_cta * sizeof(uint32_t) : 0);
+    return sizeof(SelShared) + (per_cta <= kSelSmemKeysPerCta ? (size_t)padded(per_cta) * sizeof(uint32_t) : 0);
 }
 
 int launch_select(const ResolvedParams& rp, const float* scores, int n_sig, const int32_t* idx_in,
@@ -519,7 +521,7 @@ int launch_select(const ResolvedParams& rp, const float* scores, int n_sig, cons
         cudaGetDevice(&dev);
         if (dev >= 0 && dev < 64 && !attr_done[dev]) {
             cudaError_t e = cudaFuncSetAttribute(select_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                 (int)(sizeof(SelShared) + (size_t)kSelSmemKeysPerCta * sizeof(uint32_t)));
+                                                 (int)(sizeof(SelShared) + (size_t)padded(kSelSmemKeysPerCta) * sizeof(uint32_t)));
             if (e == cudaSuccess)
                 e = cudaFuncSetAttribute(select_topk_cta_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)(sizeof(Sel1Shared) + ((size_t)padded(kSel1MaxKeys) + kSel1MaxKeys) * sizeof(uint32_t)));
