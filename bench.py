@@ -35,7 +35,7 @@ UNIT = "us/layer"
 
 # DRAM bytes per launch of the dominant kernel from the ncu capture summarised under profiles/
 # (dram__bytes_read.sum + dram__bytes_write.sum); None where no capture exists for the workload.
-Q_IN_PLACE_MIN_K = 4096     # from this many important tokens on, the layer is called without a packed-Q buffer
+Q_IN_PLACE_MIN_K = 16384    # from this many important tokens on, the layer is called without a packed-Q buffer
 NCU_TRAFFIC_BYTES = {"c1": 21736704, "c3": 147695616}   # joint attention launch, profiles/attn_fwd_kernel_c1_c3.md
 
 
@@ -223,8 +223,9 @@ def run_ours(args, w: W.Workload):
 
     # All launches below go to torch's current stream (the capture stream while a graph is recorded).
     # With both stages present the layer needs no packed copy of the Q rows: step 2 can read them in place.
-    # That saves most of the gather traffic but costs each work item a scattered fetch of its Q rows, which
-    # pays off once the items are long (measured: c3, k = 6554: 428 -> 416 us/layer; c1, k = 922: 43 -> 47.5).
+    # That saves most of the gather traffic but costs each work item a scattered fetch of its Q rows; measured
+    # on B200 the layer time changes by -2 % (k = 41780), +-1 % (k = 6554) and +10 % (k = 922), so only very
+    # long condensed sequences are run that way.
     both = w.k > 0 and w.L_q > 0
     q_in_place = both and w.k >= Q_IN_PLACE_MIN_K
 

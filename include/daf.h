@@ -149,8 +149,8 @@ int daf_qd_attn(const daf_params* p, const void* q_question, const void* kv_k, c
  *   q_pack, k_pack, v_pack   the k packed rows left by daf_select.  q_pack may be NULL: the Q row of
  *            packed row j is then read in place, row idx[j] of q_fresh ([>= L_d, n_q_heads, 128]),
  *            which saves writing and re-reading the largest of the packed tensors but costs every
- *            work item a scattered fetch; measured on B200 it pays off for k in the thousands
- *            (k = 6554: -3 % layer time) and not for small k (k = 922: +10 %).
+ *            work item a scattered fetch; measured on B200 the layer time changes by -2 % at
+ *            k = 41780, +-1 % at k = 6554 and +10 % at k = 922.
  *   q_question, kv_k, kv_v   as in daf_qd_attn
  *   idx      int32 [k] positions of the packed rows; read iff p->fuse_mode == 1 or q_pack == NULL
  *   hidden   bf16, row stride n_q_heads * 256 bytes.  fuse_mode 0: rows 0..k-1 are the

@@ -333,8 +333,8 @@ void carve_arena(const ResolvedParams& rp, int n_sig, char* base, Arena* a) {
 }
 constexpr int kArenaSignalRows = 8;   // arena is sized for up to this many signal rows
 // From this many important tokens on the host-buffer layer skips the packed copy of the Q rows (step 2 reads
-// them in place): measured faster at k = 6554 (-3 % layer time), slower at k = 922 (+10 %).
-constexpr int kQInPlaceMinK = 4096;
+// them in place): measured -2 % layer time at k = 41780, +-1 % at k = 6554, +10 % at k = 922.
+constexpr int kQInPlaceMinK = 16384;
 }  // namespace
 
 size_t daf_layer_host_arena_bytes(const daf_params* p) {

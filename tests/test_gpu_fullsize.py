@@ -80,9 +80,9 @@ def test_layer_at_benchmark_size(name, layer, n_imp_rows, n_q_rows, n_full_rows)
     n_sig = L["scores"].shape[0]
 
     def run():
-        # as the benchmark calls it: from 4096 important tokens on without a packed copy of the Q rows
+        # as the benchmark calls it: from 16384 important tokens on without a packed copy of the Q rows
         api.check(api.daf_layer(p, L["scores"], n_sig, None, L["q_fresh"], L["k_fresh"], L["v_fresh"], kv_k, kv_v,
-                                idx_out, None if k >= 4096 else q_pack, k_pack, v_pack, hidden, None, ws), "daf_layer")
+                                idx_out, None if k >= 16384 else q_pack, k_pack, v_pack, hidden, None, ws), "daf_layer")
 
     run()  # eager once (sets kernel attributes), then the timed configuration: a graph replay
     torch.cuda.synchronize()
