@@ -515,3 +515,52 @@ def test_both_attention_stages_from_one_work_list(k, L_d, L_q, Hq, Hkv, fuse_mod
         _assert_close(h[L_d:], ref_q, "question rows")
         others = np.setdiff1d(np.arange(L_d), idx.numpy())
         assert torch.all(h[others] == -9.0), "a row that is neither important nor a question row was written"
+
+
+@pytest.mark.parametrize("fuse_mode", [0, 1])
+def test_layer_without_packed_q_buffer(fuse_mode):
+    """daf_layer with q_pack = NULL (step 2 reads its Q rows in place) gives the same bits as with the buffer,
+    and daf_select with q_pack = NULL still packs K/V and updates the cache."""
+    w = W.Workload("t", 11, 8, 2, 128, 1, 1500, 500, 70, 0.3, "lognormal", 2)
+    L = W.make_layer(w, 0)
+    dev = "cuda"
+    p = api.make_params(w.L_d, w.L_q, w.r, w.n_q_heads, w.n_kv_heads, fuse_mode=fuse_mode)
+    k = api.daf_num_important(w.L_d, w.r)
+    g = {n: (None if t is None else t.to(dev)) for n, t in L.items()}
+    rows = k + w.L_q if fuse_mode == 0 else w.N
+    outs = []
+    for with_q in (True, False):
+        ws = api.alloc_workspace(p)
+        kv_k = torch.zeros(w.N, w.n_kv_heads, 128, dtype=torch.bfloat16, device=dev)
+        kv_v = torch.zeros_like(kv_k)
+        kv_k[: w.L_d], kv_v[: w.L_d] = g["k_cached"], g["v_cached"]
+        idx_out = torch.full((k,), -1, dtype=torch.int32, device=dev)
+        qp = torch.full((k, w.n_q_heads, 128), 7.0, dtype=torch.bfloat16, device=dev)
+        kp = torch.zeros(k, w.n_kv_heads, 128, dtype=torch.bfloat16, device=dev)
+        vp = torch.zeros_like(kp)
+        hidden = torch.full((rows, w.n_q_heads, 128), -9.0, dtype=torch.bfloat16, device=dev)
+        _ok(api.daf_layer(p, g["scores"], 2, None, g["q_fresh"], g["k_fresh"], g["v_fresh"], kv_k, kv_v, idx_out,
+                          qp if with_q else None, kp, vp, hidden, None, ws), ws, "daf_layer")
+        outs.append((hidden.cpu(), idx_out.cpu(), kp.cpu(), vp.cpu(), kv_k.cpu(), kv_v.cpu()))
+        if with_q:
+            assert torch.equal(qp.cpu(), L["q_fresh"][idx_out.cpu().long()])
+    for a, b in zip(outs[0], outs[1]):
+        assert torch.equal(a, b)
+    ref = _oracle_layer(w, L, fuse_mode)
+    hid = outs[1][0]
+    if fuse_mode == 0:
+        _assert_close(hid, ref["hidden"], "hidden rows (compact), Q read in place")
+    else:
+        _assert_close(hid[ref["row_pos"]], ref["hidden"][ref["row_pos"]], "hidden rows (scatter), Q read in place")
+    # the selection step alone, without a packed-Q buffer
+    ws = api.alloc_workspace(p)
+    kv_k = torch.zeros(w.N, w.n_kv_heads, 128, dtype=torch.bfloat16, device=dev)
+    kv_v = torch.zeros_like(kv_k)
+    kv_k[: w.L_d], kv_v[: w.L_d] = g["k_cached"], g["v_cached"]
+    idx_out = torch.full((k,), -1, dtype=torch.int32, device=dev)
+    kp = torch.zeros(k, w.n_kv_heads, 128, dtype=torch.bfloat16, device=dev)
+    vp = torch.zeros_like(kp)
+    _ok(api.daf_select(p, g["scores"], 2, None, g["q_fresh"], g["k_fresh"], g["v_fresh"], kv_k, kv_v, idx_out, None, kp, vp,
+                       ws), ws, "daf_select")
+    assert torch.equal(idx_out.cpu(), outs[0][1]) and torch.equal(kp.cpu(), outs[0][2]) and torch.equal(vp.cpu(), outs[0][3])
+    assert torch.equal(kv_k.cpu(), outs[0][4]) and torch.equal(kv_v.cpu(), outs[0][5])
