@@ -714,8 +714,14 @@ attn_combine_kernel(const CombineSeg s0, const CombineSeg s1) {
     }
     const float* part_o = DAF_CS(part_o);
     const float* part_lse = DAF_CS(part_lse);
-    // lane s holds the log-sum-exp of partial s (at most 32 of them), so all of them are fetched at once
+    // lane s holds the log-sum-exp of partial s (at most 32 of them), so all of them are fetched at once;
+    // the first eight partial rows are requested in the same breath, before the weights are known
+    const float4* src = reinterpret_cast<const float4*>(part_o + first * kD) + lane;
     const float my_lse = lane < n_splits ? part_lse[first + (size_t)lane * stride] : -INFINITY;
+    float4 head_v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u)
+        head_v[u] = u < n_splits ? __ldcs(src + (size_t)u * stride * (kD / 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
     float mx = my_lse;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
@@ -724,8 +730,12 @@ attn_combine_kernel(const CombineSeg s0, const CombineSeg s1) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) wsum += __shfl_xor_sync(0xFFFFFFFFu, wsum, o);
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    const float4* src = reinterpret_cast<const float4*>(part_o + first * kD) + lane;
-    int s = 0;
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+        const float w = __shfl_sync(0xFFFFFFFFu, my_w, u);     // zero for u >= n_splits
+        acc.x += w * head_v[u].x; acc.y += w * head_v[u].y; acc.z += w * head_v[u].z; acc.w += w * head_v[u].w;
+    }
+    int s = 8;
     for (; s + 4 <= n_splits; s += 4) {
         float4 v[4];
 #pragma unroll
