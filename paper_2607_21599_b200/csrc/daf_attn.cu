@@ -400,7 +400,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
     unsigned char* v_smem = smem + 2 * (size_t)kTileBytes;        // two sub-step slots
     AttnSmem* sm = reinterpret_cast<AttnSmem*>(smem + 3 * (size_t)kTileBytes);
 
-    pdl_wait();                // inputs may come from the kernel launched just before (gather / hybrid-cache update)
     pdl_launch_dependents();   // a dependent kernel (the split merge) may start launching; it waits for this grid
 
     if (threadIdx.x == 0) DAF_STAMP(0);
@@ -416,16 +415,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
     const int h0 = a.hb * a.Gp;
     const int g_kv = h0 / a.G;
     const int t0 = a.unit * a.Tt;
-    // sub-steps of this item: the keys of its range that the tile's last token may see
     const int key_begin = a.j_begin * kBlockN;
-    int n_t = 0;
-    if (a.unit < a.n_tb) {
-        const int max_tok = min(a.n_q, t0 + a.Tt) - 1;
-        const long long last_key = a.q_pos ? (long long)__ldg(a.q_pos + max_tok) : (long long)max_tok + a.causal_off;
-        long long hi = min((long long)a.n_kv, last_key + 1);
-        hi = min(hi, (long long)a.j_end * kBlockN);
-        if (hi > key_begin) n_t = (int)((hi - key_begin + kSubN - 1) / kSubN);
-    }
 
     // Loads K (kv = 0) or V (kv = 1) of sub-step t into its ring slot (the slot must be free).
     auto issue_kv = [&](int t, int kv) {
@@ -441,8 +431,14 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
     // Set-up.  The producer thread prepares the barriers and at once starts the loads that need no free
     // slot (Q and the first two sub-steps), so that their latency overlaps the rest of the set-up: the
     // status check (a global read) and the tensor-memory allocation.
+    // Everything up to the wait below touches no memory an earlier kernel writes, so with programmatic
+    // dependent launch it runs while the kernel launched just before (gather / hybrid-cache update) drains.
     __shared__ int skip_cta;
     const int32_t* const q_idx = DAF_SEG(q_idx);     // non-null: the softmax warps fetch the Q rows themselves
+    if (warp == 5) {
+        tmem_alloc(&sm->tmem_base, kAttnTmemCols);
+        tmem_relinquish();
+    }
     if (warp == 4 && lane == 0) {
         mbar_init(&sm->q_full, q_idx != nullptr ? 4 : 1);
         for (int s = 0; s < 2; ++s) {
@@ -453,11 +449,23 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
         mbar_init(&sm->pv_done, 1);
         sm->abort_flag = 0;
         mbar_fence_init();
+        tma_prefetch_desc(tmap_k);
+        tma_prefetch_desc(tmap_v);
+        if (q_idx == nullptr) tma_prefetch_desc(tmap_q);
+    }
+    pdl_wait();                // from here on: inputs that the kernel launched just before may have written
+    // sub-steps of this item: the keys of its range that the tile's last token may see
+    int n_t = 0;
+    if (a.unit < a.n_tb) {
+        const int max_tok = min(a.n_q, t0 + a.Tt) - 1;
+        const long long last_key = a.q_pos ? (long long)__ldg(a.q_pos + max_tok) : (long long)max_tok + a.causal_off;
+        long long hi = min((long long)a.n_kv, last_key + 1);
+        hi = min(hi, (long long)a.j_end * kBlockN);
+        if (hi > key_begin) n_t = (int)((hi - key_begin + kSubN - 1) / kSubN);
+    }
+    if (warp == 4 && lane == 0) {
         if (n_t > 0) {
-            tma_prefetch_desc(tmap_k);
-            tma_prefetch_desc(tmap_v);
             if (q_idx == nullptr) {
-                tma_prefetch_desc(tmap_q);
                 mbar_arrive_expect_tx(&sm->q_full, 2u * 128u * (uint32_t)(a.Gp * a.Tt));
                 tma_load_3d(q_smem, tmap_q, &sm->q_full, 0, h0, t0);
                 tma_load_3d(q_smem + kHalfBytes, tmap_q, &sm->q_full, 64, h0, t0);
@@ -493,10 +501,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
     }
     // a CTA of this grid (or an earlier kernel sharing the workspace) has already given up: do nothing
     if (threadIdx.x == 0) skip_cta = (status != nullptr && *reinterpret_cast<volatile int*>(&status->code) != 0) ? 1 : 0;
-    if (warp == 5) {
-        tmem_alloc(&sm->tmem_base, kAttnTmemCols);
-        tmem_relinquish();
-    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
