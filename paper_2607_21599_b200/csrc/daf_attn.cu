@@ -86,8 +86,8 @@ extern "C" int daf_dbg_read_laps(void* host, size_t bytes) {
 #define DAF_LAP(acc) do {} while (0)
 #endif
 
-// One online-softmax step of one query row (one thread) over NCH * 32 keys starting at `key0`: reads the
-// row's logits from tensor memory, writes P = exp(s - m) as bf16 over the first half of the same columns,
+// One online-softmax step of one query row (one thread) over NCH * 32 keys starting at `key0` (the kernel
+// uses NCH = 2, a 64-key sub-step): reads the row's logits from tensor memory, writes P = exp(s - m) as bf16 over the first half of the same columns,
 // keeps the running maximum m and sum l.  Returns the factor the row of O has to be multiplied by (1
 // unless the maximum grew past the lazy threshold).  `limit` is the last key the row may see;
 // c = softmax scale * log2(e).
@@ -167,16 +167,6 @@ __device__ __forceinline__ void rescale_o(uint32_t o_addr, float alpha) {
         for (int i = 0; i < 32; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * alpha);
         tmem_st32(o_addr + (uint32_t)(cchunk * 32), orr);
     }
-}
-
-// A whole 128-key step: the commit that released S_j also covers the previous P V product, so O is
-// quiescent when the row has to be rescaled.
-__device__ __forceinline__ void softmax_step(uint32_t s_addr, uint32_t o_addr, int key0, int limit, float c, bool first,
-                                             float& m, float& l) {
-    const float alpha = softmax_core<4>(s_addr, key0, limit, c, m, l);
-    if (!first && __any_sync(0xFFFFFFFFu, alpha != 1.f)) rescale_o(o_addr, alpha);
-    tc_wait_st();
-    tc_fence_before();
 }
 
 // Picks a field of the problem a CTA works on (seg_id is uniform across the CTA).

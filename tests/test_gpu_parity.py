@@ -564,3 +564,43 @@ def test_layer_without_packed_q_buffer(fuse_mode):
                        ws), ws, "daf_select")
     assert torch.equal(idx_out.cpu(), outs[0][1]) and torch.equal(kp.cpu(), outs[0][2]) and torch.equal(vp.cpu(), outs[0][3])
     assert torch.equal(kv_k.cpu(), outs[0][4]) and torch.equal(kv_v.cpu(), outs[0][5])
+
+
+def test_work_list_shapes_drawn_at_random():
+    """Seeded random shapes through daf_imp_qd_attn: group sizes 1-8, condensed sequences around multiples of
+    the 128-row tile and of the 64-key sub-step, question blocks that see different numbers of key tiles."""
+    rng = np.random.default_rng(20260721)
+    dev = "cuda"
+    scale = 1.0 / math.sqrt(128)
+    for case in range(10):
+        Hkv = int(rng.choice([1, 2, 4]))
+        G = int(rng.choice([1, 2, 4, 7, 8]))
+        Hq = Hkv * G
+        k = int(rng.choice([1, 63, 64, 65, 127, 128, 129, 191, 257, 500, 640]))
+        L_d = k + int(rng.integers(0, 700))
+        L_q = int(rng.choice([1, 2, 17, 64, 130, 300]))
+        fuse_mode = int(rng.integers(0, 2))
+        N = L_d + L_q
+        r = k / L_d
+        p = api.make_params(L_d, L_q, r, Hq, Hkv, fuse_mode=fuse_mode)
+        if api.daf_num_important(L_d, r) != k:
+            continue
+        ws = api.alloc_workspace(p)
+        qp, kp, vp = _normal((k, Hq, 128), 100 + case), _normal((k, Hkv, 128), 200 + case), _normal((k, Hkv, 128), 300 + case)
+        qq = _normal((L_q, Hq, 128), 400 + case)
+        kv_k, kv_v = _normal((N, Hkv, 128), 500 + case), _normal((N, Hkv, 128), 600 + case)
+        idx = torch.from_numpy(np.sort(rng.choice(L_d, k, replace=False)).astype(np.int32))
+        rows = k + L_q if fuse_mode == 0 else N
+        hidden = torch.full((rows, Hq, 128), -9.0, dtype=torch.bfloat16, device=dev)
+        what = f"case {case}: k={k} L_d={L_d} L_q={L_q} Hq={Hq} Hkv={Hkv} fuse={fuse_mode}"
+        _ok(api.daf_imp_qd_attn(p, qp.to(dev), None, kp.to(dev), vp.to(dev), qq.to(dev), kv_k.to(dev), kv_v.to(dev),
+                                idx.to(dev), hidden, ws), ws, what)
+        ref_i = oracle.important_attn(_f(qp), _f(kp), _f(vp), scale)
+        ref_q = oracle.qd_attn(_f(qq), _f(kv_k), _f(kv_v), L_d, scale)
+        h = hidden.cpu()
+        if fuse_mode == 0:
+            _assert_close(h[:k], ref_i, what + " important rows")
+            _assert_close(h[k:], ref_q, what + " question rows")
+        else:
+            _assert_close(h[idx.long()], ref_i, what + " important rows")
+            _assert_close(h[L_d:], ref_q, what + " question rows")
