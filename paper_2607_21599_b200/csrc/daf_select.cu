@@ -198,8 +198,8 @@ select_topk_kernel(const float* __restrict__ scores, int n_sig, int L_d, int k,
 // CTA with no cluster traffic.  The keys are first reduced to their offset from the smallest key.  One
 // pass over all keys histograms the top 11 of the bits that offset needs (typically 24-27 of 32, fewer
 // when the scores are close together) with shared-memory atomics and finds the bin that holds the k-th
-// largest key; only the keys of that bin (typically well under one per cent) go on to passes of 9 bits
-// that fix the remaining bits.  Because the offsets of real scores spread over the whole histogram,
+// largest key; only the keys of that bin (typically well under one per cent) go on: when they are few,
+// each is ranked against the others directly, otherwise passes of 9 bits fix the remaining bits.  Because the offsets of real scores spread over the whole histogram,
 // the atomics rarely collide; scores that are all (nearly) equal collide more, and all of them become
 // candidates, but the result stays correct.  An ordered compaction then emits the positions.
 constexpr int kSel1Threads = 1024;
@@ -332,8 +332,26 @@ select_topk_cta_kernel(const float* __restrict__ scores, int n_sig, int L_d, int
     if (tid < kSel1Bins) sh->hist[tid] = 0u;
     __syncthreads();
     const int n_cand = (int)sh->n_cand;    // at most L_d, the capacity of the list
-    const int passes = (low_bits + kSel1Bits - 1) / kSel1Bits;
+    int passes = (low_bits + kSel1Bits - 1) / kSel1Bits;
     uint32_t prefix = 0u;      // the low digits fixed so far
+    if (passes > 0 && n_cand <= kSel1Threads) {
+        // few candidates (the usual case): each thread ranks one candidate by counting the larger and the
+        // equal ones; the candidate whose rank interval holds the remaining rank is the threshold
+        const uint32_t k_rem = sh->pick[1];
+        if (tid < n_cand) {
+            const uint32_t mine = cand[tid];
+            uint32_t n_gt = 0, n_eq = 0;
+            for (int j = 0; j < n_cand; ++j) {
+                const uint32_t other = cand[j];
+                n_gt += other > mine;
+                n_eq += other == mine;
+            }
+            if (k_rem > n_gt && k_rem <= n_gt + n_eq) { sh->pick[0] = mine; sh->pick[1] = k_rem - n_gt; }   // equal candidates write the same
+        }
+        __syncthreads();
+        prefix = sh->pick[0];
+        passes = 0;
+    }
     for (int p = 0; p < passes; ++p) {
         const int shift = (passes - 1 - p) * kSel1Bits;
         for (int i = tid; i < n_cand; i += kSel1Threads) {
