@@ -86,6 +86,20 @@ def test_host_side_argument_validation(lib):
     assert api.daf_important_attn(ok, 2, buf, buf, buf, buf, 1000, None, None, ws) == api.DAF_ERR_ALIGNMENT
     assert api.daf_important_attn(ok, 2, buf, buf, buf, buf, 512, None, None, ws) == api.DAF_ERR_INVALID_ARG
     assert api.daf_important_attn(ok, 2, buf[8:], buf, buf, buf, 1024, None, None, ws) == api.DAF_ERR_ALIGNMENT
+    # both stages from one work list: needs packed K/V, the question rows, the cache, and either packed Q
+    # rows or (q_fresh, idx); idx also for scattered output rows
+    both = lambda p, q_pack, q_fresh, idx, hidden=buf: api.daf_imp_qd_attn(p, q_pack, q_fresh, buf, buf, buf, buf, buf, idx,  # noqa: E731
+                                                                         hidden, ws)
+    assert both(ok, None, None, None) == api.DAF_ERR_INVALID_ARG            # no Q rows at all
+    assert both(ok, None, buf, None) == api.DAF_ERR_INVALID_ARG             # Q in place needs idx
+    assert both(ok, buf, None, None, hidden=None) == api.DAF_ERR_INVALID_ARG
+    assert both(ok, buf[8:], None, None) == api.DAF_ERR_ALIGNMENT
+    assert both(api.make_params(256, 16, 0.25, 4, 2, fuse_mode=1), buf, None, None) == api.DAF_ERR_INVALID_ARG
+    assert both(api.make_params(256, 0, 0.25, 4, 2), buf, None, None) == api.DAF_ERR_INVALID_ARG   # no question rows
+    assert both(api.make_params(256, 16, 0.0, 4, 2), buf, None, None) == api.DAF_ERR_INVALID_ARG   # no important rows
+    # a layer without question rows cannot read Q in place (only the joint launch does)
+    no_q = api.make_params(256, 0, 0.25, 4, 2)
+    assert api.daf_layer(no_q, buf, 1, None, buf, buf, buf, buf, buf, buf, None, buf, buf, buf, None, ws) == api.DAF_ERR_INVALID_ARG
     assert api.daf_launch_count() == 0
     assert "workspace" in api.daf_strerror(api.DAF_ERR_WORKSPACE)
     assert api.daf_layer_host(ok, None, 1, None, None, None, None, None, None, 0, None, None, None) == api.DAF_ERR_WORKSPACE
