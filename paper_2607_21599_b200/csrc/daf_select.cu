@@ -455,7 +455,6 @@ struct FuseArgs {
     const int4* o_imp; const int4* o_q; int4* hidden;
     const int32_t* idx; int32_t* row_pos;
     int k, L_d, L_q, cq, mode;
-    DeviceStatus* status;
 };
 
 __global__ void __launch_bounds__(kRowThreads)
@@ -608,7 +607,6 @@ int launch_fuse(const ResolvedParams& rp, const int32_t* idx, const void* o_imp,
     a.hidden = reinterpret_cast<int4*>(hidden);
     a.idx = idx; a.row_pos = row_pos_out;
     a.k = rp.k; a.L_d = rp.L_d; a.L_q = rp.L_q; a.cq = rp.Hq * 16; a.mode = rp.fuse_mode;
-    a.status = nullptr;
     fuse_rows_kernel<<<rows, kRowThreads, 0, stream>>>(a);
     count_launch();
     return check_launch();
