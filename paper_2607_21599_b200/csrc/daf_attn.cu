@@ -10,6 +10,12 @@
 #include <math.h>
 #include <string.h>
 
+#include <functional>
+#include <map>
+#include <mutex>
+#include <queue>
+#include <vector>
+
 #include "daf_common.cuh"
 
 namespace daf {
@@ -808,7 +814,6 @@ static int set_kernel_attributes() {
 
 // How a single problem is cut into CTAs: one per (head block, token block), and for the question rows,
 // where there are few query tiles and a long KV axis, also per range of the KV axis.
-static float g_joint_factor = 1.0f;   // longest item of a joint launch, as a fraction of the mean load of a CTA slot
 
 AttnPlan plan_attention(int n_q, int n_kv, int Hq, int G, int causal_off, bool pack_group, bool allow_split) {
     AttnPlan pl;
@@ -849,50 +854,147 @@ static int slots_before(int n_units, int chunk) {
     return chunk * g * (g + 1) / 2 + (n_units - g * chunk) * (g + 1);
 }
 
-// Steps 2 and 3 of one layer as one list of work items.  The longest item is held to a fraction of the
-// mean load of a CTA slot: long causal chains of the important-token stage are cut into ranges (merged
-// afterwards like the KV splits of the question stage), short ones are left whole.
+// Steps 2 and 3 of one layer as one list of work items.  Two things are free: into how many balanced
+// ranges the long causal chains of the important-token stage are cut (`chunk`), and into how many KV
+// ranges the question rows are cut.  Finer ranges balance the 296 CTA slots better but cost a fixed
+// time per item, partial-result traffic and a longer merge, and the optimum jumps around with the tile
+// counts.  So the choice is made by replaying the hardware's dispatch (items in grid order onto the
+// slot that frees first) for a handful of candidates with a three-constant cost model and keeping the
+// cheapest; the result is cached per problem shape.
+namespace {
+constexpr float kCostItemUs = 5.5f;        // set-up, first logits and row epilogue of an item (measured 5-6 us)
+constexpr float kCostSubStepUs = 1.05f;    // 64 keys through one tile with two CTAs per SM (measured 0.95-1.1 us)
+constexpr float kCostMergeUs = 2.0f;       // merge launch
+constexpr float kCostMergeUsPerMB = 1.0f;  // plus writing and re-reading the partial rows (fitted: 0.25-0.4 picked too many ranges)
+
+int g_force_chunk = 0, g_force_splits_q = 0;   // tuning builds can pin the choice
+float g_last_predicted_us = 0.f;
+
+struct JointShape { int k, L_q, L_d, Hq, G; };
+bool operator<(const JointShape& a, const JointShape& b) {
+    if (a.k != b.k) return a.k < b.k;
+    if (a.L_q != b.L_q) return a.L_q < b.L_q;
+    if (a.L_d != b.L_d) return a.L_d < b.L_d;
+    if (a.Hq != b.Hq) return a.Hq < b.Hq;
+    return a.G < b.G;
+}
+
+// Fills the fields of `jp` that follow from (chunk, n_splits_q).
+void set_choice(JointPlan& jp, int chunk, int n_splits_q, int L_q, int L_d, int Hq) {
+    if (chunk < (jp.n_tb_i + 31) / 32) chunk = (jp.n_tb_i + 31) / 32;   // at most 32 ranges per token block
+    if (chunk < 1) chunk = 1;
+    if (chunk > jp.n_tb_i) chunk = jp.n_tb_i;
+    jp.chunk = chunk;
+    jp.n_slots = slots_before(jp.n_tb_i, chunk);
+    jp.part_bytes_i = 0;
+    if (chunk < jp.n_tb_i) {
+        const size_t rows = (size_t)jp.n_slots * kBlockM * Hq;
+        jp.part_bytes_i = rows * kD * sizeof(float) + (rows * sizeof(float) + 255) / 256 * 256;
+    }
+    jp.items_i = Hq * jp.n_slots;
+    const int tiles_q = (L_d + L_q + kBlockN - 1) / kBlockN;
+    if (n_splits_q < 1) n_splits_q = 1;
+    jp.tiles_per_split_q = (tiles_q + n_splits_q - 1) / n_splits_q;
+    jp.n_splits_q = (tiles_q + jp.tiles_per_split_q - 1) / jp.tiles_per_split_q;
+    jp.items_q = jp.head_blocks_q * jp.n_tb_q * jp.n_splits_q;
+    jp.part_bytes_q = attn_partial_bytes(L_q, Hq, jp.n_splits_q);
+}
+
+// Predicted time of the attention launch + merge for a filled plan, in microseconds.
+float predict_us(const JointPlan& jp, int k, int L_q, int L_d, int Hq) {
+    const int slots = kNumSMs * 2;
+    std::priority_queue<float, std::vector<float>, std::greater<float>> free_at;
+    for (int i = 0; i < slots; ++i) free_at.push(0.f);
+    float makespan = 0.f;
+    auto run = [&](int count, int tiles) {
+        const float cost = kCostItemUs + kCostSubStepUs * 2.f * (float)tiles;
+        for (int i = 0; i < count; ++i) {
+            const float t = free_at.top() + cost;
+            free_at.pop();
+            free_at.push(t);
+            if (t > makespan) makespan = t;
+        }
+    };
+    // question items: split-major, token blocks from the last one down, head blocks together
+    for (int s = 0; s < jp.n_splits_q; ++s)
+        for (int u = jp.n_tb_q - 1; u >= 0; --u) {
+            const int last_tok = (u + 1) * jp.Tt_q < L_q ? (u + 1) * jp.Tt_q : L_q;
+            const int tiles_total = (L_d + last_tok + kBlockN - 1) / kBlockN;
+            int tiles = tiles_total - s * jp.tiles_per_split_q;
+            if (tiles > jp.tiles_per_split_q) tiles = jp.tiles_per_split_q;
+            if (tiles > 0) run(jp.head_blocks_q, tiles);
+        }
+    // important-token items: slots from the top down, all heads together
+    size_t part_rows_i = 0;
+    for (int slot = jp.n_slots - 1; slot >= 0; --slot) {
+        int g = 0;
+        while (jp.chunk * (g + 1) * (g + 2) / 2 <= slot) ++g;
+        const int rem = slot - jp.chunk * g * (g + 1) / 2;
+        const int unit = g * jp.chunk + rem / (g + 1), range = rem % (g + 1);
+        const int n_tiles = unit + 1 < jp.n_tb_i ? unit + 1 : jp.n_tb_i;
+        run(Hq, (range + 1) * n_tiles / (g + 1) - range * n_tiles / (g + 1));
+        if (g >= 1) part_rows_i += (size_t)kBlockM * Hq;
+    }
+    (void)k;
+    const float merge_mb = (float)(jp.part_bytes_q + part_rows_i * 516) / 1e6f;
+    const bool merges = jp.n_splits_q > 1 || jp.chunk < jp.n_tb_i;
+    return makespan + (merges ? kCostMergeUs + kCostMergeUsPerMB * merge_mb : 0.f);
+}
+}  // namespace
+
 JointPlan plan_joint(int k, int L_q, int L_d, int Hq, int G) {
+    static std::mutex mu;
+    static std::map<JointShape, JointPlan> cache;
+    const JointShape shape{k, L_q, L_d, Hq, G};
+    const bool forced = g_force_chunk > 0 || g_force_splits_q > 0;
+    if (!forced) {
+        std::lock_guard<std::mutex> lock(mu);
+        auto it = cache.find(shape);
+        if (it != cache.end()) return it->second;
+    }
     JointPlan jp;
-    const int N = L_d + L_q;
     jp.n_tb_i = (k + kBlockM - 1) / kBlockM;
     jp.Gp_q = G > 128 ? 1 : G;
     jp.Tt_q = kBlockM / jp.Gp_q;
     jp.n_tb_q = (L_q + jp.Tt_q - 1) / jp.Tt_q;
     jp.head_blocks_q = Hq / jp.Gp_q;
-    const int tiles_q = (N + kBlockN - 1) / kBlockN;
-    // work in CTA steps (one 128-key tile through one query tile)
-    long long work = (long long)Hq * jp.n_tb_i * (jp.n_tb_i + 1) / 2 + (long long)jp.head_blocks_q * jp.n_tb_q * tiles_q;
-    const int slots = kNumSMs * 2;
-    int longest = (int)ceilf(g_joint_factor * (float)work / (float)slots);
-    if (longest < 2) longest = 2;
-    auto set_chunk = [&](int chunk) {
-        if (chunk < 1) chunk = 1;
-        if (chunk < (jp.n_tb_i + 31) / 32) chunk = (jp.n_tb_i + 31) / 32;   // at most 32 ranges per token block
-        if (chunk > jp.n_tb_i) chunk = jp.n_tb_i;
-        jp.chunk = chunk;
-        jp.n_slots = slots_before(jp.n_tb_i, chunk);
-        jp.part_bytes_i = 0;
-        if (chunk < jp.n_tb_i) {
-            const size_t rows = (size_t)jp.n_slots * kBlockM * Hq;
-            jp.part_bytes_i = rows * kD * sizeof(float) + (rows * sizeof(float) + 255) / 256 * 256;
+    const int tiles_q = (L_d + L_q + kBlockN - 1) / kBlockN;
+    if (forced) {
+        set_choice(jp, g_force_chunk > 0 ? g_force_chunk : jp.n_tb_i, g_force_splits_q > 0 ? g_force_splits_q : 1, L_q, L_d, Hq);
+        g_last_predicted_us = predict_us(jp, k, L_q, L_d, Hq);
+        return jp;
+    }
+    // candidates: the causal chains whole, or cut so that the longest has 2..6 ranges; every distinct
+    // number of question ranges up to 32
+    JointPlan best = jp;
+    float best_us = -1.f;
+    for (int m = 1; m <= 6; ++m) {
+        const int chunk = (jp.n_tb_i + m - 1) / m;
+        if (m > 1 && chunk == (jp.n_tb_i + m - 2) / (m - 1)) continue;   // same cut as the previous candidate
+        int last_tps = -1;
+        for (int n = 1; n <= kMaxSplits && n <= tiles_q; ++n) {
+            JointPlan cand = jp;
+            set_choice(cand, chunk, n, L_q, L_d, Hq);
+            if (cand.tiles_per_split_q == last_tps) continue;
+            last_tps = cand.tiles_per_split_q;
+            if (cand.part_bytes_i > ((size_t)256 << 20)) continue;   // partials of a large problem: not worth their memory
+            const float us = predict_us(cand, k, L_q, L_d, Hq);
+            if (best_us < 0.f || us < best_us) { best_us = us; best = cand; }
         }
-    };
-    set_chunk(longest);
-    if (jp.part_bytes_i > ((size_t)256 << 20)) set_chunk(jp.n_tb_i);   // partials of a large problem: not worth their traffic
-    jp.items_i = Hq * jp.n_slots;
-    int want = (tiles_q + longest - 1) / longest;
-    if (want > kMaxSplits) want = kMaxSplits;
-    if (want < 1) want = 1;
-    jp.tiles_per_split_q = (tiles_q + want - 1) / want;
-    jp.n_splits_q = (tiles_q + jp.tiles_per_split_q - 1) / jp.tiles_per_split_q;
-    jp.items_q = jp.head_blocks_q * jp.n_tb_q * jp.n_splits_q;
-    jp.part_bytes_q = attn_partial_bytes(L_q, Hq, jp.n_splits_q);
-    return jp;
+    }
+    g_last_predicted_us = best_us;
+    std::lock_guard<std::mutex> lock(mu);
+    cache[shape] = best;
+    return best;
 }
 
 #ifdef DAF_TRACE
-extern "C" void daf_dbg_joint_factor(float f) { g_joint_factor = f; }
+extern "C" void daf_dbg_joint_force(int chunk, int n_splits_q) { g_force_chunk = chunk; g_force_splits_q = n_splits_q; }
+extern "C" float daf_dbg_joint_predicted_us(void) { return g_last_predicted_us; }
+extern "C" void daf_dbg_joint_plan(int k, int L_q, int L_d, int Hq, int G, int* out) {
+    const JointPlan jp = plan_joint(k, L_q, L_d, Hq, G);
+    out[0] = jp.chunk; out[1] = jp.n_tb_i; out[2] = jp.n_splits_q; out[3] = jp.items_i + jp.items_q;
+}
 #endif
 
 static void fill_problem(SegArgs* s, int n_q, int n_kv, int Hq, int G, int Gp, int causal_off, const int32_t* q_pos,
