@@ -862,10 +862,10 @@ static int slots_before(int n_units, int chunk) {
 // slot that frees first) for a handful of candidates with a three-constant cost model and keeping the
 // cheapest; the result is cached per problem shape.
 namespace {
-constexpr float kCostItemUs = 5.5f;        // set-up, first logits and row epilogue of an item (measured 5-6 us)
+constexpr float kCostItemUs = 7.0f;        // set-up, first logits and row epilogue of an item (5-6 us alone; fitted)
 constexpr float kCostSubStepUs = 1.05f;    // 64 keys through one tile with two CTAs per SM (measured 0.95-1.1 us)
 constexpr float kCostMergeUs = 2.0f;       // merge launch
-constexpr float kCostMergeUsPerMB = 1.0f;  // plus writing and re-reading the partial rows (fitted: 0.25-0.4 picked too many ranges)
+constexpr float kCostMergeUsPerMB = 0.15f; // plus re-reading the partial rows (fitted together with the item cost)
 
 int g_force_chunk = 0, g_force_splits_q = 0;   // tuning builds can pin the choice
 float g_last_predicted_us = 0.f;
