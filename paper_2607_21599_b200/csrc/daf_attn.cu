@@ -537,55 +537,78 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
         }
     } else if (warp == 5) {
         // ------------------------------------------------------------ MMA issuer
-        if (lane == 0 && n_t > 0) {
+        // The whole warp walks the loop and waits on the barriers, one elected lane issues: control flow
+        // stays uniform across the warp, so the operand descriptors can live in uniform registers.
+        if (n_t > 0) {
             constexpr uint32_t idesc_qk = make_idesc_bf16(kBlockM, kSubN, 0);
             constexpr uint32_t idesc_pv = make_idesc_bf16(kBlockM, kD, 1);
             const uint32_t qa = smem_u32(q_smem);
             // S_b = Q K_t^T for the 64 keys in K slot b (= t & 1)
-            auto issue_qk = [&](int b) {
-                const uint32_t ka = smem_u32(k_smem + (size_t)b * kSubBytes);
+            // every operand descriptor is fixed for the whole item: they are built once, ahead of the loop
+            uint64_t qd[kD / 16], kd[2][kD / 16], vd[2][kSubN / 16];
 #pragma unroll
-                for (int kk = 0; kk < kD / 16; ++kk) {
-                    const uint32_t qoff = (uint32_t)((kk & 3) * 32 + (kk >> 2) * kHalfBytes);
-                    const uint32_t koff = (uint32_t)((kk & 3) * 32 + (kk >> 2) * kSubHalfBytes);
-                    tc_mma_ss(tmem + (uint32_t)(b * kSubN), make_smem_desc(qa + qoff, 16, 1024), make_smem_desc(ka + koff, 16, 1024),
-                              idesc_qk, kk > 0 ? 1u : 0u);
-                }
+            for (int kk = 0; kk < kD / 16; ++kk) {
+                qd[kk] = make_smem_desc(qa + (uint32_t)((kk & 3) * 32 + (kk >> 2) * kHalfBytes), 16, 1024);
+#pragma unroll
+                for (int b = 0; b < 2; ++b)
+                    kd[b][kk] = make_smem_desc(smem_u32(k_smem + (size_t)b * kSubBytes) + (uint32_t)((kk & 3) * 32 + (kk >> 2) * kSubHalfBytes), 16, 1024);
+            }
+#pragma unroll
+            for (int kk = 0; kk < kSubN / 16; ++kk)
+#pragma unroll
+                for (int b = 0; b < 2; ++b)
+                    vd[b][kk] = make_smem_desc(smem_u32(v_smem + (size_t)b * kSubBytes) + (uint32_t)kk * 2048u, kSubHalfBytes, 1024);
+            auto issue_qk = [&](int b) {
+#pragma unroll
+                for (int kk = 0; kk < kD / 16; ++kk)
+                    tc_mma_ss(tmem + (uint32_t)(b * kSubN), qd[kk], b ? kd[1][kk] : kd[0][kk], idesc_qk, kk > 0 ? 1u : 0u);
             };
             // O (+)= P_b V_t for the 64 keys in V slot b; P (bf16) sits in the first 32 columns of S_b
             auto issue_pv = [&](int b, bool first) {
-                const uint32_t va = smem_u32(v_smem + (size_t)b * kSubBytes);
 #pragma unroll
                 for (int kk = 0; kk < kSubN / 16; ++kk)
-                    tc_mma_ts(tmem + (uint32_t)kBlockN, tmem + (uint32_t)(b * kSubN + kk * 8),
-                              make_smem_desc(va + (uint32_t)kk * 2048u, kSubHalfBytes, 1024), idesc_pv, (first && kk == 0) ? 0u : 1u);
+                    tc_mma_ts(tmem + (uint32_t)kBlockN, tmem + (uint32_t)(b * kSubN + kk * 8), b ? vd[1][kk] : vd[0][kk], idesc_pv,
+                              (first && kk == 0) ? 0u : 1u);
             };
             bool ok = mbar_wait(&sm->q_full, 0, abort_flag, status, 20);
+            ok = __all_sync(0xFFFFFFFFu, ok);
             for (int t = 0; t < 2 && t < n_t && ok; ++t) {   // the first two S tiles
                 ok = mbar_wait(&sm->k_full[t], 0, abort_flag, status, 30 + t);
+                ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) break;
                 tc_fence_after();
-                issue_qk(t);
-                tc_commit(&sm->s_full[t]);
-                tc_commit(&sm->k_empty[t]);
+                if (elect_one()) {
+                    issue_qk(t);
+                    tc_commit(&sm->s_full[t]);
+                    tc_commit(&sm->k_empty[t]);
+                }
+                __syncwarp();
             }
             for (int t = 0; t < n_t && ok; ++t) {
                 const int b = t & 1;
                 const uint32_t par = (uint32_t)((t >> 1) & 1);
                 ok = mbar_wait(&sm->v_full[b], par, abort_flag, status, 32 + b);
                 if (ok) ok = mbar_wait(&sm->p_full[b], par, abort_flag, status, 40 + b);
+                ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) break;
                 tc_fence_after();
-                issue_pv(b, t == 0);
-                tc_commit(&sm->v_empty[b]);
-                tc_commit(&sm->pv_done);
+                if (elect_one()) {
+                    issue_pv(b, t == 0);
+                    tc_commit(&sm->v_empty[b]);
+                    tc_commit(&sm->pv_done);
+                }
+                __syncwarp();
                 if (t + 2 < n_t) {
                     ok = mbar_wait(&sm->k_full[b], (uint32_t)(((t + 2) >> 1) & 1), abort_flag, status, 34 + b);
+                    ok = __all_sync(0xFFFFFFFFu, ok);
                     if (!ok) break;
                     tc_fence_after();
-                    issue_qk(b);
-                    tc_commit(&sm->s_full[b]);
-                    tc_commit(&sm->k_empty[b]);
+                    if (elect_one()) {
+                        issue_qk(b);
+                        tc_commit(&sm->s_full[b]);
+                        tc_commit(&sm->k_empty[b]);
+                    }
+                    __syncwarp();
                 }
             }
         }
@@ -670,6 +693,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
     }
 #endif
 }
+
 
 #undef DAF_SEG
 

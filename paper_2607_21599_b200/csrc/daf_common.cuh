@@ -132,6 +132,16 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
+// True in exactly one lane of a converged warp (the same lane every time).
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "elect.sync _|p, 0xffffffff;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(pred));
+    return pred != 0;
+}
 // Bounded wait: gives up after `limit` polls or as soon as another thread of the
 // CTA has raised *abort_flag.  Returns false on give-up (the caller unwinds).
 constexpr uint32_t kWaitLimitPolls = 1u << 22;          // hard cap on polls
