@@ -47,7 +47,7 @@ struct SelShared {
     uint32_t scan_gt[kSelWarps];
     uint32_t scan_eq[kSelWarps];
     uint32_t cta_counts[2];    // this CTA's number of keys above / equal to the threshold (read by peers)
-    uint32_t pick[2];          // chosen prefix, remaining rank
+    uint32_t pick[3];          // chosen prefix, remaining rank, number of keys in the chosen bin
 };
 
 __global__ void __cluster_dims__(kSelCluster, 1, 1) __launch_bounds__(kSelThreads, 1)
@@ -78,9 +78,12 @@ select_topk_kernel(const float* __restrict__ scores, int n_sig, int L_d, int k,
         keys[at(i)] = score_key(acc);
     }
     if (tid < 256) { sh->hist[0][tid] = 0u; sh->hist[1][tid] = 0u; }
-    if (tid == 0) { sh->pick[0] = 0u; sh->pick[1] = (uint32_t)k; }
+    if (tid == 0) { sh->pick[0] = 0u; sh->pick[1] = (uint32_t)k; sh->pick[2] = 0u; }
     __syncthreads();
 
+    // Radix selection from the top byte down.  It stops as soon as every key left in the chosen bin is taken
+    // (with distinct scores usually after three passes): the comparisons below then look only at the bits
+    // resolved so far.
     uint32_t prefix = 0u, mask = 0u;
     int pass = 0;
     for (int shift = 24; shift >= 0; shift -= 8, ++pass) {
@@ -133,6 +136,7 @@ select_topk_kernel(const float* __restrict__ scores, int n_sig, int L_d, int k,
                     if (k_rem <= a + c) {
                         sh->pick[0] = prefix | ((uint32_t)(base + b) << shift);
                         sh->pick[1] = k_rem - a;
+                        sh->pick[2] = c;
                         break;
                     }
                     a += c;
@@ -142,16 +146,17 @@ select_topk_kernel(const float* __restrict__ scores, int n_sig, int L_d, int k,
         __syncthreads();
         prefix = sh->pick[0];
         mask |= 0xFFu << shift;
+        if (sh->pick[2] == sh->pick[1]) break;   // every key left in the bin is taken: no need to tell them apart
     }
-    const uint32_t thr = prefix;           // key of the k-th largest score
-    const uint32_t need_eq = sh->pick[1];  // how many keys equal to thr are taken (lowest positions first)
+    const uint32_t thr = prefix;           // the resolved bits of the k-th largest key
+    const uint32_t need_eq = sh->pick[1];  // how many keys matching thr are taken (lowest positions first)
 
     // ordered compaction: thread t owns the contiguous local positions [t*E, (t+1)*E)
     const int E = (per_cta + kSelThreads - 1) / kSelThreads;
     const int lo = min(n_loc, tid * E), hi = min(n_loc, lo + E);
     uint32_t n_gt = 0, n_eq = 0;
     for (int i = lo; i < hi; ++i) {
-        const uint32_t key = keys[at(i)];
+        const uint32_t key = keys[at(i)] & mask;
         n_gt += key > thr;
         n_eq += key == thr;
     }
@@ -183,7 +188,7 @@ select_topk_kernel(const float* __restrict__ scores, int n_sig, int L_d, int k,
     if (k > 0) {
         uint32_t pos = gt_before + min(eq_before, need_eq);
         for (int i = lo; i < hi; ++i) {
-            const uint32_t key = keys[at(i)];
+            const uint32_t key = keys[at(i)] & mask;
             bool take = key > thr;
             if (key == thr) { take = eq_before < need_eq; ++eq_before; }
             if (take) idx_out[pos++] = lo_cta + i;
@@ -510,8 +515,8 @@ deviation_scores_kernel(const int4* __restrict__ k_fresh, const int4* __restrict
 }
 
 // ----------------------------------------------------------------- host side
-// Measured on B200 (selection alone): one CTA 5.1 / 6.9 / 6.8 / 9.9 us at 1K / 6K / 8K / 16K tokens, the cluster
-// of eight 7.6 / 8.4 / 8.4 / 9.0 us: one CTA up to 8K tokens, the cluster beyond.
+// Measured on B200 (selection alone): one CTA 4.9 / 5.3 / 8.1 us at 6K / 8K / 16K tokens, the cluster of eight
+// 7.0 / 5.8 / 7.6 us: one CTA up to 8K tokens, the cluster beyond.
 static int g_sel1_max_keys = 8192;
 #ifdef DAF_TRACE
 extern "C" void daf_dbg_sel1_max_keys(int n) { g_sel1_max_keys = n < kSel1MaxKeys ? n : kSel1MaxKeys; }
