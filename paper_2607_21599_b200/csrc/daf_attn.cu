@@ -516,7 +516,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
         }
     } else if (warp == 4) {
         // ------------------------------------------------------------ TMA producer (the rest of the sub-steps)
-        if (lane == 0 && n_t > 2) {
+        if (n_t > 2) {   // the whole warp walks the loop, one elected lane issues (uniform control flow)
             bool ok = true;
             for (int t = 2; t < n_t && ok; ++t) {
                 const int slot = t & 1;
@@ -524,10 +524,12 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
                 for (int kv = 0; kv < 2 && ok; ++kv) {
                     uint64_t* empty = kv == 0 ? &sm->k_empty[slot] : &sm->v_empty[slot];
                     ok = mbar_wait(empty, (round - 1) & 1u, abort_flag, status, 10 + 2 * kv + slot);
-                    if (ok) issue_kv(t, kv);
+                    ok = __all_sync(0xFFFFFFFFu, ok);
+                    if (ok && elect_one()) issue_kv(t, kv);
+                    __syncwarp();
                 }
             }
-            if (!ok) {
+            if (!ok && lane == 0) {
                 // give loads already in flight a bounded chance to land before the CTA retires
                 for (int s = 0; s < 2; ++s) {
                     for (int i = 0; i < 4096 && !mbar_try_wait(&sm->k_full[s], 0) && !mbar_try_wait(&sm->k_full[s], 1); ++i) {}
