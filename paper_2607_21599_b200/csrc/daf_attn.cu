@@ -356,9 +356,9 @@ extern "C" int daf_dbg_read_trace(void* host, size_t bytes) {
 // A tile's rows are (token, head) pairs: `Gp` query heads of one KV group times 128/Gp consecutive
 // tokens.  Gp = 1 for the packed causal attention; Gp = group size for the question rows, so that
 // one pass over the KV cache serves every query head of the group.
-//   - one thread issues TMA loads of Q and of K/V sub-tiles of 64 keys into shared-memory rings,
-//   - one thread issues tcgen05 MMAs: S = Q K^T into tensor memory, then O += P V with P read back
-//     from tensor memory,
+//   - one warp issues TMA loads of Q and of K/V sub-tiles of 64 keys into shared-memory rings,
+//   - one warp issues tcgen05 MMAs: S = Q K^T into tensor memory, then O += P V with P read back
+//     from tensor memory (in both, the warp walks its loop as a whole and an elected lane issues),
 //   - four warps run the online softmax, one thread per row, straight out of tensor memory, and
 //     write the final rows.
 // The keys go through in sub-steps of 64 and S is double-buffered (two 64-column halves of the
