@@ -235,6 +235,15 @@ int daf_layer_host(const daf_params* p, const float* h_scores, int32_t n_sig, co
  * DAF_OK, DAF_ERR_TIMEOUT or DAF_ERR_BOUNDS; the word is cleared. */
 int daf_poll_status(void* workspace, void* stream);
 
+/* Self-test of the failure path (no counterpart in the paper): launches one small CTA that waits, with the
+ * same bounded wait all kernels of this library use, on a barrier that nothing ever signals.  The wait gives
+ * up after `limit_ms` milliseconds (1..1000), the CTA records DAF_ERR_TIMEOUT in the status word of
+ * `workspace` (device memory, at least 256 bytes, e.g. a layer workspace) and returns normally: nothing
+ * traps and the context stays usable.  daf_poll_status then returns DAF_ERR_TIMEOUT once.  Returns DAF_OK
+ * when the launch was enqueued; DAF_ERR_WORKSPACE / DAF_ERR_INVALID_ARG for a missing workspace or a
+ * limit outside the range. */
+int daf_selftest_bounded_wait(void* workspace, size_t workspace_bytes, int32_t limit_ms, void* stream);
+
 /* Text for a daf_status; the numeric cudaError_t behind the last DAF_ERR_CUDA of this thread. */
 const char* daf_strerror(int status);
 int daf_last_cuda_error(void);

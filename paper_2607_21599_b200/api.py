@@ -31,7 +31,7 @@ EXPORTS = [
     "daf_qd_attn", "daf_fuse", "daf_full_causal_attn", "daf_layer", "daf_layer_host_arena_bytes",
     "daf_layer_host", "daf_poll_status", "daf_strerror", "daf_last_cuda_error", "daf_launch_count",
     "daf_qd_attn_static", "daf_qd_attn_static_max_bytes", "daf_deviation_scores", "daf_blend_attn",
-    "daf_imp_qd_attn",
+    "daf_imp_qd_attn", "daf_selftest_bounded_wait",
 ]
 
 
@@ -108,6 +108,8 @@ def lib() -> ctypes.CDLL:
         L.daf_layer_host.argtypes = [pp, vp, i32, vp] + [vp] * 3 + [vp, vp, i32] + [vp, vp] + [vp, sz, vp]
         L.daf_poll_status.restype = ctypes.c_int
         L.daf_poll_status.argtypes = [vp, vp]
+        L.daf_selftest_bounded_wait.restype = ctypes.c_int
+        L.daf_selftest_bounded_wait.argtypes = [vp, ctypes.c_size_t, ctypes.c_int32, vp]
         L.daf_strerror.restype = ctypes.c_char_p
         L.daf_strerror.argtypes = [ctypes.c_int]
         L.daf_last_cuda_error.restype = ctypes.c_int
@@ -259,6 +261,10 @@ def daf_layer_host(p, h_scores, n_sig, h_idx_in, h_q_fresh, h_k_fresh, h_v_fresh
 
 def daf_poll_status(workspace, stream=None) -> int:
     return lib().daf_poll_status(_ptr(workspace), _stream(stream))
+
+
+def daf_selftest_bounded_wait(workspace, limit_ms: int, stream=None) -> int:
+    return lib().daf_selftest_bounded_wait(_ptr(workspace), _nbytes(workspace), int(limit_ms), _stream(stream))
 
 
 def check(status: int, where: str = "daf") -> None:

@@ -408,6 +408,12 @@ int daf_poll_status(void* workspace, void* stream) {
     return hs.code;
 }
 
+int daf_selftest_bounded_wait(void* workspace, size_t workspace_bytes_, int32_t limit_ms, void* stream) {
+    if (workspace == nullptr || workspace_bytes_ < kStatusBytes) return DAF_ERR_WORKSPACE;
+    if (limit_ms < 1 || limit_ms > 1000) return DAF_ERR_INVALID_ARG;
+    return launch_bounded_wait_selftest(reinterpret_cast<DeviceStatus*>(workspace), limit_ms, (cudaStream_t)stream);
+}
+
 const char* daf_strerror(int status) {
     switch (status) {
         case DAF_OK: return "ok";

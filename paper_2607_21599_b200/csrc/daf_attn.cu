@@ -1104,6 +1104,27 @@ int launch_attention(const void* q, const void* k, const void* v, int n_q, int n
     return DAF_OK;
 }
 
+// Self-test of the bounded wait every kernel here relies on: two warps wait on a barrier that nothing ever
+// signals.  The wait has to give up within `limit_ns`, record DAF_ERR_TIMEOUT and let the CTA return.
+__global__ void __launch_bounds__(64)
+bounded_wait_selftest_kernel(DeviceStatus* status, unsigned long long limit_ns) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        abort_flag = 0;
+        mbar_fence_init();
+    }
+    __syncthreads();
+    mbar_wait(&bar, 0, &abort_flag, status, 900, limit_ns);
+}
+
+int launch_bounded_wait_selftest(DeviceStatus* status, int limit_ms, cudaStream_t stream) {
+    bounded_wait_selftest_kernel<<<1, 64, 0, stream>>>(status, (unsigned long long)limit_ms * 1000000ull);
+    count_launch();
+    return check_launch();
+}
+
 size_t joint_partial_bytes(const JointPlan& jp) { return jp.part_bytes_q + jp.part_bytes_i; }
 
 int launch_attention_joint(const void* q_imp, const void* q_fresh, const int32_t* idx, const void* k_imp, const void* v_imp,

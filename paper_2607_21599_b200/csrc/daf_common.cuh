@@ -60,6 +60,7 @@ struct JointPlan {
 };
 JointPlan plan_joint(int k, int L_q, int L_d, int Hq, int G);
 size_t joint_partial_bytes(const JointPlan& jp);
+int launch_bounded_wait_selftest(DeviceStatus* status, int limit_ms, cudaStream_t stream);
 // q_imp == nullptr: the important rows' Q is read in place, row idx[j] of q_fresh
 int launch_attention_joint(const void* q_imp, const void* q_fresh, const int32_t* idx, const void* k_imp, const void* v_imp,
                            int k, void* out_imp, const int32_t* dst_rows_imp, const void* q_question, const void* kv_k,
@@ -170,14 +171,14 @@ __device__ __forceinline__ unsigned long long global_ns() {
 #define DAF_KT_END(id) do {} while (0)
 #endif
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                          DeviceStatus* st, int where) {
+                                          DeviceStatus* st, int where, unsigned long long limit_ns = kWaitLimitNs) {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_ns();
     for (uint32_t it = 0; it < kWaitLimitPolls; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 31u) == 31u) {
             if (*abort_flag != 0) return false;
-            if (global_ns() - t0 > kWaitLimitNs) break;
+            if (global_ns() - t0 > limit_ns) break;
         }
     }
     *abort_flag = 1;

@@ -100,6 +100,11 @@ def test_host_side_argument_validation(lib):
     # a layer without question rows cannot read Q in place (only the joint launch does)
     no_q = api.make_params(256, 0, 0.25, 4, 2)
     assert api.daf_layer(no_q, buf, 1, None, buf, buf, buf, buf, buf, buf, None, buf, buf, buf, None, ws) == api.DAF_ERR_INVALID_ARG
+    # the self-test of the bounded wait checks its arguments before it launches anything
+    assert api.daf_selftest_bounded_wait(None, 50) == api.DAF_ERR_WORKSPACE
+    assert api.daf_selftest_bounded_wait(ws[:64], 50) == api.DAF_ERR_WORKSPACE
+    assert api.daf_selftest_bounded_wait(ws, 0) == api.DAF_ERR_INVALID_ARG
+    assert api.daf_selftest_bounded_wait(ws, 5000) == api.DAF_ERR_INVALID_ARG
     assert api.daf_launch_count() == 0
     assert "workspace" in api.daf_strerror(api.DAF_ERR_WORKSPACE)
     assert api.daf_layer_host(ok, None, 1, None, None, None, None, None, None, 0, None, None, None) == api.DAF_ERR_WORKSPACE

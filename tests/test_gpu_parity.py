@@ -442,6 +442,27 @@ def test_status_word_makes_kernels_stand_down_and_is_reported_once():
     _assert_close(out, oracle.important_attn(_f(q), _f(k), _f(v), 1.0 / math.sqrt(128)), "after clearing")
 
 
+def test_bounded_wait_runs_out_reports_and_leaves_the_context_usable():
+    """The wait every kernel relies on, pointed at a barrier that nothing signals: it gives up after the
+    limit, the status word says so, nothing faults, and the next call computes as usual."""
+    import time
+    n, Hq, Hkv = 200, 4, 2
+    p = api.make_params(n, 0, 1.0, Hq, Hkv)
+    ws = api.alloc_workspace(p)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    api.check(api.daf_selftest_bounded_wait(ws, 50), "self-test launch")
+    torch.cuda.synchronize()
+    waited = time.perf_counter() - t0
+    assert 0.04 <= waited < 5.0, f"the wait took {waited:.3f} s for a 50 ms limit"
+    assert api.daf_poll_status(ws) == api.DAF_ERR_TIMEOUT
+    assert api.daf_poll_status(ws) == api.DAF_OK
+    q, k, v = _normal((n, Hq, 128), 91), _normal((n, Hkv, 128), 92), _normal((n, Hkv, 128), 93)
+    out = torch.zeros((n, Hq, 128), dtype=torch.bfloat16, device="cuda")
+    _ok(api.daf_important_attn(p, n, q.cuda(), k.cuda(), v.cuda(), out, Hq * 256, None, None, ws), ws, "after the self-test")
+    _assert_close(out, oracle.important_attn(_f(q), _f(k), _f(v), 1.0 / math.sqrt(128)), "after the self-test")
+
+
 def test_out_of_range_index_is_skipped_and_reported():
     L_d, L_q, Hq, Hkv = 64, 2, 4, 2
     p = api.make_params(L_d, L_q, 4 / 64, Hq, Hkv)
