@@ -60,6 +60,10 @@ def _normal(shape, seed, scale=1.0):
     (16384, 0.10, 1, "constant"), (20000, 0.3, 2, "ties"), (40960, 0.2, 1, "lognormal"), (40961, 0.2, 1, "lognormal"),
     (7, 0.5, 1, "lognormal"), (1, 1.0, 1, "lognormal"), (12000, 0.2, 1, "special"), (16384, 0.5, 1, "ties"),
     (16385, 0.5, 1, "ties"), (2048, 0.05, 1, "narrow"),
+    # either side of the size at which the cluster kernel takes over; a cluster-sized problem whose keys differ
+    # only in their last byte (every radix pass is needed) and one whose keys differ only in the first two
+    (8192, 0.15, 1, "lognormal"), (8193, 0.15, 1, "lognormal"), (20000, 0.2, 1, "lowbyte"), (24000, 0.1, 1, "highbytes"),
+    (30000, 1.0, 1, "lognormal"), (30000, 0.0, 1, "lognormal"),
 ])
 def test_select_indices_bit_exact(L_d, r, n_sig, kind):
     if kind == "pareto":
@@ -74,6 +78,10 @@ def test_select_indices_bit_exact(L_d, r, n_sig, kind):
             S = torch.full_like(S, 1.5)
         if kind == "narrow":      # scores within a few ulps of each other: the key range needs only a few bits
             S = 1.0 + torch.floor(S * 4) * 2.0 ** -22
+        if kind == "lowbyte":     # 256 distinct values one ulp apart: many ties, decided by the last byte only
+            S = (1.0 + torch.floor(S * 37).remainder(256) * 2.0 ** -23).float()
+        if kind == "highbytes":   # powers of two times {1, 1.5}: the low two bytes of every key are zero
+            S = torch.pow(2.0, torch.floor(S * 3).remainder(40) - 20) * (1.0 + 0.5 * (torch.floor(S * 11).remainder(2)))
         if kind == "special":
             S[0, 3] = float("nan"); S[0, 4] = float("inf"); S[0, 5] = -float("inf")
             S[0, 6] = 0.0; S[0, 7] = -0.0; S[0, 8] = float("nan"); S[0, 9:40] = -S[0, 9:40]
