@@ -1,7 +1,12 @@
 #!/usr/bin/env python
 """Benchmark of the DAF prefill-attention path on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--config c1] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl ours|reference]
+
+Without --config the run covers the context range the metric is quoted on: the 32k
+configuration (c3, the largest single-GPU one) is the headline (`value`, `config`,
+`roofline`, `e2e`, `cpu_baseline`), and the 6k and 16k configurations (c1, c2) are
+measured the same way in the same process and reported under `by_config`.
 
 One step = one pass of the whole path (select + gather + hybrid-cache update,
 important-token attention, question-document attention with the fusion done by
@@ -17,6 +22,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import statistics
 import sys
@@ -33,10 +39,11 @@ from paper_2607_21599_b200 import workloads as W  # noqa: E402
 METRIC = "daf_prefill_attention_us_per_layer"
 UNIT = "us/layer"
 
-# DRAM bytes per launch of the dominant kernel from the ncu capture summarised under profiles/
-# (dram__bytes_read.sum + dram__bytes_write.sum); None where no capture exists for the workload.
 Q_IN_PLACE_MIN_K = 16384    # from this many important tokens on, the layer is called without a packed-Q buffer
-NCU_TRAFFIC_BYTES = {"c1": 21743104, "c3": 148381184}   # joint attention launch, profiles/attn_fwd_kernel_c1_c3.md
+# DRAM bytes per launch of the dominant kernel (the joint attention launch), dram__bytes_read.sum +
+# dram__bytes_write.sum of the committed ncu capture of that workload; no entry where none was captured.
+NCU_TRAFFIC_BYTES = {"c1": 21743104, "c3": 148381184}
+DEFAULT_PRIMARY, DEFAULT_OTHERS = "c3", ("c1", "c2")
 
 
 def _peaks():
@@ -133,6 +140,48 @@ def _config_dict(w: W.Workload, n_gpus: int):
             "l2_policy": "inputs larger than L2: every layer has its own tensors, a step touches far more than 126 MB"}
 
 
+# ----------------------------------------------------------------------------- the CPU oracle, timed
+ORACLE_PAIR_BUDGET = 6.0e7     # (row, key, head) triples per timed oracle call: about a second on 16 cores
+
+
+def _host_arrays(L):
+    f = lambda t: t.float().cpu().numpy()  # noqa: E731
+    return {n: (None if t is None else (f(t) if t.dtype == torch.bfloat16 else t.cpu().numpy())) for n, t in L.items()}
+
+
+def oracle_layer_seconds(oracle, A, w: W.Workload):
+    """Times the oracle, as it stands, on one layer.  Small layers run whole (oracle.daf_layer).  Layers
+    whose attention would take much longer than a second run selection, gather and cache update in full and
+    the two attention stages on every s-th query row; the attention time is scaled by the share of the
+    visible (row, key) pairs that the sampled rows cover.  Returns (seconds for the whole layer, description)."""
+    pairs = W.attention_pairs(w)
+    triples = (pairs["important"] + pairs["question"]) * w.n_q_heads
+    if triples <= ORACLE_PAIR_BUDGET:
+        t0 = time.perf_counter()
+        oracle.daf_layer(A["q_fresh"], A["k_fresh"], A["v_fresh"], A["k_cached"], A["v_cached"], w.L_d, w.L_q,
+                         w.softmax_scale, scores=A["scores"], idx=A["idx_in"], r=w.r)
+        return time.perf_counter() - t0, "whole layer"
+    import numpy as np
+    stride = int(math.ceil(triples / ORACLE_PAIR_BUDGET))
+    t0 = time.perf_counter()
+    k = oracle.num_important(w.L_d, w.r)
+    idx = oracle.select(A["scores"], k) if A["scores"] is not None else A["idx_in"]
+    q_pack, k_pack, v_pack = (oracle.gather_rows(A[n], idx) for n in ("q_fresh", "k_fresh", "v_fresh"))
+    kv_k = oracle.hybrid_kv(A["k_cached"], A["k_fresh"], idx, w.L_d, w.L_q)
+    kv_v = oracle.hybrid_kv(A["v_cached"], A["v_fresh"], idx, w.L_d, w.L_q)
+    t_move = time.perf_counter() - t0
+    rows_i = np.arange(stride // 2, k, stride, dtype=np.int32)
+    rows_q = np.arange(min(stride // 2, w.L_q - 1), w.L_q, stride, dtype=np.int32)
+    t0 = time.perf_counter()
+    oracle.important_attn(q_pack, k_pack, v_pack, w.softmax_scale, rows=rows_i)
+    oracle.qd_attn(A["q_fresh"][w.L_d:], kv_k, kv_v, w.L_d, w.softmax_scale, rows=rows_q)
+    t_attn = time.perf_counter() - t0
+    covered = int((rows_i.astype(np.int64) + 1).sum()) + int((rows_q.astype(np.int64) + 1 + w.L_d).sum())
+    share = covered / float(pairs["important"] + pairs["question"])
+    return t_move + t_attn / share, (f"selection, gather and cache update in full; attention on every {stride}th query row "
+                                    f"({share:.3%} of the visible pairs), attention time scaled by that share (extrapolated)")
+
+
 # ----------------------------------------------------------------------------- reference arm (the CPU oracle)
 def run_reference(args, w: W.Workload):
     rank, _, world = _dist_env()
@@ -140,26 +189,19 @@ def run_reference(args, w: W.Workload):
         return
     import oracle
     cores = oracle.num_threads()
-    f = lambda t: t.float().numpy()  # noqa: E731
-    layers = [W.make_layer(w, i % w.layers) for i in range(min(w.layers, max(1, args.steps + args.warmup)))]
-    arrs = [{n: (None if t is None else (f(t) if t.dtype == torch.bfloat16 else t.numpy())) for n, t in L.items()}
-            for L in layers]
-
-    def one(i):
-        A = arrs[i % len(arrs)]
-        oracle.daf_layer(A["q_fresh"], A["k_fresh"], A["v_fresh"], A["k_cached"], A["v_cached"], w.L_d, w.L_q,
-                         w.softmax_scale, scores=A["scores"], idx=A["idx_in"], r=w.r)
-
+    n_layers = min(w.layers, max(1, min(args.steps + args.warmup, 4)))
+    arrs = [_host_arrays(W.make_layer(w, i)) for i in range(n_layers)]
+    how = ""
     for i in range(args.warmup):
-        one(i)
-    t0 = time.perf_counter()
+        oracle_layer_seconds(oracle, arrs[i % n_layers], w)
+    total = 0.0
     for i in range(args.steps):
-        one(args.warmup + i)
-    dt = time.perf_counter() - t0
-    us_per_layer = dt / args.steps * 1e6
-    sample = f"each step = one layer of {w.name} through the fp64 CPU oracle (all {cores} OpenMP threads)"
+        dt, how = oracle_layer_seconds(oracle, arrs[(args.warmup + i) % n_layers], w)
+        total += dt
+    us_per_layer = total / args.steps * 1e6
+    sample = f"each step = one layer of {w.name} through the fp64 CPU oracle ({cores} OpenMP threads): {how}"
     line = {"impl": "reference", "metric": METRIC, "value": us_per_layer, "unit": UNIT, "n_gpus": args.gpus,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": total / args.steps * 1e3,
             "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": _config_dict(w, args.gpus),
             "cpu_baseline": {"value": us_per_layer, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
@@ -190,29 +232,45 @@ class LayerBuffers:
         self.k_pack = torch.empty(max(k, 1), Hkv, 128, dtype=bf, device=dev)
         self.v_pack = torch.empty(max(k, 1), Hkv, 128, dtype=bf, device=dev)
         self.hidden = torch.empty(k + w.L_q, Hq, 128, dtype=bf, device=dev)
-        self.full_out = None
         self.n_sig = 0 if L["scores"] is None else L["scores"].shape[0]
 
 
-def run_ours(args, w: W.Workload):
-    rank, local_rank, world = _dist_env()
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the DAF library has no CPU fallback")
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist_mod
-        dist = dist_mod
-        dist.init_process_group("nccl", device_id=dev)
-    from paper_2607_21599_b200 import api, build
-    if rank == 0 or world == 1:
-        build.build()
-    if dist is not None:
-        dist.barrier()
-    api.lib()
-    peaks = _peaks()
+class Env:
+    """What every measured configuration shares: the device, the rank plumbing, the library, the peaks."""
 
+    def __init__(self, args):
+        self.args = args
+        self.rank, self.local_rank, self.world = _dist_env()
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device: the DAF library has no CPU fallback")
+        torch.cuda.set_device(self.local_rank)
+        self.dev = torch.device("cuda", self.local_rank)
+        self.dist = None
+        if self.world > 1:
+            import torch.distributed as dist_mod
+            self.dist = dist_mod
+            self.dist.init_process_group("nccl", device_id=self.dev)
+        from paper_2607_21599_b200 import api, build
+        if self.rank == 0 or self.world == 1:
+            build.build()
+        if self.dist is not None:
+            self.dist.barrier()
+        api.lib()
+        self.api = api
+        self.peaks = _peaks()
+        self.use_graph = not args.no_graph
+
+    def barrier(self):
+        torch.cuda.synchronize()
+        if self.dist is not None:
+            self.dist.barrier()
+            torch.cuda.synchronize()
+
+
+def measure_config(env: Env, w: W.Workload, primary: bool):
+    """All measurements of one workload.  Returns the fields of the JSON line that belong to it."""
+    args, api, dev, dist, rank, world, peaks = env.args, env.api, env.dev, env.dist, env.rank, env.world, env.peaks
+    use_graph, barrier = env.use_graph, env.barrier
     p = api.make_params(w.L_d, w.L_q, w.r, w.n_q_heads, w.n_kv_heads)
     ws = api.alloc_workspace(p, dev)
     # every rank owns its own replica of the workload (distinct seeds per rank): weak scaling, no exchange
@@ -249,9 +307,12 @@ def run_ours(args, w: W.Workload):
         api.check(api.daf_qd_attn(p, b.L["q_fresh"][w.L_d:], b.kv_k, b.kv_v, b.hidden, row_bytes, None, None, ws,
                                   out_offset_bytes=b.k * row_bytes), "daf_qd_attn")
 
-    def st_both(b):
-        api.check(api.daf_imp_qd_attn(p, None if q_in_place else b.q_pack, b.L["q_fresh"], b.k_pack, b.v_pack,
-                                      b.L["q_fresh"][w.L_d:], b.kv_k, b.kv_v, b.idx_out, b.hidden, ws), "daf_imp_qd_attn")
+    def st_both_launches(which):
+        def run(b):
+            api.check(api.daf_imp_qd_attn_launches(p, None if q_in_place else b.q_pack, b.L["q_fresh"], b.k_pack, b.v_pack,
+                                                   b.L["q_fresh"][w.L_d:], b.kv_k, b.kv_v, b.idx_out, b.hidden, ws, which),
+                      "daf_imp_qd_attn_launches")
+        return run
 
     n_full = min(len(bufs), 4)
     pf = api.make_params(w.N, 0, 1.0, w.n_q_heads, w.n_kv_heads)
@@ -267,12 +328,6 @@ def run_ours(args, w: W.Workload):
             for b in items:
                 fn(b)
         return run
-
-    def barrier():
-        torch.cuda.synchronize()
-        if dist is not None:
-            dist.barrier()
-            torch.cuda.synchronize()
 
     def capture(run):
         """Records `run` (one pass over the layers) into a CUDA graph: a replay issues the same kernels
@@ -299,7 +354,7 @@ def run_ours(args, w: W.Workload):
     barrier()
     api.check(api.daf_poll_status(ws), "warm-up (device status)")
 
-    use_graph = not args.no_graph
+    launches_per_step = 0
     if use_graph:
         g_step, launches_per_step = capture(step)
         g_step.replay()
@@ -308,7 +363,7 @@ def run_ours(args, w: W.Workload):
     stream = torch.cuda.current_stream()
     launches0 = api.daf_launch_count()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    with ClockSampler(local_rank) as clocks:
+    with ClockSampler(env.local_rank) as clocks:
         barrier()
         e0.record(stream)
         for _ in range(args.steps):
@@ -360,26 +415,41 @@ def run_ours(args, w: W.Workload):
     us_select = time_stage(st_select, bufs)
     us_imp = time_stage(st_imp, bufs) if w.k > 0 else 0.0
     us_qd = time_stage(st_qd, bufs) if w.L_q > 0 else 0.0
-    # the two attention stages the way the layer runs them: one launch over both stages' work items, one merge launch
-    us_both = time_stage(st_both, bufs) if both else (us_imp + us_qd)
+    # the two attention stages the way the layer runs them: one launch over both stages' work items and one merge
+    # launch; each launch is also timed alone (the attention launch writes the partial rows the merge launch reads)
+    if both:
+        with ClockSampler(env.local_rank) as clocks_attn:
+            us_kernel = time_stage(st_both_launches(1), bufs)
+        us_merge = time_stage(st_both_launches(2), bufs)
+        us_both = time_stage(st_both_launches(3), bufs)
+    else:
+        clocks_attn = clocks
+        us_kernel, us_merge, us_both = us_imp + us_qd, 0.0, us_imp + us_qd
     # full recompute on the same kernel (comparison path), bounded number of layers
-    us_full = time_stage(st_full, bufs[:n_full], reps=3)
+    with ClockSampler(env.local_rank) as clocks_full:
+        us_full = time_stage(st_full, bufs[:n_full], reps=3)
     # selective recomputation over the FULL context on the same kernel (the r L_d^2 + L_d L_q scheme of the
     # paper's complexity analysis): the compact rows attend every earlier key of the hybrid cache
-    blend_rows, blend_pairs = [], 0
-    for b in bufs[:n_full]:
-        pos = torch.cat([b.idx_out[: b.k], torch.arange(w.L_d, w.N, dtype=torch.int32, device=dev)])
-        b.row_pos = pos.contiguous()
-        b.q_rows = b.L["q_fresh"][pos.long()].contiguous()
-        blend_pairs += int((pos.long() + 1).sum().item())
-    blend_out = torch.empty(w.k + w.L_q, Hq, 128, dtype=torch.bfloat16, device=dev)
+    blend = None
+    if primary or args.config is not None:
+        blend_pairs = 0
+        for b in bufs[:n_full]:
+            pos = torch.cat([b.idx_out[: b.k], torch.arange(w.L_d, w.N, dtype=torch.int32, device=dev)])
+            b.row_pos = pos.contiguous()
+            b.q_rows = b.L["q_fresh"][pos.long()].contiguous()
+            blend_pairs += int((pos.long() + 1).sum().item())
+        blend_out = torch.empty(w.k + w.L_q, Hq, 128, dtype=torch.bfloat16, device=dev)
 
-    def st_blend(b):
-        api.check(api.daf_blend_attn(p, w.k + w.L_q, b.q_rows, b.kv_k, b.kv_v, b.row_pos, blend_out, row_bytes, None,
-                                     ws), "daf_blend_attn")
+        def st_blend(b):
+            api.check(api.daf_blend_attn(p, w.k + w.L_q, b.q_rows, b.kv_k, b.kv_v, b.row_pos, blend_out, row_bytes, None,
+                                         ws), "daf_blend_attn")
 
-    us_blend = time_stage(st_blend, bufs[:n_full], reps=3)
-    blend_flops = 4.0 * w.head_dim * Hq * blend_pairs / n_full
+        us_blend = time_stage(st_blend, bufs[:n_full], reps=3)
+        blend_flops = 4.0 * w.head_dim * Hq * blend_pairs / n_full
+        blend = {"us_per_layer": us_blend, "tflops": blend_flops / (us_blend * 1e-6) / 1e12,
+                 "flop_ratio_vs_daf": blend_flops / daf_flops,
+                 "time_ratio_vs_daf_attention": us_blend / max(us_both, 1e-9),
+                 "note": "comparison only: important + question rows attend the whole hybrid cache"}
     api.check(api.daf_poll_status(wsf), "full recompute (device status)")
     api.check(api.daf_poll_status(ws), "stage timing (device status)")
 
@@ -390,24 +460,31 @@ def run_ours(args, w: W.Workload):
     gather_bytes = 2 * w.k * packed_heads * 256 + (w.k + 2 * w.L_q) * 2 * w.n_kv_heads * 256
     dev_bytes = 4 * w.L_d * w.n_kv_heads * 256 + 4 * w.L_d
 
+    kernel_tflops = daf_flops / (us_kernel * 1e-6) / 1e12 if us_kernel else 0.0
     both_tflops = daf_flops / (us_both * 1e-6) / 1e12 if us_both else 0.0
+    pairs = W.attention_pairs(w)
     roofline = {
-        "kernel": "attn_fwd_kernel (important-token and question stages as one launch; the time includes the merge launch)",
+        "kernel": "attn_fwd_kernel, the launch a layer makes: important-token and question work items in one grid",
         "bound": "tensor",
-        "achieved": both_tflops,
+        "flops_per_launch": daf_flops,
+        "flops_formula": f"4*D*Hq*pairs = 4*128*{Hq}*({pairs['important']} + {pairs['question']})",
+        "kernel_us": us_kernel, "merge_us": us_merge, "kernel_plus_merge_us": us_both,
+        "achieved": kernel_tflops,
         "peak": peaks["bf16_tflops"],
         "unit": "TFLOP/s",
-        "frac": both_tflops / peaks["bf16_tflops"],
-        "peak_source": f"{peaks['source']} bf16 burst (kernel timed alone)",
+        "frac": kernel_tflops / peaks["bf16_tflops"],
+        "frac_with_merge": both_tflops / peaks["bf16_tflops"],
+        "peak_source": f"{peaks['source']} bf16 burst (kernel timed alone, all layers back to back)",
         "traffic": NCU_TRAFFIC_BYTES.get(w.name),
+        "clocks": clocks_attn.summary(),
     }
 
     # ---- end to end through the host-buffer entry point (pinned host tensors, copies inside the timed region)
     e2e = None
-    if rank == 0 or world > 1:
+    if primary and (rank == 0 or world > 1):
         per_layer_in = (w.N * (w.n_q_heads + 2 * w.n_kv_heads) + 2 * w.L_d * w.n_kv_heads) * 256 + \
                        (w.L_d * 4 * max(bufs[0].n_sig, 1))
-        n_e2e = max(1, min(w.layers, int(4e9 // per_layer_in)))
+        n_e2e = max(1, min(w.layers, int(2e9 // per_layer_in)))
         arena = torch.zeros(api.daf_layer_host_arena_bytes(p), dtype=torch.uint8, device=dev)
         host = []
         for b in bufs[:n_e2e]:
@@ -443,57 +520,89 @@ def run_ours(args, w: W.Workload):
 
     # ---- CPU oracle on this machine's cores, bounded sample (rank 0, N = 1 only)
     cpu_baseline = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if primary and rank == 0 and world == 1 and not args.no_cpu_baseline:
         import oracle
-        f = lambda t: t.float().cpu().numpy()  # noqa: E731
-        t_cpu, n_cpu = 0.0, 0
-        while t_cpu < 10.0 and n_cpu < w.layers:
-            L = bufs[n_cpu].L
-            A = {n: (None if t is None else (f(t) if t.dtype == torch.bfloat16 else t.cpu().numpy())) for n, t in L.items()}
-            t0 = time.perf_counter()
-            oracle.daf_layer(A["q_fresh"], A["k_fresh"], A["v_fresh"], A["k_cached"], A["v_cached"], w.L_d, w.L_q,
-                             w.softmax_scale, scores=A["scores"], idx=A["idx_in"], r=w.r)
-            t_cpu += time.perf_counter() - t0
+        t_cpu, n_cpu, how = 0.0, 0, ""
+        while t_cpu < 10.0 and n_cpu < min(w.layers, 8):
+            dt, how = oracle_layer_seconds(oracle, _host_arrays(bufs[n_cpu].L), w)
+            t_cpu += dt
             n_cpu += 1
         cpu_baseline = {"value": t_cpu / n_cpu * 1e6, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-                        "sample": f"first {n_cpu} of {w.layers} layers of {w.name}, whole DAF path per layer, fp64 oracle"}
+                        "sample": f"first {n_cpu} of {w.layers} layers of {w.name}, fp64 oracle: {how}"}
 
-    if rank == 0:
+    speedup = us_full / us_per_layer / world if world == 1 else None
+    flop_ratio = flops["full"] / daf_flops
+    res = {
+        "value": us_per_layer, "unit": UNIT, "ms_per_step": ms_per_step, "config": _config_dict(w, world),
+        "tflops": tflops, "frac_of_bf16_peak": tflops / (peaks["bf16_tflops"] * world),
+        "roofline": roofline,
+        "stages_us": {"select_gather_update": us_select, "imp_qd_attn": us_both, "imp_qd_attn_kernel_only": us_kernel,
+                      "merge_only": us_merge, "important_attn_alone": us_imp, "question_attn_alone": us_qd},
+        "stages": {
+            "important_attn": {"bound": "tensor", "tflops": imp_tflops, "frac": imp_tflops / peaks["bf16_tflops"]},
+            "question_attn": {"bound": "tensor", "tflops": qd_tflops, "frac": qd_tflops / peaks["bf16_tflops"],
+                              "kv_gbs": 2 * w.N * w.n_kv_heads * 256 / (us_qd * 1e-6) / 1e9 if us_qd else None},
+            "deviation_scores": {"bound": "hbm", "us": us_dev, "gbs": dev_bytes / (us_dev * 1e-6) / 1e9,
+                                 "frac": dev_bytes / (us_dev * 1e-6) / 1e9 / peaks["hbm_gbs"],
+                                 "note": "signal layers only; not part of the per-layer step"},
+            "select_gather_update": {"bound": "hbm", "gbs": gather_bytes / (us_select * 1e-6) / 1e9,
+                                     "frac": gather_bytes / (us_select * 1e-6) / 1e9 / peaks["hbm_gbs"],
+                                     "note": "includes the latency-bound top-k kernel"},
+        },
+        "full_recompute": {"us_per_layer": us_full, "tflops": full_tflops, "frac": full_tflops / peaks["bf16_tflops"],
+                           "speedup_daf_vs_full": speedup, "flop_ratio": flop_ratio,
+                           "speedup_over_flop_ratio": (speedup / flop_ratio) if speedup else None,
+                           "layers_timed": n_full, "clocks": clocks_full.summary()},
+        "clocks": clocks.summary(),
+        "gpu_launches": int(launches),
+    }
+    if "sw_power_cap" in res["clocks"]["reasons"] or "sw_power_cap" in roofline["clocks"]["reasons"]:
+        res["clocks_note"] = "sw_power_cap was active during the timed region (1 kW part under dense tensor work); number kept"
+    if blend is not None:
+        res["full_context_variant"] = blend
+    if e2e is not None:
+        res["e2e"] = e2e
+    if cpu_baseline is not None:
+        res["cpu_baseline"] = cpu_baseline
+    del bufs, ws, wsf, full_out
+    torch.cuda.empty_cache()
+    return res
+
+
+def run_ours(args, primary_w: W.Workload, others):
+    env = Env(args)
+    by_config = {}
+    for w in others:
+        by_config[w.name] = measure_config(env, w, primary=False)
+    res = measure_config(env, primary_w, primary=True)
+    if env.rank == 0:
         line = {
-            "metric": METRIC, "value": us_per_layer, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak",
-            "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": _config_dict(w, world),
-            "tflops": tflops, "frac_of_bf16_peak": tflops / (peaks["bf16_tflops"] * world),
-            "roofline": roofline,
-            "stages_us": {"select_gather_update": us_select, "imp_qd_attn": us_both, "important_attn_alone": us_imp,
-                          "question_attn_alone": us_qd},
-            "stages": {
-                "imp_qd_attn": {"bound": "tensor", "tflops": both_tflops, "frac": both_tflops / peaks["bf16_tflops"]},
-                "important_attn": {"bound": "tensor", "tflops": imp_tflops, "frac": imp_tflops / peaks["bf16_tflops"]},
-                "question_attn": {"bound": "tensor", "tflops": qd_tflops, "frac": qd_tflops / peaks["bf16_tflops"],
-                                  "kv_gbs": 2 * w.N * w.n_kv_heads * 256 / (us_qd * 1e-6) / 1e9 if us_qd else None},
-                "deviation_scores": {"bound": "hbm", "us": us_dev, "gbs": dev_bytes / (us_dev * 1e-6) / 1e9,
-                                     "frac": dev_bytes / (us_dev * 1e-6) / 1e9 / peaks["hbm_gbs"],
-                                     "note": "signal layers only; not part of the per-layer step"},
-                "select_gather_update": {"bound": "hbm", "gbs": gather_bytes / (us_select * 1e-6) / 1e9,
-                                         "frac": gather_bytes / (us_select * 1e-6) / 1e9 / peaks["hbm_gbs"],
-                                         "note": "includes the latency-bound top-k kernel"},
-            },
-            "full_recompute": {"us_per_layer": us_full, "tflops": full_tflops, "frac": full_tflops / peaks["bf16_tflops"],
-                               "speedup_daf_vs_full": us_full / us_per_layer / world if world == 1 else None,
-                               "flop_ratio": flops["full"] / daf_flops, "layers_timed": n_full},
-            "full_context_variant": {"us_per_layer": us_blend, "tflops": blend_flops / (us_blend * 1e-6) / 1e12,
-                                     "flop_ratio_vs_daf": blend_flops / daf_flops,
-                                     "time_ratio_vs_daf_attention": us_blend / max(us_both, 1e-9),
-                                     "note": "comparison only: important + question rows attend the whole hybrid cache"},
-            "launch_mode": "cuda_graph_replay" if use_graph else "eager",
-            "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks.summary(),
-            "peaks": peaks, "cpu_baseline": cpu_baseline,
+            "metric": METRIC, "value": res.pop("value"), "unit": res.pop("unit"), "n_gpus": env.world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": res.pop("ms_per_step"), "higher_is_better": False,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": res.pop("config"),
         }
+        line.update(res)
+        line["launch_mode"] = "cuda_graph_replay" if env.use_graph else "eager"
+        line["peaks"] = env.peaks
+        line.setdefault("e2e", None)
+        line.setdefault("cpu_baseline", None)
+        if by_config:
+            line["by_config"] = by_config
         print(json.dumps(line))
-    if dist is not None:
-        dist.barrier()
-        dist.destroy_process_group()
+    if env.dist is not None:
+        env.dist.barrier()
+        env.dist.destroy_process_group()
+
+
+def _lookup(name, num_important):
+    if name in W.CONFIGS:
+        return W.CONFIGS[name]
+    if name in W.EXTRA_CONFIGS:
+        return W.EXTRA_CONFIGS[name]
+    pts = {x.name: x for x in W.sweep_points(num_important)}
+    if name not in pts:
+        raise SystemExit(f"unknown config {name}; choose from {list(W.CONFIGS) + list(W.EXTRA_CONFIGS) + list(pts)}")
+    return pts[name]
 
 
 def main():
@@ -502,27 +611,28 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--config", default="c1", help="c0..c3, a sweep point name (c4_L<L_d>_r<r>) or x136k")
+    ap.add_argument("--config", default=None,
+                    help="one workload only: c0..c3, a sweep point name (c4_L<L_d>_r<r>) or x136k; "
+                         f"default: {DEFAULT_PRIMARY} as the headline with {', '.join(DEFAULT_OTHERS)} under by_config")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying a CUDA graph")
     ap.add_argument("--layers", type=int, default=0, help="use only the first LAYERS layers (profiling captures)")
     args = ap.parse_args()
-    if args.config in W.CONFIGS:
-        w = W.CONFIGS[args.config]
-    elif args.config in W.EXTRA_CONFIGS:
-        w = W.EXTRA_CONFIGS[args.config]
-    else:
-        pts = {x.name: x for x in W.sweep_points()}
-        if args.config not in pts:
-            raise SystemExit(f"unknown config {args.config}; choose from {list(W.CONFIGS) + list(pts)}")
-        w = pts[args.config]
-    if args.layers > 0:
-        import dataclasses
-        w = dataclasses.replace(w, layers=min(args.layers, w.layers))
+    import dataclasses
+    cut = (lambda w: dataclasses.replace(w, layers=min(args.layers, w.layers))) if args.layers > 0 else (lambda w: w)
     if args.impl == "reference":
-        run_reference(args, w)
+        import oracle
+        count = oracle.num_important
     else:
-        run_ours(args, w)
+        from paper_2607_21599_b200 import api, build
+        build.build()
+        count = api.daf_num_important
+    primary = cut(_lookup(args.config or DEFAULT_PRIMARY, count))
+    others = [] if args.config else [cut(_lookup(n, count)) for n in DEFAULT_OTHERS]
+    if args.impl == "reference":
+        run_reference(args, primary)
+    else:
+        run_ours(args, primary, others)
 
 
 if __name__ == "__main__":

@@ -64,7 +64,7 @@ typedef struct daf_params {
 
 /* Number of important tokens k = ceil(r * L_d), clamped to [0, L_d].  r*L_d is
  * shrunk by a relative 1e-6 first so that an r rounded to single precision gives
- * the intended count.  (Notation paragraph: "r is the fraction of important tokens".) */
+ * the intended count.  (Methods, notation paragraph: r, the share of the document tokens that is recomputed.) */
 int32_t daf_num_important(int32_t L_d, double r);
 
 /* Bytes of device scratch every call below may need for this problem (selection
@@ -162,6 +162,16 @@ int daf_imp_qd_attn(const daf_params* p, const void* q_pack, const void* q_fresh
                     const void* q_question, const void* kv_k, const void* kv_v, const int32_t* idx,
                     void* hidden, void* workspace, size_t workspace_bytes, void* stream);
 
+/* Measurement aid (no counterpart in the paper): daf_imp_qd_attn with only part of its work enqueued, so
+ * that the attention launch and the merge launch can be timed apart.  launches = 1: the attention launch
+ * alone (final rows of the items that cover all their keys, partial results of the others, into the
+ * workspace); 2: the merge launch alone (reads the partial results a launches = 1 call left in the same
+ * workspace); 3: both, i.e. daf_imp_qd_attn.  Other values: DAF_ERR_INVALID_ARG. */
+int daf_imp_qd_attn_launches(const daf_params* p, const void* q_pack, const void* q_fresh, const void* k_pack,
+                             const void* v_pack, const void* q_question, const void* kv_k, const void* kv_v,
+                             const int32_t* idx, void* hidden, void* workspace, size_t workspace_bytes, void* stream,
+                             int32_t launches);
+
 /* daf_qd_attn for callers that cannot provide a workspace.  (The paper has no
  * counterpart of this entry point; it exists for integration only.)
  *
@@ -182,12 +192,16 @@ int daf_imp_qd_attn(const daf_params* p, const void* q_pack, const void* q_fresh
  *   - All calls on one device share the array, and it keeps the previous call's
  *     contents; the call clears the part that must start at zero.  Two calls that
  *     may overlap on the GPU (different streams) race on it: serialise them.
- *   - Device-side status is not reported through daf_poll_status here; results
- *     are exactly those of daf_qd_attn. */
+ *   - Device-side status (a bounded wait that ran out) is kept at the head of
+ *     that array: daf_qd_attn_static_poll_status reads and clears it, as
+ *     daf_poll_status does for a workspace, also without allocating.
+ *   - Host threads may make their first calls concurrently; they resolve the same
+ *     address.  Results are exactly those of daf_qd_attn. */
 int daf_qd_attn_static(const daf_params* p, const void* q_question, const void* kv_k, const void* kv_v,
                        void* out, int64_t out_row_stride_bytes, const int32_t* dst_rows, float* lse,
                        void* stream);
 size_t daf_qd_attn_static_max_bytes(void);
+int daf_qd_attn_static_poll_status(void* stream);
 
 /* Step 4 (Methods item 3), stand-alone form: copy o_imp [k, n_q_heads*128] and
  * o_q [L_q, n_q_heads*128] into `hidden`: compact mode -> rows 0..k+L_q-1 of a

@@ -46,7 +46,7 @@
 #endif
 
 /* Number of important tokens for a fraction r of L_d document tokens
- * (Methods, notation paragraph: "r is the fraction of important tokens").
+ * (Methods, notation paragraph: r, the share of the document tokens that is recomputed).
  * Reading: k = ceil(r * L_d), clamped to [0, L_d].  The product is shrunk by a
  * relative 1e-6 before the ceiling so that an r that was rounded to single
  * precision (0.1f * 1000 = 100.0000015) still gives the intended count. */

@@ -31,7 +31,8 @@ EXPORTS = [
     "daf_qd_attn", "daf_fuse", "daf_full_causal_attn", "daf_layer", "daf_layer_host_arena_bytes",
     "daf_layer_host", "daf_poll_status", "daf_strerror", "daf_last_cuda_error", "daf_launch_count",
     "daf_qd_attn_static", "daf_qd_attn_static_max_bytes", "daf_deviation_scores", "daf_blend_attn",
-    "daf_imp_qd_attn", "daf_selftest_bounded_wait",
+    "daf_imp_qd_attn", "daf_selftest_bounded_wait", "daf_qd_attn_static_poll_status",
+    "daf_imp_qd_attn_launches",
 ]
 
 
@@ -90,8 +91,12 @@ def lib() -> ctypes.CDLL:
         L.daf_qd_attn_static.argtypes = [pp, vp, vp, vp, vp, i64, vp, vp, vp]
         L.daf_qd_attn_static_max_bytes.restype = sz
         L.daf_qd_attn_static_max_bytes.argtypes = []
+        L.daf_qd_attn_static_poll_status.restype = ctypes.c_int
+        L.daf_qd_attn_static_poll_status.argtypes = [vp]
         L.daf_imp_qd_attn.restype = ctypes.c_int
         L.daf_imp_qd_attn.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.daf_imp_qd_attn_launches.restype = ctypes.c_int
+        L.daf_imp_qd_attn_launches.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp, i32]
         L.daf_blend_attn.restype = ctypes.c_int
         L.daf_blend_attn.argtypes = [pp, i32, vp, vp, vp, vp, vp, i64, vp, vp, sz, vp]
         L.daf_deviation_scores.restype = ctypes.c_int
@@ -209,10 +214,21 @@ def daf_qd_attn_static_max_bytes() -> int:
     return int(lib().daf_qd_attn_static_max_bytes())
 
 
+def daf_qd_attn_static_poll_status(stream=None) -> int:
+    return lib().daf_qd_attn_static_poll_status(_stream(stream))
+
+
 def daf_imp_qd_attn(p, q_pack, q_fresh, k_pack, v_pack, q_question, kv_k, kv_v, idx, hidden, workspace, stream=None) -> int:
     return lib().daf_imp_qd_attn(ctypes.byref(p), _ptr(q_pack), _ptr(q_fresh), _ptr(k_pack), _ptr(v_pack), _ptr(q_question),
                                  _ptr(kv_k), _ptr(kv_v), _ptr(idx), _ptr(hidden), _ptr(workspace), _nbytes(workspace),
                                  _stream(stream))
+
+
+def daf_imp_qd_attn_launches(p, q_pack, q_fresh, k_pack, v_pack, q_question, kv_k, kv_v, idx, hidden, workspace, launches,
+                             stream=None) -> int:
+    return lib().daf_imp_qd_attn_launches(ctypes.byref(p), _ptr(q_pack), _ptr(q_fresh), _ptr(k_pack), _ptr(v_pack),
+                                          _ptr(q_question), _ptr(kv_k), _ptr(kv_v), _ptr(idx), _ptr(hidden), _ptr(workspace),
+                                          _nbytes(workspace), _stream(stream), int(launches))
 
 
 def daf_blend_attn(p, n_rows, q_rows, kv_k, kv_v, row_pos, out, out_row_stride_bytes, lse, workspace, stream=None) -> int:

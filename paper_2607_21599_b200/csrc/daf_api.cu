@@ -181,6 +181,14 @@ int daf_qd_attn(const daf_params* p, const void* q_question, const void* kv_k, c
 int daf_imp_qd_attn(const daf_params* p, const void* q_pack, const void* q_fresh, const void* k_pack, const void* v_pack,
                     const void* q_question, const void* kv_k, const void* kv_v, const int32_t* idx,
                     void* hidden, void* workspace, size_t workspace_bytes_, void* stream) {
+    return daf_imp_qd_attn_launches(p, q_pack, q_fresh, k_pack, v_pack, q_question, kv_k, kv_v, idx, hidden, workspace,
+                                    workspace_bytes_, stream, 3);
+}
+
+int daf_imp_qd_attn_launches(const daf_params* p, const void* q_pack, const void* q_fresh, const void* k_pack, const void* v_pack,
+                             const void* q_question, const void* kv_k, const void* kv_v, const int32_t* idx,
+                             void* hidden, void* workspace, size_t workspace_bytes_, void* stream, int32_t launches) {
+    if (launches < 1 || launches > 3) return DAF_ERR_INVALID_ARG;
     ResolvedParams rp;
     if (int rc = resolve_params(p, &rp)) return rc;
     Workspace ws;
@@ -198,7 +206,7 @@ int daf_imp_qd_attn(const daf_params* p, const void* q_pack, const void* q_fresh
     const int64_t first_row = rp.fuse_mode == 1 ? rp.L_d : rp.k;
     return launch_attention_joint(q_pack, q_fresh, idx, k_pack, v_pack, rp.k, h, rp.fuse_mode == 1 ? idx : nullptr, q_question, kv_k, kv_v,
                                   rp.L_q, rp.L_d, h + first_row * row_bytes, row_bytes, rp.Hq, rp.Hkv, rp.scale, ws.status,
-                                  ws.attn_scratch, ws.attn_bytes, (cudaStream_t)stream, /*after_kernel=*/false);
+                                  ws.attn_scratch, ws.attn_bytes, (cudaStream_t)stream, /*after_kernel=*/false, launches);
 }
 
 int daf_blend_attn(const daf_params* p, int32_t n_rows, const void* q_rows, const void* kv_k, const void* kv_v,
@@ -272,6 +280,10 @@ int daf_layer(const daf_params* p, const float* scores, int32_t n_sig, const int
     if (rp.k + rp.L_q == 0) return DAF_OK;
     if (rp.k > 0 && idx_out == nullptr) return DAF_ERR_INVALID_ARG;
     if (rp.k > 0 && rp.L_q == 0 && q_pack == nullptr) return DAF_ERR_INVALID_ARG;   // only the joint launch reads Q in place
+    // the question rows are read from q_fresh even when nothing is selected (r = 0)
+    if (rp.L_q > 0 && (q_fresh == nullptr || kv_k == nullptr || kv_v == nullptr)) return DAF_ERR_INVALID_ARG;
+    if (rp.k > 0 && (q_fresh == nullptr || k_pack == nullptr || v_pack == nullptr)) return DAF_ERR_INVALID_ARG;
+    if (q_fresh != nullptr && !aligned16(q_fresh)) return DAF_ERR_ALIGNMENT;
     const int64_t row_bytes = (int64_t)rp.Hq * 256;
     if (int rc = check_out(hidden, row_bytes, rp.Hq)) return rc;
     if (int rc = do_select(rp, scores, n_sig, idx_in, q_fresh, k_fresh, v_fresh, kv_k, kv_v, idx_out, q_pack, k_pack,

@@ -10,6 +10,7 @@
 #include <math.h>
 #include <string.h>
 
+#include <atomic>
 #include <functional>
 #include <map>
 #include <mutex>
@@ -827,13 +828,14 @@ static int make_tmap(CUtensorMap* m, const void* base, int tokens, int heads, in
 }
 
 static int set_kernel_attributes() {
-    static bool attr_done[64] = {false};
+    // per device, set once; concurrent first calls may both set it (the same value), which is harmless
+    static std::atomic<bool> attr_done[64];
     int dev = 0;
     cudaGetDevice(&dev);
-    if (dev >= 0 && dev < 64 && !attr_done[dev]) {
+    if (dev >= 0 && dev < 64 && !attr_done[dev].load(std::memory_order_acquire)) {
         cudaError_t e = cudaFuncSetAttribute(attn_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttnSmemBytes);
         if (e != cudaSuccess) { set_cuda_error(e); return DAF_ERR_CUDA; }
-        attr_done[dev] = true;
+        attr_done[dev].store(true, std::memory_order_release);
     }
     return DAF_OK;
 }
@@ -1132,7 +1134,7 @@ int launch_attention_joint(const void* q_imp, const void* q_fresh, const int32_t
                            const void* kv_v,
                            int L_q, int L_d, void* out_question, long long out_row_stride_bytes, int Hq, int Hkv,
                            float scale, DeviceStatus* status, void* scratch, size_t scratch_bytes, cudaStream_t stream,
-                           bool after_kernel) {
+                           bool after_kernel, int launches) {
     const int G = Hq / Hkv, N = L_d + L_q;
     const JointPlan jp = plan_joint(k, L_q, L_d, Hq, G);
     if (joint_partial_bytes(jp) > scratch_bytes) return DAF_ERR_WORKSPACE;
@@ -1180,11 +1182,14 @@ int launch_attention_joint(const void* q_imp, const void* q_fresh, const int32_t
     a.status = status;
 
     const int items = jp.items_q + jp.items_i;
-    const cudaError_t e = launch_kernel(attn_fwd_kernel, dim3((unsigned)items), dim3(kAttnThreads), kAttnSmemBytes, stream,
-                                        after_kernel, tq0, tk0, tv0, tq1, tk1, tv1, a);
-    count_launch();
-    if (e != cudaSuccess) { set_cuda_error(e); return DAF_ERR_CUDA; }
-    if (int rc = check_launch()) return rc;
+    if (launches & 1) {
+        const cudaError_t e = launch_kernel(attn_fwd_kernel, dim3((unsigned)items), dim3(kAttnThreads), kAttnSmemBytes, stream,
+                                            after_kernel, tq0, tk0, tv0, tq1, tk1, tv1, a);
+        count_launch();
+        if (e != cudaSuccess) { set_cuda_error(e); return DAF_ERR_CUDA; }
+        if (int rc = check_launch()) return rc;
+    }
+    if (!(launches & 2)) return DAF_OK;
     CombineSeg ci, cq;
     fill_combine(&ci, si);
     fill_combine(&cq, sq);
@@ -1209,7 +1214,8 @@ namespace {
 constexpr size_t kStaticScratchBytes = (size_t)16 << 20;   // 16 MiB: status word + split-KV partials
 static __device__ __align__(256) unsigned char g_qd_static_scratch[kStaticScratchBytes];
 constexpr int kMaxDevices = 64;
-void* g_static_scratch_addr[kMaxDevices] = {nullptr};
+// one slot per device; concurrent first calls on a device resolve the same address and store the same value
+std::atomic<void*> g_static_scratch_addr[kMaxDevices];
 
 // In host code the array's name is only a handle for the runtime, not an address
 // a kernel can use, so the device address is looked up once per device.
@@ -1218,16 +1224,18 @@ int static_scratch_address(void** out) {
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) { daf::set_cuda_error(e); return DAF_ERR_CUDA; }
     if (dev < 0 || dev >= kMaxDevices) return DAF_ERR_UNSUPPORTED;
-    if (g_static_scratch_addr[dev] == nullptr) {
+    void* known = g_static_scratch_addr[dev].load(std::memory_order_acquire);
+    if (known == nullptr) {
         void* ptr = nullptr;
         e = cudaGetSymbolAddress(&ptr, g_qd_static_scratch);
         if (e != cudaSuccess || ptr == nullptr) {
             daf::set_cuda_error(e != cudaSuccess ? e : cudaErrorInvalidSymbol);
             return DAF_ERR_CUDA;
         }
-        g_static_scratch_addr[dev] = ptr;
+        g_static_scratch_addr[dev].store(ptr, std::memory_order_release);
+        known = ptr;
     }
-    *out = g_static_scratch_addr[dev];
+    *out = known;
     return DAF_OK;
 }
 }  // namespace
@@ -1258,4 +1266,22 @@ extern "C" int daf_qd_attn_static(const daf_params* p, const void* q_question, c
     return launch_attention(q_question, kv_k, kv_v, rp.L_q, rp.N, rp.Hq, rp.Hkv, rp.L_d, rp.scale, true, true, out,
                             out_row_stride_bytes, dst_rows, lse, reinterpret_cast<DeviceStatus*>(base),
                             reinterpret_cast<char*>(base) + kStatusBytes, kStaticScratchBytes - kStatusBytes, st);
+}
+
+// Status of the calls made through daf_qd_attn_static on the current device since the last poll: the
+// status word sits at the head of the fixed array, so it is read (and cleared) from there.  No allocation.
+extern "C" int daf_qd_attn_static_poll_status(void* stream) {
+    using namespace daf;
+    void* base = nullptr;
+    if (int rc = static_scratch_address(&base)) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    DeviceStatus hs;
+    cudaError_t e = cudaMemcpyAsync(&hs, base, sizeof(hs), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e == cudaSuccess && hs.code != 0) {
+        e = cudaMemsetAsync(base, 0, sizeof(hs), st);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    }
+    if (e != cudaSuccess) { set_cuda_error(e); return DAF_ERR_CUDA; }
+    return hs.code;
 }

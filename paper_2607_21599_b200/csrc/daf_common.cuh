@@ -67,7 +67,7 @@ int launch_attention_joint(const void* q_imp, const void* q_fresh, const int32_t
                            const void* kv_v,
                            int L_q, int L_d, void* out_question, long long out_row_stride_bytes, int Hq, int Hkv,
                            float scale, DeviceStatus* status, void* scratch, size_t scratch_bytes, cudaStream_t stream,
-                           bool after_kernel);
+                           bool after_kernel, int launches = 3);   // launches: bit 0 the attention launch, bit 1 the merge
 
 // ---------------------------------------------------------------- device side
 #ifdef __CUDACC__

@@ -6,6 +6,8 @@
 // kernels with no tensor-core work.
 #include <cooperative_groups.h>
 
+#include <atomic>
+
 #include "daf_common.cuh"
 
 namespace daf {
@@ -35,6 +37,14 @@ __device__ __forceinline__ uint32_t score_key(float s) {
     if ((b & 0x7FFFFFFFu) > 0x7F800000u) return 0u;   // NaN
     if (b == 0x80000000u) b = 0u;                     // -0 -> +0
     return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+
+// fp32 add, round to nearest, subnormals kept (the library is built with flush-to-zero arithmetic; the
+// aggregation of the signal rows must not flush, or tiny sums would all rank as ties at zero).
+__device__ __forceinline__ float add_rn_keep_subnormals(float a, float b) {
+    float d;
+    asm("add.rn.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
+    return d;
 }
 
 // Keys sit in shared memory with one word of padding per 32, so that both access patterns are free of bank
@@ -74,7 +84,7 @@ select_topk_kernel(const float* __restrict__ scores, int n_sig, int L_d, int k,
     for (int i = tid; i < n_loc; i += kSelThreads) {
         const int g = lo_cta + i;
         float acc = scores[g];
-        for (int l = 1; l < n_sig; ++l) acc = __fadd_rn(acc, scores[(size_t)l * L_d + g]);
+        for (int l = 1; l < n_sig; ++l) acc = add_rn_keep_subnormals(acc, scores[(size_t)l * L_d + g]);
         keys[at(i)] = score_key(acc);
     }
     if (tid < 256) { sh->hist[0][tid] = 0u; sh->hist[1][tid] = 0u; }
@@ -129,6 +139,7 @@ select_topk_kernel(const float* __restrict__ scores, int n_sig, int L_d, int k,
             }
             const uint32_t above = incl - sgrp;
             const uint32_t k_rem = sh->pick[1];
+            __syncwarp();   // every lane has read the rank before one of them replaces it
             if (k_rem > above && k_rem <= incl) {
                 uint32_t a = above;
                 for (int b = 7; b >= 0; --b) {
@@ -253,12 +264,14 @@ __device__ __forceinline__ void block_excl_scan2(uint32_t a, uint32_t b, uint32_
 // bins in descending order; the result goes to pick[0] (bin) and pick[1] (rank inside that bin).
 __device__ __forceinline__ void pick_bin(Sel1Shared* sh, int n_bins, int per) {
     const int top = n_bins - 1 - (int)threadIdx.x * per;   // this thread's highest bin
+    // the remaining rank is read here, ahead of the scan: the scan's barriers then separate every
+    // thread's read from the one thread that writes the reduced rank below
+    const uint32_t k_rem = sh->pick[1];
     uint32_t c = 0;
     if (top >= 0)
         for (int b = 0; b < per; ++b) c += sh->hist[top - b];
     uint32_t above, dummy, tot, tot2;
     block_excl_scan2(c, 0u, sh->warp_a, sh->warp_b, above, dummy, tot, tot2);
-    const uint32_t k_rem = sh->pick[1];
     if (top >= 0 && k_rem > above && k_rem <= above + c) {
         uint32_t acc = above;
         for (int b = 0; b < per; ++b) {
@@ -298,7 +311,7 @@ select_topk_cta_kernel(const float* __restrict__ scores, int n_sig, int L_d, int
                 nxt[u] = i < L_d ? scores[(size_t)l * L_d + i] : 0.f;
             }
 #pragma unroll
-            for (int u = 0; u < 8; ++u) acc[u] = __fadd_rn(acc[u], nxt[u]);
+            for (int u = 0; u < 8; ++u) acc[u] = add_rn_keep_subnormals(acc[u], nxt[u]);
         }
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
@@ -343,6 +356,7 @@ select_topk_cta_kernel(const float* __restrict__ scores, int n_sig, int L_d, int
         // few candidates (the usual case): each thread ranks one candidate by counting the larger and the
         // equal ones; the candidate whose rank interval holds the remaining rank is the threshold
         const uint32_t k_rem = sh->pick[1];
+        __syncthreads();   // every thread has read the rank before one of them replaces it
         if (tid < n_cand) {
             const uint32_t mine = cand[tid];
             uint32_t n_gt = 0, n_eq = 0;
@@ -538,17 +552,17 @@ int launch_select(const ResolvedParams& rp, const float* scores, int n_sig, cons
                   DeviceStatus* status, void* scratch, cudaStream_t stream) {
     const int32_t* idx_src = idx_in;
     if (scores != nullptr && rp.L_d > 0) {
-        static bool attr_done[64] = {false};
+        static std::atomic<bool> attr_done[64];   // per device; a concurrent first call sets the same values
         int dev = 0;
         cudaGetDevice(&dev);
-        if (dev >= 0 && dev < 64 && !attr_done[dev]) {
+        if (dev >= 0 && dev < 64 && !attr_done[dev].load(std::memory_order_acquire)) {
             cudaError_t e = cudaFuncSetAttribute(select_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                  (int)(sizeof(SelShared) + (size_t)padded(kSelSmemKeysPerCta) * sizeof(uint32_t)));
             if (e == cudaSuccess)
                 e = cudaFuncSetAttribute(select_topk_cta_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)(sizeof(Sel1Shared) + ((size_t)padded(kSel1MaxKeys) + kSel1MaxKeys) * sizeof(uint32_t)));
             if (e != cudaSuccess) { set_cuda_error(e); return DAF_ERR_CUDA; }
-            attr_done[dev] = true;
+            attr_done[dev].store(true, std::memory_order_release);
         }
         if (rp.L_d <= g_sel1_max_keys) {
             const size_t smem1 = sizeof(Sel1Shared) + ((size_t)padded(rp.L_d) + rp.L_d) * sizeof(uint32_t);   // keys and candidate list

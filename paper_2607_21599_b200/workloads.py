@@ -20,7 +20,7 @@ from __future__ import annotations
 
 import dataclasses
 import math
-from typing import Dict, Iterator, List, Optional, Tuple
+from typing import Callable, Dict, Iterator, List, Optional, Tuple
 
 import torch
 
@@ -113,6 +113,8 @@ class Workload:
     r: float
     selection: str
     n_sig: int = 1
+    k: int = -1     # number of important tokens; stated for the named configurations, otherwise supplied by
+                    # the caller through with_k() (the counting rule belongs to the library and to the oracle)
 
     @property
     def N(self) -> int:
@@ -126,46 +128,49 @@ class Workload:
     def softmax_scale(self) -> float:
         return 1.0 / math.sqrt(self.head_dim)
 
-    @property
-    def k(self) -> int:
-        """Number of important tokens, ceil(r * L_d) (input sizing only; the
-        library and the oracle each compute their own)."""
-        return max(0, min(self.L_d, int(math.ceil(self.r * self.L_d * (1.0 - 1e-6)))))
+    def with_k(self, num_important: Callable[[int, float], int]) -> "Workload":
+        """The same workload with k filled in by `num_important(L_d, r)` (the library's or the oracle's)."""
+        return self if self.k >= 0 else dataclasses.replace(self, k=int(num_important(self.L_d, self.r)))
 
 
 CONFIGS: Dict[str, Workload] = {
-    "c0": Workload("c0", 0, 28, 4, 128, 1, 1024, 256, 32, 0.15, "given"),
-    "c1": Workload("c1", 1, 28, 4, 128, 28, 6144, 512, 64, 0.15, "lognormal"),
-    "c2": Workload("c2", 2, 32, 8, 128, 32, 16384, 512, 128, 0.10, "lognormal"),
-    "c3": Workload("c3", 3, 28, 4, 128, 28, 32768, 512, 128, 0.20, "pareto_clustered"),
+    "c0": Workload("c0", 0, 28, 4, 128, 1, 1024, 256, 32, 0.15, "given", k=154),
+    "c1": Workload("c1", 1, 28, 4, 128, 28, 6144, 512, 64, 0.15, "lognormal", k=922),
+    "c2": Workload("c2", 2, 32, 8, 128, 32, 16384, 512, 128, 0.10, "lognormal", k=1639),
+    "c3": Workload("c3", 3, 28, 4, 128, 28, 32768, 512, 128, 0.20, "pareto_clustered", k=6554),
 }
 
 
 # Beyond the five stated configurations: the shape of the paper's longest evaluation point (a 136k-token
 # context with r = 0.3, Table 1), four layers of it.  Used by the benchmark and one sampled parity test.
 EXTRA_CONFIGS: Dict[str, Workload] = {
-    "x136k": Workload("x136k", 5, 28, 4, 128, 4, 139264, 512, 128, 0.30, "lognormal"),
+    "x136k": Workload("x136k", 5, 28, 4, 128, 4, 139264, 512, 128, 0.30, "lognormal", k=41780),
 }
 
 
-def sweep_points() -> List[Workload]:
-    """The single-layer sweep on the Qwen2.5-14B attention shape."""
+def sweep_points(num_important: Optional[Callable[[int, float], int]] = None) -> List[Workload]:
+    """The single-layer sweep on the Qwen2.5-14B attention shape.  k is filled in when the caller hands over
+    the counting function (the library's or the oracle's)."""
     pts = []
     for L_d in (2048, 8192, 16384, 32768):
         for r in (0.05, 0.10, 0.20, 0.30):
-            pts.append(Workload(f"c4_L{L_d}_r{r:.2f}", 4, 40, 8, 128, 1, L_d, 512, 128, r, "lognormal"))
+            w = Workload(f"c4_L{L_d}_r{r:.2f}", 4, 40, 8, 128, 1, L_d, 512, 128, r, "lognormal")
+            pts.append(w.with_k(num_important) if num_important is not None else w)
     return pts
 
 
 def tiny(name: str = "tiny", L_d: int = 48, doc_len: int = 16, L_q: int = 5, r: float = 0.25,
          n_q_heads: int = 4, n_kv_heads: int = 2, head_dim: int = 8, selection: str = "lognormal",
-         n_sig: int = 3, config_id: int = 99) -> Workload:
+         n_sig: int = 3, config_id: int = 99, num_important: Optional[Callable[[int, float], int]] = None) -> Workload:
     """A small shape for brute-force checks."""
-    return Workload(name, config_id, n_q_heads, n_kv_heads, head_dim, 1, L_d, doc_len, L_q, r, selection, n_sig)
+    w = Workload(name, config_id, n_q_heads, n_kv_heads, head_dim, 1, L_d, doc_len, L_q, r, selection, n_sig)
+    return w.with_k(num_important) if num_important is not None else w
 
 
 def given_indices(w: Workload, layer: int = 0) -> torch.Tensor:
     """k distinct positions: the first k entries of a seeded Fisher-Yates shuffle of 0..L_d-1, sorted."""
+    if w.k < 0:
+        raise ValueError("workload without a count of important tokens: use with_k()")
     seed = tensor_seed(w.config_id, layer, TENSOR_IDS["idx_perm"])
     perm = list(range(w.L_d))
     for i in range(w.L_d - 1, 0, -1):
@@ -230,6 +235,8 @@ def iter_layers(w: Workload, device="cpu") -> Iterator[Dict[str, Optional[torch.
 def attention_pairs(w: Workload) -> Dict[str, int]:
     """Visible (query, key) pairs of each stage; 4 * head_dim * n_q_heads flop per pair."""
     k, L_q, L_d, N = w.k, w.L_q, w.L_d, w.N
+    if k < 0:
+        raise ValueError("workload without a count of important tokens: use with_k()")
     return {
         "important": k * (k + 1) // 2,
         "question": L_q * L_d + L_q * (L_q + 1) // 2,

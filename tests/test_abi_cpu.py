@@ -100,6 +100,13 @@ def test_host_side_argument_validation(lib):
     # a layer without question rows cannot read Q in place (only the joint launch does)
     no_q = api.make_params(256, 0, 0.25, 4, 2)
     assert api.daf_layer(no_q, buf, 1, None, buf, buf, buf, buf, buf, buf, None, buf, buf, buf, None, ws) == api.DAF_ERR_INVALID_ARG
+    # nothing selected (r = 0) but question rows present: they are read from q_fresh, so it is required
+    r0 = api.make_params(256, 16, 0.0, 4, 2)
+    assert api.daf_layer(r0, None, 0, None, None, buf, buf, buf, buf, None, None, None, None, buf, None, ws) == api.DAF_ERR_INVALID_ARG
+    assert api.daf_layer(r0, None, 0, None, buf[8:], buf, buf, buf, buf, None, None, None, None, buf, None, ws) == api.DAF_ERR_ALIGNMENT
+    assert api.daf_layer(r0, None, 0, None, buf, buf, buf, None, buf, None, None, None, None, buf, None, ws) == api.DAF_ERR_INVALID_ARG
+    # important rows without packed K/V buffers
+    assert api.daf_layer(ok, buf, 1, None, buf, buf, buf, buf, buf, buf, buf, None, buf, buf, None, ws) == api.DAF_ERR_INVALID_ARG
     # the self-test of the bounded wait checks its arguments before it launches anything
     assert api.daf_selftest_bounded_wait(None, 50) == api.DAF_ERR_WORKSPACE
     assert api.daf_selftest_bounded_wait(ws[:64], 50) == api.DAF_ERR_WORKSPACE

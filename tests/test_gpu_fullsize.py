@@ -1,10 +1,11 @@
 """Parity at the full benchmark sizes, through the same entry point and launch mode the
-benchmark times (daf_layer replayed from a CUDA graph), on outputs the oracle can
-afford: selection, gather and hybrid cache are compared in full (bit-exact); the
-attention rows are compared on a sample of rows (first, last, tile edges, seeded
-random rows) against the oracle evaluated row by row; full recompute likewise."""
-import math
+benchmark times (daf_layer replayed from a CUDA graph).
 
+Selection, gather and hybrid cache are always compared in full (bit-exact).  The hidden
+rows are compared with the oracle in full where the oracle can afford it (every layer of
+the 6k configuration, three layers of the 16k one) and on a sample of rows elsewhere
+(first, last, every tile edge and its neighbours, seeded random rows; all question rows at
+32k); full recompute likewise on sampled rows."""
 import numpy as np
 import pytest
 import torch
@@ -22,9 +23,12 @@ def _f(t):
     return t.float().cpu().numpy()
 
 
-def _sample_rows(n, count, seed):
+def _sample_rows(n, count, seed, all_edges=False):
+    """Rows 0, 1, n-2, n-1, tile edges (every 128 rows) with both neighbours -- all of them, or about six
+    spread over the range -- and seeded random rows up to `count`."""
     edges = [0, 1, n - 1, n - 2]
-    for t in range(128, n, max(128, (n // 128 // 6) * 128)):
+    step = 128 if all_edges else max(128, (n // 128 // 6) * 128)
+    for t in range(128, n, step):
         edges += [t - 1, t, t + 1]
     rng = np.random.default_rng(seed)
     rows = set(int(r) for r in edges if 0 <= r < n)
@@ -46,18 +50,12 @@ def _workload(name):
         return W.CONFIGS[name]
     if name in W.EXTRA_CONFIGS:
         return W.EXTRA_CONFIGS[name]
-    return {w.name: w for w in W.sweep_points()}[name]
+    return {w.name: w for w in W.sweep_points(api.daf_num_important)}[name]
 
 
-@pytest.mark.parametrize("name,layer,n_imp_rows,n_q_rows,n_full_rows", [
-    ("c1", 3, 160, 64, 96),
-    ("c2", 17, 120, 48, 48),
-    ("c3", 27, 100, 32, 32),
-    ("c4_L32768_r0.30", 0, 64, 24, 0),
-    ("c4_L2048_r0.05", 0, 103, 128, 64),
-    ("x136k", 1, 24, 12, 0),
-])
-def test_layer_at_benchmark_size(name, layer, n_imp_rows, n_q_rows, n_full_rows):
+def _layer_parity(name, layer, rows_imp, rows_q, n_full_rows):
+    """Runs one layer the way the benchmark does and compares it with the oracle.  rows_imp / rows_q:
+    None = every row, an int = that many sampled rows, "edges:<n>" = every tile edge and n rows in all."""
     assert torch.cuda.is_available()
     build.build()
     w = _workload(name)
@@ -65,7 +63,7 @@ def test_layer_at_benchmark_size(name, layer, n_imp_rows, n_q_rows, n_full_rows)
     L = W.make_layer(w, layer, dev)
     p = api.make_params(w.L_d, w.L_q, w.r, w.n_q_heads, w.n_kv_heads)
     k = api.daf_num_important(w.L_d, w.r)
-    assert k == w.k == oracle.num_important(w.L_d, w.r)
+    assert k == oracle.num_important(w.L_d, w.r)
     N, Hq, Hkv = w.N, w.n_q_heads, w.n_kv_heads
     ws = api.alloc_workspace(p)
     bf = torch.bfloat16
@@ -100,7 +98,7 @@ def test_layer_at_benchmark_size(name, layer, n_imp_rows, n_q_rows, n_full_rows)
     idx = oracle.select(scores, k)
     assert np.array_equal(idx_out.cpu().numpy(), idx), "selected positions differ"
     idx_t = torch.from_numpy(idx).long().to(dev)
-    q_pack = L["q_fresh"][idx_t]          # what a packed copy would hold (the layer did not write one)
+    q_pack = L["q_fresh"][idx_t]          # what a packed copy would hold (the layer may not have written one)
     assert torch.equal(k_pack, L["k_fresh"][idx_t])
     assert torch.equal(v_pack, L["v_fresh"][idx_t])
     exp_k = torch.cat([L["k_cached"], L["k_fresh"][w.L_d:]], 0)
@@ -110,14 +108,23 @@ def test_layer_at_benchmark_size(name, layer, n_imp_rows, n_q_rows, n_full_rows)
     assert torch.equal(kv_k, exp_k) and torch.equal(kv_v, exp_v), "hybrid cache differs"
     assert torch.all(hidden[k + w.L_q] == -9.0), "row past the end was written"
 
-    # --- attention rows on a sample
+    # --- attention rows
+    def pick(spec, n, seed):
+        if spec is None:
+            return None
+        if isinstance(spec, str):
+            return _sample_rows(n, int(spec.split(":")[1]), seed, all_edges=True)
+        return _sample_rows(n, spec, seed)
+
     scale = w.softmax_scale
-    rows_imp = _sample_rows(k, n_imp_rows, 1)
-    ref_imp = oracle.important_attn(_f(q_pack), _f(k_pack), _f(v_pack), scale, rows=rows_imp)
-    _check(hidden[torch.from_numpy(rows_imp).long().to(dev)], ref_imp, f"{name}: important rows")
-    rows_q = _sample_rows(w.L_q, n_q_rows, 2)
-    ref_q = oracle.qd_attn(_f(L["q_fresh"][w.L_d:]), _f(kv_k), _f(kv_v), w.L_d, scale, rows=rows_q)
-    _check(hidden[(k + torch.from_numpy(rows_q).long()).to(dev)], ref_q, f"{name}: question rows")
+    ri = pick(rows_imp, k, 1)
+    ref_imp = oracle.important_attn(_f(q_pack), _f(k_pack), _f(v_pack), scale, rows=ri)
+    got_imp = hidden[:k] if ri is None else hidden[torch.from_numpy(ri).long().to(dev)]
+    _check(got_imp, ref_imp, f"{name} layer {layer}: important rows")
+    rq = pick(rows_q, w.L_q, 2)
+    ref_q = oracle.qd_attn(_f(L["q_fresh"][w.L_d:]), _f(kv_k), _f(kv_v), w.L_d, scale, rows=rq)
+    got_q = hidden[k: k + w.L_q] if rq is None else hidden[(k + torch.from_numpy(rq).long()).to(dev)]
+    _check(got_q, ref_q, f"{name} layer {layer}: question rows")
 
     # --- full recompute at the same size, sampled rows
     if n_full_rows:
@@ -132,3 +139,29 @@ def test_layer_at_benchmark_size(name, layer, n_imp_rows, n_q_rows, n_full_rows)
         _check(out[torch.from_numpy(rows_f).long().to(dev)], ref_f, f"{name}: full recompute rows")
         # property that holds at any size: the first row equals its value row
         assert torch.equal(out[0], L["v_fresh"][0].repeat_interleave(Hq // Hkv, dim=0))
+
+
+@pytest.mark.parametrize("layer", range(W.CONFIGS["c1"].layers))
+def test_c1_every_layer_every_row(layer):
+    _layer_parity("c1", layer, None, None, 96 if layer == 3 else 0)
+
+
+@pytest.mark.parametrize("layer", [0, 16, 31])
+def test_c2_three_layers_every_row(layer):
+    _layer_parity("c2", layer, None, None, 48 if layer == 16 else 0)
+
+
+@pytest.mark.parametrize("layer", [0, 14, 27])
+def test_c3_three_layers_all_tile_edges_all_question_rows(layer):
+    _layer_parity("c3", layer, "edges:544", None, 32 if layer == 27 else 0)
+
+
+@pytest.mark.parametrize("name", [w.name for w in W.sweep_points()])
+def test_c4_every_sweep_point(name):
+    w = _workload(name)
+    big = w.N > 8320
+    _layer_parity(name, 0, 96 if big else None, 32 if big else None, 0 if big else 64)
+
+
+def test_x136k_sampled_rows():
+    _layer_parity("x136k", 1, 24, 12, 0)

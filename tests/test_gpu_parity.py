@@ -64,6 +64,8 @@ def _normal(shape, seed, scale=1.0):
     # only in their last byte (every radix pass is needed) and one whose keys differ only in the first two
     (8192, 0.15, 1, "lognormal"), (8193, 0.15, 1, "lognormal"), (20000, 0.2, 1, "lowbyte"), (24000, 0.1, 1, "highbytes"),
     (30000, 1.0, 1, "lognormal"), (30000, 0.0, 1, "lognormal"),
+    # sums of two signal rows that are subnormal in fp32: the aggregation must keep them apart, not flush them to 0
+    (3000, 0.2, 2, "denormal"), (12000, 0.1, 3, "denormal"),
 ])
 def test_select_indices_bit_exact(L_d, r, n_sig, kind):
     if kind == "pareto":
@@ -82,6 +84,9 @@ def test_select_indices_bit_exact(L_d, r, n_sig, kind):
             S = (1.0 + torch.floor(S * 37).remainder(256) * 2.0 ** -23).float()
         if kind == "highbytes":   # powers of two times {1, 1.5}: the low two bytes of every key are zero
             S = torch.pow(2.0, torch.floor(S * 3).remainder(40) - 20) * (1.0 + 0.5 * (torch.floor(S * 11).remainder(2)))
+        if kind == "denormal":    # distinct multiples of the smallest subnormal, a few normal values among them
+            S = (torch.floor(S * 1000).remainder(4000) * 2.0 ** -149).float()
+            S[0, ::97] = 1.0e-37
         if kind == "special":
             S[0, 3] = float("nan"); S[0, 4] = float("inf"); S[0, 5] = -float("inf")
             S[0, 6] = 0.0; S[0, 7] = -0.0; S[0, 8] = float("nan"); S[0, 9:40] = -S[0, 9:40]
@@ -225,6 +230,41 @@ def test_important_attention_scatters_rows_through_dst_rows():
     _assert_close(out[dst.long().cuda()], ref, "scattered rows")
     others = np.setdiff1d(np.arange(400), dst.numpy())
     assert torch.all(out[torch.from_numpy(others).cuda()] == 5.0)
+
+
+@pytest.mark.parametrize("L_d,L_q,r,Hq,Hkv,mode", [(1024, 32, 0.15, 28, 4, 0), (1024, 32, 0.15, 28, 4, 1), (3000, 130, 0.3, 8, 2, 1),
+                                                  (700, 9, 0.5, 5, 5, 0)])
+def test_fused_epilogue_rows_equal_unfused_rows_plus_daf_fuse_bit_for_bit(L_d, L_q, r, Hq, Hkv, mode):
+    """State fusion done by the attention epilogues (out / dst_rows of the two stand-alone attention calls)
+    gives exactly the bytes of the same two calls writing their own buffers followed by daf_fuse."""
+    dev = "cuda"
+    N = L_d + L_q
+    p = api.make_params(L_d, L_q, r, Hq, Hkv, fuse_mode=mode)
+    k = api.daf_num_important(L_d, r)
+    ws = api.alloc_workspace(p)
+    qp, kp, vp = (_normal((k, h, 128), 70 + i).to(dev) for i, h in enumerate((Hq, Hkv, Hkv)))
+    qq, kk, vv = _normal((L_q, Hq, 128), 80).to(dev), _normal((N, Hkv, 128), 81).to(dev), _normal((N, Hkv, 128), 82).to(dev)
+    idx = torch.randperm(L_d, generator=torch.Generator().manual_seed(3))[:k].sort().values.to(torch.int32).to(dev)
+    row = Hq * 256
+    # unfused: each stage into its own buffer, then the stand-alone fusion
+    o_imp = torch.zeros(k, Hq, 128, dtype=torch.bfloat16, device=dev)
+    o_q = torch.zeros(L_q, Hq, 128, dtype=torch.bfloat16, device=dev)
+    _ok(api.daf_important_attn(p, k, qp, kp, vp, o_imp, row, None, None, ws), ws, "imp")
+    _ok(api.daf_qd_attn(p, qq, kk, vv, o_q, row, None, None, ws), ws, "qd")
+    rows_total = N if mode == 1 else k + L_q
+    unfused = torch.full((rows_total, Hq, 128), 3.0, dtype=torch.bfloat16, device=dev)
+    api.check(api.daf_fuse(p, k, idx, o_imp, o_q, unfused, None), "daf_fuse")
+    # fused: the same two calls write the final rows themselves
+    fused = torch.full((rows_total, Hq, 128), 3.0, dtype=torch.bfloat16, device=dev)
+    if mode == 0:
+        _ok(api.daf_important_attn(p, k, qp, kp, vp, fused, row, None, None, ws), ws, "imp fused")
+        _ok(api.daf_qd_attn(p, qq, kk, vv, fused, row, None, None, ws, out_offset_bytes=k * row), ws, "qd fused")
+    else:
+        dst_q = torch.arange(L_d, N, dtype=torch.int32, device=dev)
+        _ok(api.daf_important_attn(p, k, qp, kp, vp, fused, row, idx, None, ws), ws, "imp fused")
+        _ok(api.daf_qd_attn(p, qq, kk, vv, fused, row, dst_q, None, ws), ws, "qd fused")
+    torch.cuda.synchronize()
+    assert torch.equal(fused.view(torch.int16), unfused.view(torch.int16))
 
 
 @pytest.mark.parametrize("L_d,L_q,Hq,Hkv,qscale", [(1024, 32, 28, 4, 1.0), (1000, 1, 4, 4, 1.0), (333, 17, 8, 2, 1.0),

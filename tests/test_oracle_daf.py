@@ -38,7 +38,7 @@ def _brute_force(q, kh, vh, idx, L_d, scale):
 @pytest.mark.parametrize("seed_layer,L_d,L_q,r,Hq,Hkv", [(0, 48, 5, 0.25, 4, 2), (1, 64, 1, 0.1, 6, 2),
                                                          (2, 32, 9, 0.5, 7, 1), (3, 40, 4, 1.0, 2, 2)])
 def test_layer_equals_brute_force_masked_attention(seed_layer, L_d, L_q, r, Hq, Hkv):
-    w = W.tiny(L_d=L_d, doc_len=8, L_q=L_q, r=r, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=8, n_sig=3)
+    w = W.tiny(L_d=L_d, doc_len=8, L_q=L_q, r=r, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=8, n_sig=3, num_important=oracle.num_important)
     L = W.make_layer(w, seed_layer)
     q, kf, vf, kc, vc = (_np(L[n]) for n in ("q_fresh", "k_fresh", "v_fresh", "k_cached", "v_cached"))
     res = oracle.daf_layer(q, kf, vf, kc, vc, L_d, L_q, w.softmax_scale, scores=L["scores"].numpy(), r=r)
@@ -63,7 +63,7 @@ def test_layer_equals_brute_force_masked_attention(seed_layer, L_d, L_q, r, Hq, 
 
 
 def test_r_one_without_question_is_full_causal_attention():
-    w = W.tiny(L_d=40, doc_len=8, L_q=0, r=1.0, n_q_heads=4, n_kv_heads=2, head_dim=8)
+    w = W.tiny(L_d=40, doc_len=8, L_q=0, r=1.0, n_q_heads=4, n_kv_heads=2, head_dim=8, num_important=oracle.num_important)
     L = W.make_layer(w, 0)
     q, kf, vf, kc, vc = (_np(L[n]) for n in ("q_fresh", "k_fresh", "v_fresh", "k_cached", "v_cached"))
     res = oracle.daf_layer(q, kf, vf, kc, vc, 40, 0, w.softmax_scale, scores=L["scores"].numpy(), r=1.0)
@@ -79,7 +79,7 @@ def test_r_one_without_question_is_full_causal_attention():
 
 
 def test_question_stage_equals_full_recompute_when_cache_is_fresh():
-    w = W.tiny(L_d=48, doc_len=16, L_q=6, r=0.25)
+    w = W.tiny(L_d=48, doc_len=16, L_q=6, r=0.25, num_important=oracle.num_important)
     L = W.make_layer(w, 4)
     q, kf, vf = (_np(L[n]) for n in ("q_fresh", "k_fresh", "v_fresh"))
     res = oracle.daf_layer(q, kf, vf, kf[:48], vf[:48], 48, 6, w.softmax_scale, scores=L["scores"].numpy(), r=0.25)
@@ -88,7 +88,7 @@ def test_question_stage_equals_full_recompute_when_cache_is_fresh():
 
 
 def test_hybrid_cache_reading_important_rows_are_overwritten():
-    w = W.tiny(L_d=48, doc_len=16, L_q=4, r=0.25)
+    w = W.tiny(L_d=48, doc_len=16, L_q=4, r=0.25, num_important=oracle.num_important)
     L = W.make_layer(w, 5)
     q, kf, vf, kc, vc = (_np(L[n]) for n in ("q_fresh", "k_fresh", "v_fresh", "k_cached", "v_cached"))
     sc = L["scores"].numpy()
@@ -134,7 +134,7 @@ def test_full_context_variant_against_masked_library_attention():
     """Rows at positions row_pos attend every key up to their position (selective recomputation over the
     full context): pinned by a library attention with an explicit mask, by the identity position map
     (plain causal attention) and by the question rows of the DAF layer."""
-    w = W.tiny(L_d=40, doc_len=8, L_q=4, r=0.25, n_q_heads=6, n_kv_heads=2, head_dim=8)
+    w = W.tiny(L_d=40, doc_len=8, L_q=4, r=0.25, n_q_heads=6, n_kv_heads=2, head_dim=8, num_important=oracle.num_important)
     L = W.make_layer(w, 7)
     q, kf, vf, kc, vc = (_np(L[n]) for n in ("q_fresh", "k_fresh", "v_fresh", "k_cached", "v_cached"))
     base = oracle.daf_layer(q, kf, vf, kc, vc, 40, 4, w.softmax_scale, scores=L["scores"].numpy(), r=0.25)

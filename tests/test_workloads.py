@@ -31,7 +31,7 @@ def test_generator_is_deterministic_and_counter_based():
 
 
 def test_layers_and_tensors_are_independent():
-    w = W.tiny()
+    w = W.tiny(num_important=oracle.num_important)
     a, b = W.make_layer(w, 0), W.make_layer(w, 1)
     assert not torch.equal(a["q_fresh"], b["q_fresh"])
     assert not torch.equal(a["k_fresh"][: w.L_d], a["k_cached"])
@@ -42,10 +42,15 @@ def test_layers_and_tensors_are_independent():
 def test_workload_sizes_match_the_stated_configurations():
     c = W.CONFIGS
     assert (c["c0"].k, c["c1"].k, c["c2"].k, c["c3"].k) == (154, 922, 1639, 6554)
+    # the stated counts are what the oracle's and the library's counting rules give
+    from paper_2607_21599_b200 import api, build
+    build.build()
+    for w in list(c.values()) + list(W.EXTRA_CONFIGS.values()):
+        assert w.k == oracle.num_important(w.L_d, w.r) == api.daf_num_important(w.L_d, w.r), w.name
     assert c["c0"].n_docs == 4 and c["c1"].n_docs == 12 and c["c2"].n_docs == 32 and c["c3"].n_docs == 64
     idx = W.given_indices(c["c0"])
     assert len(idx) == 154 and torch.all(idx[1:] > idx[:-1]) and 0 <= int(idx[0]) and int(idx[-1]) < 1024
-    pts = W.sweep_points()
+    pts = W.sweep_points(oracle.num_important)
     assert len(pts) == 16 and {p.L_d for p in pts} == {2048, 8192, 16384, 32768}
     assert {p.name: p.k for p in pts}["c4_L32768_r0.30"] == 9831
 
@@ -73,7 +78,7 @@ def _rank_main(rank, world, port, root):
     import bench
     dist.init_process_group("gloo", rank=rank, world_size=world)
     try:
-        w = W.tiny(L_d=32, doc_len=8, L_q=3)
+        w = W.tiny(L_d=32, doc_len=8, L_q=3, num_important=oracle.num_important)
         layers = bench.replica_layers(rank, w)
         mine = W.make_layer(w, layers[0])["q_fresh"].float().sum().reshape(1).double()
         sums = [torch.zeros(1, dtype=torch.float64) for _ in range(world)]

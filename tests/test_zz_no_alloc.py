@@ -21,7 +21,7 @@ pytestmark = pytest.mark.gpu
 MAX_ABS, MEAN_ABS = 2e-2, 2e-3
 
 
-def _run_both(L_d, L_q, Hq, Hkv, seed):
+def _run_both(L_d, L_q, Hq, Hkv, seed, warm=True):
     N = L_d + L_q
     dev = "cuda"
     q = W.normal_bf16((L_q, Hq, 128), seed).to(dev)
@@ -34,11 +34,19 @@ def _run_both(L_d, L_q, Hq, Hkv, seed):
     api.check(api.daf_qd_attn(p, q, k, v, ref, Hq * 256, None, ref_lse, ws), "daf_qd_attn")
     got = torch.full((L_q + 1, Hq, 128), 5.0, dtype=torch.bfloat16, device=dev)
     got_lse = torch.zeros(Hq, L_q, dtype=torch.float32, device=dev)
+    if warm:
+        # lazy loading of the library's device image happens at the first launch; it is not the call's doing
+        api.check(api.daf_qd_attn_static(p, q, k, v, got, Hq * 256, None, got_lse), "daf_qd_attn_static (warm-up)")
+        torch.cuda.synchronize()
     before = torch.cuda.memory_allocated()
+    free_before, _ = torch.cuda.mem_get_info()
     api.check(api.daf_qd_attn_static(p, q, k, v, got, Hq * 256, None, got_lse), "daf_qd_attn_static")
     assert torch.cuda.memory_allocated() == before, "the call went through torch's allocator"
     torch.cuda.synchronize()
-    api.check(api.daf_poll_status(ws), "device status")
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after >= free_before, "the call took device memory from the driver"
+    api.check(api.daf_poll_status(ws), "device status (workspace call)")
+    api.check(api.daf_qd_attn_static_poll_status(), "device status (static call)")
     return ref, ref_lse, got, got_lse, L_q
 
 
