@@ -81,18 +81,6 @@ __device__ long long g_laps[8 * 65536];
 extern "C" int daf_dbg_read_laps(void* host, size_t bytes) {
     return (int)cudaMemcpyFromSymbol(host, g_laps, bytes < sizeof(g_laps) ? bytes : sizeof(g_laps));
 }
-__device__ long long g_laps_mma[8 * 65536];
-extern "C" int daf_dbg_read_laps_mma(void* host, size_t bytes) {
-    return (int)cudaMemcpyFromSymbol(host, g_laps_mma, bytes < sizeof(g_laps_mma) ? bytes : sizeof(g_laps_mma));
-}
-__device__ long long g_ev[4][128][8];
-__device__ int g_ev_cta = 1000;
-extern "C" int daf_dbg_read_ev(void* host, size_t bytes) {
-    return (int)cudaMemcpyFromSymbol(host, g_ev, bytes < sizeof(g_ev) ? bytes : sizeof(g_ev));
-}
-#define DAF_EV(t, slot) do { const int d_ = (int)blockIdx.x - g_ev_cta; if (d_ >= 0 && d_ < 4 && (t) < 128 && (threadIdx.x & 31) == 0) g_ev[d_][(t)][(slot)] = clock64(); } while (0)
-#define DAF_MLAP_DECL long long ml_v = 0, ml_p = 0, ml_k = 0, ml_i = 0, ml_t = clock64(); const long long ml_begin = ml_t
-#define DAF_MLAP(acc) do { const long long now_ = clock64(); acc += now_ - ml_t; ml_t = now_; } while (0)
 #define DAF_LAP_DECL long long lap_s = 0, lap_soft = 0, lap_pv = 0, lap_t = clock64(); const long long lap_begin = lap_t
 #define DAF_LAP(acc) do { const long long now_ = clock64(); acc += now_ - lap_t; lap_t = now_; } while (0)
 #define DAF_STAMP(slot)                                                                         \
@@ -104,9 +92,6 @@ extern "C" int daf_dbg_read_ev(void* host, size_t bytes) {
 #define DAF_STAMP(slot) do {} while (0)
 #define DAF_LAP_DECL do {} while (0)
 #define DAF_LAP(acc) do {} while (0)
-#define DAF_MLAP_DECL do {} while (0)
-#define DAF_MLAP(acc) do {} while (0)
-#define DAF_EV(t, slot) do {} while (0)
 #endif
 
 // One online-softmax step of one query row (one thread) over NCH * 32 keys starting at `key0` (the kernel
@@ -196,28 +181,24 @@ __device__ __forceinline__ void rescale_o(uint32_t o_addr, float alpha) {
 #define DAF_SEG(field) (seg_id ? args.seg[1].field : args.seg[0].field)
 
 // What one CTA works on: the problem's geometry and the CTA's item (one token block of one head
-// block, and a range of key tiles).  In the pair form of the kernel an item is two consecutive token
-// blocks of one head block with the same key range, one per CTA of the pair ("unit" below is then a
-// pair of token blocks when items are counted, and `unit` the CTA's own token block).
+// block, and a range of key tiles).
 struct CtaWork {
     int n_q, n_kv, G, Gp, Tt, n_tb, causal_off;
     const int32_t* q_pos;
     float scale_log2;
-    int seg_id, hb, unit, unit_last, j_begin, j_end, item_splits, tok_base;
+    int seg_id, hb, unit, j_begin, j_end, item_splits, tok_base;
     long long part_row0;      // the item's first row in the partial-result arrays, in tokens
 };
 
-template <bool kPair>
-__device__ __forceinline__ void decode_work(const AttnArgs& args, CtaWork& a, int rank) {
-    // ---- which item is this CTA's (uniform across the CTA, and across the pair)
-    int seg_id = 0, item = kPair ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+__device__ __forceinline__ void decode_work(const AttnArgs& args, CtaWork& a) {
+    // ---- which item is this CTA's (uniform across the CTA)
+    int seg_id = 0, item = (int)blockIdx.x;
     if (args.joint) {
         if (item < args.seg[1].n_items) seg_id = 1;
         else item -= args.seg[1].n_items;
     }
     a.n_q = DAF_SEG(n_q); a.n_kv = DAF_SEG(n_kv); a.G = DAF_SEG(G); a.Gp = DAF_SEG(Gp); a.Tt = DAF_SEG(Tt);
     a.n_tb = DAF_SEG(n_tb); a.causal_off = DAF_SEG(causal_off); a.q_pos = DAF_SEG(q_pos); a.scale_log2 = DAF_SEG(scale_log2);
-    constexpr int kUnitBlocks = kPair ? 2 : 1;            // token blocks per unit of the work list
 
     int hb, unit, j_begin, j_end, item_splits, tok_base;
     long long part_row0;      // this item's first row in the partial-result arrays, in tokens
@@ -251,16 +232,14 @@ __device__ __forceinline__ void decode_work(const AttnArgs& args, CtaWork& a, in
         const int rem = slot - chunk * g * (g + 1) / 2;
         unit = g * chunk + rem / (g + 1);
         const int range = rem % (g + 1);
-        const int n_tiles = min(kUnitBlocks * (unit + 1), a.n_tb);
+        const int n_tiles = min(unit + 1, a.n_tb);
         j_begin = range * n_tiles / (g + 1);
         j_end = (range + 1) * n_tiles / (g + 1);
         item_splits = g + 1;
-        part_row0 = (long long)slot * (kUnitBlocks * kBlockM);
-        tok_base = unit * (kUnitBlocks * kBlockM);
+        part_row0 = (long long)slot * kBlockM;
+        tok_base = unit * kBlockM;
     }
-    a.seg_id = seg_id; a.hb = hb; a.j_begin = j_begin; a.j_end = j_end;
-    a.unit = kPair ? 2 * unit + rank : unit;                          // this CTA's token block
-    a.unit_last = kPair ? min(2 * unit + 1, a.n_tb - 1) : unit;       // the token block that sees the most keys
+    a.seg_id = seg_id; a.hb = hb; a.unit = unit; a.j_begin = j_begin; a.j_end = j_end;
     a.item_splits = item_splits; a.tok_base = tok_base; a.part_row0 = part_row0;
 }
 
@@ -322,7 +301,7 @@ __device__ __forceinline__ void write_rows(const AttnArgs& args, const CtaWork& 
             if (lane == 0) mbar_arrive(rows_parked);
             if (quad == 0) {
                 // the first softmax warp waits (bounded) until all four have parked their rows; one lane stores
-                bool all = mbar_wait<false>(rows_parked, 0, abort_flag, args.status, 70);
+                bool all = mbar_wait(rows_parked, 0, abort_flag, args.status, 70);
                 all = __all_sync(0xFFFFFFFFu, all);
                 if (all && lane == 0) {
                     tma_store_3d(tmap_o, q_tile, 0, h0, t0);
@@ -428,52 +407,39 @@ extern "C" int daf_dbg_read_trace(void* host, size_t bytes) {
 // The keys go through in sub-steps of 64 and S is double-buffered (two 64-column halves of the
 // same 128 tensor-memory columns): the logits of sub-step t + 1 are computed while the softmax of
 // sub-step t runs, so the softmax warps find their next input ready.  The products O += P_t V_t are
-// issued as each P_t arrives; a row may only be rescaled, and P_{t+1} only be handed over, once the
-// product before it has completed (pv_done).  The second CTA of the SM fills what gaps remain.
-//
-// Pair form (kPair).  What bounds the key loop is shared-memory bandwidth: every 64-key sub-step
-// re-reads the 32 KB Q tile as the A operand of S = Q K^T next to 32 KB of K/V.  In the pair form two
-// CTAs on the two SMs of a TPC (a cluster of two) run two query tiles against the same keys as ONE
-// M = 256 MMA (cta_group::2): each CTA holds its own Q rows, its own S, P and O in its own tensor
-// memory, but only HALF of every K sub-tile (32 of the 64 keys) and half of every V sub-tile (64 of
-// the 128 columns); the tensor cores exchange the halves.  Per sub-step a CTA then moves 64 KB
-// through its shared memory instead of 96 KB.  The leader CTA (rank 0) issues every MMA; completion is
-// signalled to the barriers of both CTAs (multicast commit); both CTAs' loads count on the leader's
-// barriers; the peer's softmax warps hand P over by arriving on the leader's barrier.
+// issued as each P_t arrives, in order; only a row that has to be rescaled waits for the product before
+// it to complete (pv_done).  The second CTA of the SM fills what gaps remain.  Final rows in token order
+// leave by tiled bulk stores from the dead Q tile.
+// Two tiles per CTA sharing every K/V tile (half the shared-memory fill traffic, one CTA per SM)
+// measured slower at every size from 1k to 136k tokens and was removed.
 constexpr int kSubN = 64;                               // keys per sub-step
 constexpr int kSubBytes = kSubN * kD * 2;               // 16 KB: K or V of one sub-step, two 64-column halves
 constexpr int kSubHalfBytes = kSubBytes / 2;
 constexpr int kAttnThreads = 192;                      // warps 0-3 softmax, warp 4 TMA, warp 5 MMA
 constexpr int kAttnTmemCols = 256;                     // S (two halves of 64) and O (128)
-constexpr int kMaxKvStages = 4;
 
 struct AttnSmem {
     uint64_t q_full;
-    uint64_t k_full[kMaxKvStages], k_empty[kMaxKvStages], v_full[kMaxKvStages], v_empty[kMaxKvStages];
+    uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2];
     uint64_t s_full[2], p_full[2];
-    uint64_t pv_done;
+    uint64_t pv_done[2];      // O += P_t V_t has completed: sub-steps alternate between the two barriers
     uint64_t rows_parked;     // epilogue: the four softmax warps have parked their rows for the tiled store
     uint32_t tmem_base;
     int abort_flag;
 };
 constexpr size_t kAttnSmemBytes = 1024 + 3 * (size_t)kTileBytes + sizeof(AttnSmem);
 
-template <bool kPair>
 __global__ void __launch_bounds__(kAttnThreads, 2)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_constant__ CUtensorMap tmap_k0,
                   const __grid_constant__ CUtensorMap tmap_v0, const __grid_constant__ CUtensorMap tmap_q1,
                   const __grid_constant__ CUtensorMap tmap_k1, const __grid_constant__ CUtensorMap tmap_v1,
                   const __grid_constant__ CUtensorMap tmap_o0, const __grid_constant__ CUtensorMap tmap_o1,
                   const AttnArgs args) {
-    // ring of K (and of V) sub-steps: single form two slots of 16 KB, pair form four slots of 8 KB (this CTA's half)
-    constexpr int kKvStages = kPair ? 4 : 2;
-    constexpr int kSlotBytes = kPair ? kSubBytes / 2 : kSubBytes;
-    constexpr int kKHalfBytes = kSlotBytes / 2;           // K slot: two 64-column halves of (32 or 64) 128-byte rows
     extern __shared__ unsigned char attn_smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(attn_smem_raw) + 1023) & ~(uintptr_t)1023);
     unsigned char* q_smem = smem;                                 // 32 KB
-    unsigned char* k_smem = smem + kTileBytes;                    // the K ring
-    unsigned char* v_smem = smem + 2 * (size_t)kTileBytes;        // the V ring
+    unsigned char* k_smem = smem + kTileBytes;                    // two sub-step slots
+    unsigned char* v_smem = smem + 2 * (size_t)kTileBytes;        // two sub-step slots
     AttnSmem* sm = reinterpret_cast<AttnSmem*>(smem + 3 * (size_t)kTileBytes);
 
     pdl_launch_dependents();   // a dependent kernel (the split merge) may start launching; it waits for this grid
@@ -481,9 +447,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
     if (threadIdx.x == 0) DAF_STAMP(0);
     DAF_KT_BEGIN(0);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int rank = kPair ? (int)cluster_cta_rank() : 0;       // 0: the CTA that issues the pair's MMAs
     CtaWork a;
-    decode_work<kPair>(args, a, rank);
+    decode_work(args, a);
     const int seg_id = a.seg_id;
     const CUtensorMap* tmap_q = seg_id ? &tmap_q1 : &tmap_q0;
     const CUtensorMap* tmap_k = seg_id ? &tmap_k1 : &tmap_k0;
@@ -496,42 +461,34 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
 
     // Loads K (kv = 0) or V (kv = 1) of sub-step t into its ring slot (the slot must be free).
     auto issue_kv = [&](int t, int kv) {
-        const int slot = t % kKvStages;
+        const int slot = t & 1;
         uint64_t* full = kv == 0 ? &sm->k_full[slot] : &sm->v_full[slot];
-        unsigned char* dst = (kv == 0 ? k_smem : v_smem) + (size_t)slot * kSlotBytes;
+        unsigned char* dst = (kv == 0 ? k_smem : v_smem) + (size_t)slot * kSubBytes;
         const CUtensorMap* tm = kv == 0 ? tmap_k : tmap_v;
         const int key0 = key_begin + t * kSubN;
-        if constexpr (!kPair) {
-            mbar_arrive_expect_tx(full, (uint32_t)kSubBytes);
-            tma_load_3d(dst, tm, full, 0, g_kv, key0);
-            tma_load_3d(dst + kSubHalfBytes, tm, full, 64, g_kv, key0);
-        } else {
-            // the leader's barrier counts the bytes of both CTAs' halves
-            if (rank == 0) mbar_arrive_expect_tx(full, (uint32_t)kSubBytes);
-            const uint32_t bar = map_to_cta(smem_u32(full), 0);
-            if (kv == 0) {   // K: this CTA's 32 of the 64 keys, all 128 columns
-                tma_load_3d_pair(dst, tm, bar, 0, g_kv, key0 + 32 * rank);
-                tma_load_3d_pair(dst + kKHalfBytes, tm, bar, 64, g_kv, key0 + 32 * rank);
-            } else {         // V: all 64 keys, this CTA's 64 of the 128 columns
-                tma_load_3d_pair(dst, tm, bar, 64 * rank, g_kv, key0);
-            }
-        }
+        mbar_arrive_expect_tx(full, (uint32_t)kSubBytes);
+        tma_load_3d(dst, tm, full, 0, g_kv, key0);
+        tma_load_3d(dst + kSubHalfBytes, tm, full, 64, g_kv, key0);
     };
-    // Set-up.  The producer thread prepares the barriers; the loads that need no free slot (Q and the
-    // first sub-steps) are issued ahead of the set-up barrier, so that their latency overlaps the rest of
-    // the set-up: the status check (a global read) and the tensor-memory allocation.
-    // Everything up to the dependency wait below touches no memory an earlier kernel writes, so with programmatic
+    // Set-up.  The producer thread prepares the barriers and at once starts the loads that need no free
+    // slot (Q and the first two sub-steps), so that their latency overlaps the rest of the set-up: the
+    // status check (a global read) and the tensor-memory allocation.
+    // Everything up to the wait below touches no memory an earlier kernel writes, so with programmatic
     // dependent launch it runs while the kernel launched just before (gather / hybrid-cache update) drains.
     __shared__ int skip_cta;
     const int32_t* const q_idx = DAF_SEG(q_idx);     // non-null: the softmax warps fetch the Q rows themselves
+    if (warp == 5) {
+        tmem_alloc(&sm->tmem_base, kAttnTmemCols);
+        tmem_relinquish();
+    }
     if (warp == 4 && lane == 0) {
-        mbar_init(&sm->q_full, q_idx != nullptr ? (kPair ? 8 : 4) : 1);
-        for (int s = 0; s < kKvStages; ++s) {
+        mbar_init(&sm->q_full, q_idx != nullptr ? 4 : 1);
+        for (int s = 0; s < 2; ++s) {
             mbar_init(&sm->k_full[s], 1); mbar_init(&sm->k_empty[s], 1);
             mbar_init(&sm->v_full[s], 1); mbar_init(&sm->v_empty[s], 1);
+            mbar_init(&sm->s_full[s], 1); mbar_init(&sm->p_full[s], 4);
         }
-        for (int s = 0; s < 2; ++s) { mbar_init(&sm->s_full[s], 1); mbar_init(&sm->p_full[s], kPair ? 8 : 4); }
-        mbar_init(&sm->pv_done, 1);
+        mbar_init(&sm->pv_done[0], 1); mbar_init(&sm->pv_done[1], 1);
         mbar_init(&sm->rows_parked, 4);
         sm->abort_flag = 0;
         mbar_fence_init();
@@ -539,43 +496,24 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
         tma_prefetch_desc(tmap_v);
         if (q_idx == nullptr) tma_prefetch_desc(tmap_q);
     }
-    if constexpr (kPair) {
-        // first half of a pair-wide barrier: once it completes (waited for below), the barriers of both
-        // CTAs are initialised and may be signalled from the other CTA
-        __syncwarp();
-        cluster_arrive();
-    }
-    if (warp == 5) {
-        if constexpr (kPair) { tmem_alloc_pair(&sm->tmem_base, kAttnTmemCols); tmem_relinquish_pair(); }
-        else { tmem_alloc(&sm->tmem_base, kAttnTmemCols); tmem_relinquish(); }
-    }
     pdl_wait();                // from here on: inputs that the kernel launched just before may have written
-    // sub-steps of this item: the keys of its range that the last token of the item's last token block may see
+    // sub-steps of this item: the keys of its range that the tile's last token may see
     int n_t = 0;
-    if (a.unit_last < a.n_tb) {
-        const int max_tok = min(a.n_q, (a.unit_last + 1) * a.Tt) - 1;
+    if (a.unit < a.n_tb) {
+        const int max_tok = min(a.n_q, t0 + a.Tt) - 1;
         const long long last_key = a.q_pos ? (long long)__ldg(a.q_pos + max_tok) : (long long)max_tok + a.causal_off;
         long long hi = min((long long)a.n_kv, last_key + 1);
         hi = min(hi, (long long)a.j_end * kBlockN);
         if (hi > key_begin) n_t = (int)((hi - key_begin + kSubN - 1) / kSubN);
     }
-    if constexpr (kPair) cluster_wait();
     if (warp == 4 && lane == 0) {
         if (n_t > 0) {
             if (q_idx == nullptr) {
-                const uint32_t q_bytes = 2u * 128u * (uint32_t)(a.Gp * a.Tt);
-                if constexpr (!kPair) {
-                    mbar_arrive_expect_tx(&sm->q_full, q_bytes);
-                    tma_load_3d(q_smem, tmap_q, &sm->q_full, 0, h0, t0);
-                    tma_load_3d(q_smem + kHalfBytes, tmap_q, &sm->q_full, 64, h0, t0);
-                } else {
-                    if (rank == 0) mbar_arrive_expect_tx(&sm->q_full, 2u * q_bytes);
-                    const uint32_t bar = map_to_cta(smem_u32(&sm->q_full), 0);
-                    tma_load_3d_pair(q_smem, tmap_q, bar, 0, h0, t0);
-                    tma_load_3d_pair(q_smem + kHalfBytes, tmap_q, bar, 64, h0, t0);
-                }
+                mbar_arrive_expect_tx(&sm->q_full, 2u * 128u * (uint32_t)(a.Gp * a.Tt));
+                tma_load_3d(q_smem, tmap_q, &sm->q_full, 0, h0, t0);
+                tma_load_3d(q_smem + kHalfBytes, tmap_q, &sm->q_full, 64, h0, t0);
             }
-            for (int t = 0; t < kKvStages && t < n_t; ++t) { issue_kv(t, 0); issue_kv(t, 1); }
+            for (int t = 0; t < 2 && t < n_t; ++t) { issue_kv(t, 0); issue_kv(t, 1); }
         }
     }
     if (q_idx != nullptr && n_t > 0 && warp < 4) {
@@ -616,142 +554,112 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
 
     if (skip) {
         // nothing is computed; the loads already under way get a bounded chance to land before the CTA retires
-        if (warp == 4 && lane == 0 && n_t > 0 && rank == 0) {
-            for (int i = 0; i < 4096 && !mbar_try_wait<false>(&sm->q_full, 0); ++i) {}
-            for (int s = 0; s < kKvStages && s < n_t; ++s) {
-                for (int i = 0; i < 4096 && !mbar_try_wait<false>(&sm->k_full[s], 0); ++i) {}
-                for (int i = 0; i < 4096 && !mbar_try_wait<false>(&sm->v_full[s], 0); ++i) {}
+        if (warp == 4 && lane == 0 && n_t > 0) {
+            for (int i = 0; i < 4096 && !mbar_try_wait(&sm->q_full, 0); ++i) {}
+            for (int s = 0; s < 2 && s < n_t; ++s) {
+                for (int i = 0; i < 4096 && !mbar_try_wait(&sm->k_full[s], 0); ++i) {}
+                for (int i = 0; i < 4096 && !mbar_try_wait(&sm->v_full[s], 0); ++i) {}
             }
         }
     } else if (warp == 4) {
         // ------------------------------------------------------------ TMA producer (the rest of the sub-steps)
-        if (n_t > kKvStages) {   // the whole warp walks the loop, one elected lane issues (uniform control flow)
+        if (n_t > 2) {   // the whole warp walks the loop, one elected lane issues (uniform control flow)
             bool ok = true;
-            for (int t = kKvStages; t < n_t && ok; ++t) {
-                const int slot = t % kKvStages;
-                const uint32_t round = (uint32_t)(t / kKvStages);
+            for (int t = 2; t < n_t && ok; ++t) {
+                const int slot = t & 1;
+                const uint32_t round = (uint32_t)(t >> 1);
                 for (int kv = 0; kv < 2 && ok; ++kv) {
                     uint64_t* empty = kv == 0 ? &sm->k_empty[slot] : &sm->v_empty[slot];
-                    ok = mbar_wait<false>(empty, (round - 1) & 1u, abort_flag, status, 10 + 2 * kv + (slot & 1));
+                    ok = mbar_wait(empty, (round - 1) & 1u, abort_flag, status, 10 + 2 * kv + slot);
                     ok = __all_sync(0xFFFFFFFFu, ok);
                     if (ok && elect_one()) issue_kv(t, kv);
                     __syncwarp();
                 }
             }
-            if (!ok && lane == 0 && rank == 0) {
+            if (!ok && lane == 0) {
                 // give loads already in flight a bounded chance to land before the CTA retires
-                for (int s = 0; s < kKvStages; ++s) {
-                    for (int i = 0; i < 4096 && !mbar_try_wait<false>(&sm->k_full[s], 0) && !mbar_try_wait<false>(&sm->k_full[s], 1); ++i) {}
-                    for (int i = 0; i < 4096 && !mbar_try_wait<false>(&sm->v_full[s], 0) && !mbar_try_wait<false>(&sm->v_full[s], 1); ++i) {}
+                for (int s = 0; s < 2; ++s) {
+                    for (int i = 0; i < 4096 && !mbar_try_wait(&sm->k_full[s], 0) && !mbar_try_wait(&sm->k_full[s], 1); ++i) {}
+                    for (int i = 0; i < 4096 && !mbar_try_wait(&sm->v_full[s], 0) && !mbar_try_wait(&sm->v_full[s], 1); ++i) {}
                 }
             }
         }
     } else if (warp == 5) {
-        // ------------------------------------------------------------ MMA issuer (pair form: the leader CTA's)
+        // ------------------------------------------------------------ MMA issuer
         // The whole warp walks the loop and waits on the barriers, one elected lane issues: control flow
         // stays uniform across the warp, so the operand descriptors can live in uniform registers.
-        if (n_t > 0 && rank == 0) {
-            constexpr uint32_t idesc_qk = make_idesc_bf16(kPair ? 2 * kBlockM : kBlockM, kSubN, 0);
-            constexpr uint32_t idesc_pv = make_idesc_bf16(kPair ? 2 * kBlockM : kBlockM, kD, 1);
+        if (n_t > 0) {
+            constexpr uint32_t idesc_qk = make_idesc_bf16(kBlockM, kSubN, 0);
+            constexpr uint32_t idesc_pv = make_idesc_bf16(kBlockM, kD, 1);
             const uint32_t qa = smem_u32(q_smem);
-            // the operand descriptors of ring slot 0 are built once, ahead of the loop; the other slots
-            // differ only in the start address field (16-byte units in the low bits)
-            uint64_t qd[kD / 16], kd[kD / 16], vd[kSubN / 16];
+            // S_b = Q K_t^T for the 64 keys in K slot b (= t & 1)
+            // every operand descriptor is fixed for the whole item: they are built once, ahead of the loop
+            uint64_t qd[kD / 16], kd[2][kD / 16], vd[2][kSubN / 16];
 #pragma unroll
             for (int kk = 0; kk < kD / 16; ++kk) {
                 qd[kk] = make_smem_desc(qa + (uint32_t)((kk & 3) * 32 + (kk >> 2) * kHalfBytes), 16, 1024);
-                kd[kk] = make_smem_desc(smem_u32(k_smem) + (uint32_t)((kk & 3) * 32 + (kk >> 2) * kKHalfBytes), 16, 1024);
+#pragma unroll
+                for (int b = 0; b < 2; ++b)
+                    kd[b][kk] = make_smem_desc(smem_u32(k_smem + (size_t)b * kSubBytes) + (uint32_t)((kk & 3) * 32 + (kk >> 2) * kSubHalfBytes), 16, 1024);
             }
 #pragma unroll
             for (int kk = 0; kk < kSubN / 16; ++kk)
-                vd[kk] = make_smem_desc(smem_u32(v_smem) + (uint32_t)kk * 2048u, kSubHalfBytes, 1024);
-            auto commit = [&](uint64_t* bar) {
-                if constexpr (kPair) tc_commit_pair(bar); else tc_commit(bar);
-            };
-            // S_b = Q K_t^T for the 64 keys in K slot `slot`
-            auto issue_qk = [&](int b, int slot) {
-                const uint64_t off = (uint64_t)((slot * kSlotBytes) >> 4);
 #pragma unroll
-                for (int kk = 0; kk < kD / 16; ++kk) {
-                    if constexpr (kPair) tc_mma_ss_pair(tmem + (uint32_t)(b * kSubN), qd[kk], kd[kk] + off, idesc_qk, kk > 0 ? 1u : 0u);
-                    else tc_mma_ss(tmem + (uint32_t)(b * kSubN), qd[kk], kd[kk] + off, idesc_qk, kk > 0 ? 1u : 0u);
-                }
-            };
-            // O (+)= P_b V_t for the 64 keys in V slot `slot`; P (bf16) sits in the first 32 columns of S_b
-            auto issue_pv = [&](int b, int slot, bool first) {
-                const uint64_t off = (uint64_t)((slot * kSlotBytes) >> 4);
+                for (int b = 0; b < 2; ++b)
+                    vd[b][kk] = make_smem_desc(smem_u32(v_smem + (size_t)b * kSubBytes) + (uint32_t)kk * 2048u, kSubHalfBytes, 1024);
+            auto issue_qk = [&](int b) {
 #pragma unroll
-                for (int kk = 0; kk < kSubN / 16; ++kk) {
-                    const uint32_t acc = (first && kk == 0) ? 0u : 1u;
-                    if constexpr (kPair) tc_mma_ts_pair(tmem + (uint32_t)kBlockN, tmem + (uint32_t)(b * kSubN + kk * 8), vd[kk] + off, idesc_pv, acc);
-                    else tc_mma_ts(tmem + (uint32_t)kBlockN, tmem + (uint32_t)(b * kSubN + kk * 8), vd[kk] + off, idesc_pv, acc);
-                }
+                for (int kk = 0; kk < kD / 16; ++kk)
+                    tc_mma_ss(tmem + (uint32_t)(b * kSubN), qd[kk], b ? kd[1][kk] : kd[0][kk], idesc_qk, kk > 0 ? 1u : 0u);
             };
-            bool ok = mbar_wait<false>(&sm->q_full, 0, abort_flag, status, 20);
+            // O (+)= P_b V_t for the 64 keys in V slot b; P (bf16) sits in the first 32 columns of S_b
+            auto issue_pv = [&](int b, bool first) {
+#pragma unroll
+                for (int kk = 0; kk < kSubN / 16; ++kk)
+                    tc_mma_ts(tmem + (uint32_t)kBlockN, tmem + (uint32_t)(b * kSubN + kk * 8), b ? vd[1][kk] : vd[0][kk], idesc_pv,
+                              (first && kk == 0) ? 0u : 1u);
+            };
+            bool ok = mbar_wait(&sm->q_full, 0, abort_flag, status, 20);
             ok = __all_sync(0xFFFFFFFFu, ok);
             for (int t = 0; t < 2 && t < n_t && ok; ++t) {   // the first two S tiles
-                ok = mbar_wait<false>(&sm->k_full[t], 0, abort_flag, status, 30 + t);
+                ok = mbar_wait(&sm->k_full[t], 0, abort_flag, status, 30 + t);
                 ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) break;
                 tc_fence_after();
                 if (elect_one()) {
-                    issue_qk(t, t);
-                    commit(&sm->s_full[t]);
-                    commit(&sm->k_empty[t]);
+                    issue_qk(t);
+                    tc_commit(&sm->s_full[t]);
+                    tc_commit(&sm->k_empty[t]);
                 }
                 __syncwarp();
             }
-            DAF_MLAP_DECL;
-            // Two issue sections per sub-step: O += P_t V_t as soon as P_t arrives, then S for sub-step t + 2
-            // into the half that P_t frees.  (One merged section -- both products behind a single wait --
-            // measured 15 % slower: the two CTAs of an SM then take turns on the tensor pipe in runs of twelve
-            // MMAs and each one's P V product queues behind the other's Q K^T.)
             for (int t = 0; t < n_t && ok; ++t) {
                 const int b = t & 1;
-                const int slot = t % kKvStages;
-                ok = mbar_wait<false>(&sm->v_full[slot], (uint32_t)((t / kKvStages) & 1), abort_flag, status, 32 + b);
-                DAF_MLAP(ml_v);
-                if (ok) ok = mbar_wait<false>(&sm->p_full[b], (uint32_t)((t >> 1) & 1), abort_flag, status, 40 + b);
+                const uint32_t par = (uint32_t)((t >> 1) & 1);
+                ok = mbar_wait(&sm->v_full[b], par, abort_flag, status, 32 + b);
+                if (ok) ok = mbar_wait(&sm->p_full[b], par, abort_flag, status, 40 + b);
                 ok = __all_sync(0xFFFFFFFFu, ok);
-                DAF_MLAP(ml_p);
-                DAF_EV(t, 0);
                 if (!ok) break;
                 tc_fence_after();
                 if (elect_one()) {
-                    issue_pv(b, slot, t == 0);
-                    commit(&sm->v_empty[slot]);
-                    commit(&sm->pv_done);
+                    issue_pv(b, t == 0);
+                    tc_commit(&sm->v_empty[b]);
+                    tc_commit(&sm->pv_done[b]);
                 }
                 __syncwarp();
-                DAF_MLAP(ml_i);
-                DAF_EV(t, 1);
                 if (t + 2 < n_t) {
-                    const int slot2 = (t + 2) % kKvStages;
-                    ok = mbar_wait<false>(&sm->k_full[slot2], (uint32_t)(((t + 2) / kKvStages) & 1), abort_flag, status, 34 + b);
+                    ok = mbar_wait(&sm->k_full[b], (uint32_t)(((t + 2) >> 1) & 1), abort_flag, status, 34 + b);
                     ok = __all_sync(0xFFFFFFFFu, ok);
-                    DAF_MLAP(ml_k);
-                    DAF_EV(t, 2);
                     if (!ok) break;
                     tc_fence_after();
                     if (elect_one()) {
-                        issue_qk(b, slot2);
-                        commit(&sm->s_full[b]);
-                        commit(&sm->k_empty[slot2]);
+                        issue_qk(b);
+                        tc_commit(&sm->s_full[b]);
+                        tc_commit(&sm->k_empty[b]);
                     }
                     __syncwarp();
-                    DAF_MLAP(ml_i);
-                    DAF_EV(t, 3);
                 }
             }
-#ifdef DAF_TRACE
-            if (lane == 0) {
-                const unsigned cta = blockIdx.x;
-                if (cta < 65536u) {
-                    long long* tt = g_laps_mma + 8 * cta;
-                    tt[0] = clock64() - ml_begin; tt[1] = ml_v; tt[2] = ml_p; tt[3] = ml_k; tt[4] = ml_i; tt[5] = n_t;
-                }
-            }
-#endif
         }
     } else {
         // ------------------------------------------------------------ softmax + epilogue, one row per thread
@@ -767,54 +675,43 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
         const uint32_t s_addr = tmem + lane_addr;
         const uint32_t o_addr = tmem + lane_addr + (uint32_t)kBlockN;
         const float c = a.scale_log2;
-        // where this warp reports "P handed over" and "Q rows stored": the leader's barriers in the pair form
-        uint32_t p_full_addr0 = 0, p_full_addr1 = 0, q_full_addr = 0;
-        if constexpr (kPair) {
-            p_full_addr0 = map_to_cta(smem_u32(&sm->p_full[0]), 0);
-            p_full_addr1 = map_to_cta(smem_u32(&sm->p_full[1]), 0);
-            q_full_addr = map_to_cta(smem_u32(&sm->q_full), 0);
-        }
 
-        if (q_idx != nullptr && n_t > 0 && lane == 0) {   // this warp's Q rows were stored before the set-up barrier
-            if constexpr (kPair) mbar_arrive_cluster(q_full_addr); else mbar_arrive(&sm->q_full);
-        }
+        if (q_idx != nullptr && n_t > 0 && lane == 0) mbar_arrive(&sm->q_full);   // this warp's Q rows were stored before the set-up barrier
         float m = -INFINITY, l = 0.f;
         bool ok = true;
         DAF_LAP_DECL;
         for (int t = 0; t < n_t; ++t) {
             const int b = t & 1;
-            ok = mbar_wait<false>(&sm->s_full[b], (uint32_t)((t >> 1) & 1), abort_flag, status, 50 + b);
+            ok = mbar_wait(&sm->s_full[b], (uint32_t)((t >> 1) & 1), abort_flag, status, 50 + b);
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) break;
             tc_fence_after();
             if (threadIdx.x == 0 && t == 0) DAF_STAMP(2);
             DAF_LAP(lap_s);
-            if (warp == 0) DAF_EV(t, 4);
             const float alpha = softmax_core<2>(s_addr + (uint32_t)(b * kSubN), key_begin + t * kSubN, limit, c, m, l);
             DAF_LAP(lap_soft);
-            if (warp == 0) DAF_EV(t, 5);
-            if (t > 0) {
-                // O may be touched, and the next product be issued, only once the previous product has completed
-                ok = mbar_wait<false>(&sm->pv_done, (uint32_t)((t - 1) & 1), abort_flag, status, 60);
+            if (t > 0 && __any_sync(0xFFFFFFFFu, alpha != 1.f)) {
+                // A row of this warp has to be rescaled: O may be touched only once the product before has
+                // completed.  (Rare: the running maximum is kept stale up to 2^8.  When no row needs it the warp
+                // does not wait at all -- the products run in issue order, so P_t may be handed over while
+                // O += P_{t-1} V_{t-1} is still under way.)  Sub-steps alternate between two barriers, so the
+                // phase waited for is unambiguous although the warp has not observed every phase.
+                ok = mbar_wait(&sm->pv_done[(t - 1) & 1], (uint32_t)(((t - 1) >> 1) & 1), abort_flag, status, 60);
                 ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) break;
                 tc_fence_after();
-                if (warp == 0) DAF_EV(t, 6);
-                if (__any_sync(0xFFFFFFFFu, alpha != 1.f)) rescale_o(o_addr, alpha);
+                rescale_o(o_addr, alpha);
             }
             tc_wait_st();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) {   // one arrival per warp: all its rows of P (and of O) are in place
-                if constexpr (kPair) mbar_arrive_cluster(b ? p_full_addr1 : p_full_addr0); else mbar_arrive(&sm->p_full[b]);
-            }
+            if (lane == 0) mbar_arrive(&sm->p_full[b]);   // one arrival per warp: all its rows of P (and of O) are in place
             DAF_LAP(lap_pv);
-            if (warp == 0) DAF_EV(t, 7);
         }
         if (threadIdx.x == 0) DAF_STAMP(3);
         // ---- epilogue
         if (ok && n_t > 0) {
-            ok = mbar_wait<false>(&sm->pv_done, (uint32_t)((n_t - 1) & 1), abort_flag, status, 61);
+            ok = mbar_wait(&sm->pv_done[(n_t - 1) & 1], (uint32_t)(((n_t - 1) >> 1) & 1), abort_flag, status, 61);
             ok = __all_sync(0xFFFFFFFFu, ok);
         }
         if (ok) {
@@ -836,18 +733,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
 
     if (threadIdx.x == 0) DAF_STAMP(4);
     tc_fence_before();
-    if constexpr (kPair) {
-        // neither CTA may retire, or give its tensor memory back, while the other can still signal its
-        // barriers or the pair's MMAs can still write its tensor memory
-        __syncwarp();
-        cluster_arrive();
-        cluster_wait();
-    } else {
-        __syncthreads();
-    }
+    __syncthreads();
     if (warp == 5) {
         tc_fence_after();
-        if constexpr (kPair) tmem_dealloc_pair(tmem, kAttnTmemCols); else tmem_dealloc(tmem, kAttnTmemCols);
+        tmem_dealloc(tmem, kAttnTmemCols);
     }
     DAF_KT_END(0);
 #ifdef DAF_TRACE
@@ -1018,47 +907,11 @@ static int set_kernel_attributes() {
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !attr_done[dev].load(std::memory_order_acquire)) {
-        cudaError_t e = cudaFuncSetAttribute(attn_fwd_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttnSmemBytes);
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(attn_fwd_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttnSmemBytes);
+        cudaError_t e = cudaFuncSetAttribute(attn_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttnSmemBytes);
         if (e != cudaSuccess) { set_cuda_error(e); return DAF_ERR_CUDA; }
         attr_done[dev].store(true, std::memory_order_release);
     }
     return DAF_OK;
-}
-
-// Which form of the attention kernel a launch uses: the single-CTA form, unless DAF_ATTN_PAIR=1 is set in the
-// environment when the library is first used (the pair form measured slower, see the kernel's comment).
-static bool use_pair_form() {
-    static const bool pair = [] {
-        const char* e = getenv("DAF_ATTN_PAIR");
-        return e != nullptr && e[0] == '1';
-    }();
-    return pair;
-}
-
-// Launches the attention kernel over `items` work items (1-D list) or, single form only, a 3-D grid.
-static cudaError_t launch_attn_kernel(bool pair, dim3 grid, cudaStream_t stream, bool after_kernel, const CUtensorMap& tq0,
-                                      const CUtensorMap& tk0, const CUtensorMap& tv0, const CUtensorMap& tq1,
-                                      const CUtensorMap& tk1, const CUtensorMap& tv1, const CUtensorMap& to0,
-                                      const CUtensorMap& to1, const AttnArgs& a) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = grid;
-    cfg.blockDim = dim3(kAttnThreads);
-    cfg.dynamicSmemBytes = kAttnSmemBytes;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[2];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = after_kernel ? 1 : 0;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    if (pair) {
-        attr[1].id = cudaLaunchAttributeClusterDimension;
-        attr[1].val.clusterDim.x = 2; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
-        cfg.numAttrs = 2;
-        return cudaLaunchKernelEx(&cfg, attn_fwd_kernel<true>, tq0, tk0, tv0, tq1, tk1, tv1, to0, to1, a);
-    }
-    return cudaLaunchKernelEx(&cfg, attn_fwd_kernel<false>, tq0, tk0, tv0, tq1, tk1, tv1, to0, to1, a);
 }
 
 // How a single problem is cut into CTAs: one per (head block, token block), and for the question rows,
@@ -1066,7 +919,6 @@ static cudaError_t launch_attn_kernel(bool pair, dim3 grid, cudaStream_t stream,
 
 AttnPlan plan_attention(int n_q, int n_kv, int Hq, int G, int causal_off, bool pack_group, bool allow_split) {
     AttnPlan pl;
-    const bool pair = use_pair_form();
     pl.Gp = pack_group ? G : 1;
     if (pl.Gp > 128) pl.Gp = 1;
     pl.Tt = kBlockM / pl.Gp;
@@ -1078,9 +930,8 @@ AttnPlan plan_attention(int n_q, int n_kv, int Hq, int G, int causal_off, bool p
     pl.n_splits = 1;
     pl.tiles_per_split = total_tiles > 0 ? total_tiles : 1;
     if (allow_split && total_tiles > 1) {
-        // resident items: two CTAs per SM; in the pair form an item is a pair of CTAs on two SMs
-        const int ctas = (pair ? (pl.n_tb + 1) / 2 : pl.n_tb) * pl.head_blocks;
-        const int slots = pair ? kNumSMs : kNumSMs * 2;
+        const int ctas = pl.n_tb * pl.head_blocks;
+        const int slots = kNumSMs * 2;
         int want = ctas > 0 ? slots / ctas : 1;
         if (want > kMaxSplits) want = kMaxSplits;
         if (want > total_tiles) want = total_tiles;
@@ -1132,14 +983,14 @@ bool operator<(const JointShape& a, const JointShape& b) {
 
 // Fills the fields of `jp` that follow from (chunk, n_splits_q).
 void set_choice(JointPlan& jp, int chunk, int n_splits_q, int L_q, int L_d, int Hq) {
-    if (chunk < (jp.n_units_i + 31) / 32) chunk = (jp.n_units_i + 31) / 32;   // at most 32 ranges per unit
+    if (chunk < (jp.n_tb_i + 31) / 32) chunk = (jp.n_tb_i + 31) / 32;   // at most 32 ranges per token block
     if (chunk < 1) chunk = 1;
-    if (chunk > jp.n_units_i) chunk = jp.n_units_i;
+    if (chunk > jp.n_tb_i) chunk = jp.n_tb_i;
     jp.chunk = chunk;
-    jp.n_slots = slots_before(jp.n_units_i, chunk);
+    jp.n_slots = slots_before(jp.n_tb_i, chunk);
     jp.part_bytes_i = 0;
-    if (chunk < jp.n_units_i) {
-        const size_t rows = (size_t)jp.n_slots * jp.unit_blocks * kBlockM * Hq;
+    if (chunk < jp.n_tb_i) {
+        const size_t rows = (size_t)jp.n_slots * kBlockM * Hq;
         jp.part_bytes_i = rows * kD * sizeof(float) + (rows * sizeof(float) + 255) / 256 * 256;
     }
     jp.items_i = Hq * jp.n_slots;
@@ -1147,14 +998,13 @@ void set_choice(JointPlan& jp, int chunk, int n_splits_q, int L_q, int L_d, int 
     if (n_splits_q < 1) n_splits_q = 1;
     jp.tiles_per_split_q = (tiles_q + n_splits_q - 1) / n_splits_q;
     jp.n_splits_q = (tiles_q + jp.tiles_per_split_q - 1) / jp.tiles_per_split_q;
-    jp.items_q = jp.head_blocks_q * jp.n_units_q * jp.n_splits_q;
+    jp.items_q = jp.head_blocks_q * jp.n_tb_q * jp.n_splits_q;
     jp.part_bytes_q = attn_partial_bytes(L_q, Hq, jp.n_splits_q);
 }
 
 // Predicted time of the attention launch + merge for a filled plan, in microseconds.
 float predict_us(const JointPlan& jp, int k, int L_q, int L_d, int Hq) {
-    // two CTAs per SM; an item of the pair form occupies one CTA slot on each SM of a TPC
-    const int slots = jp.unit_blocks == 2 ? kNumSMs : kNumSMs * 2;
+    const int slots = kNumSMs * 2;
     std::priority_queue<float, std::vector<float>, std::greater<float>> free_at;
     for (int i = 0; i < slots; ++i) free_at.push(0.f);
     float makespan = 0.f;
@@ -1169,8 +1019,8 @@ float predict_us(const JointPlan& jp, int k, int L_q, int L_d, int Hq) {
     };
     // question items: split-major, token blocks from the last one down, head blocks together
     for (int s = 0; s < jp.n_splits_q; ++s)
-        for (int u = jp.n_units_q - 1; u >= 0; --u) {
-            const int last_tok = (u + 1) * jp.unit_blocks * jp.Tt_q < L_q ? (u + 1) * jp.unit_blocks * jp.Tt_q : L_q;
+        for (int u = jp.n_tb_q - 1; u >= 0; --u) {
+            const int last_tok = (u + 1) * jp.Tt_q < L_q ? (u + 1) * jp.Tt_q : L_q;
             const int tiles_total = (L_d + last_tok + kBlockN - 1) / kBlockN;
             int tiles = tiles_total - s * jp.tiles_per_split_q;
             if (tiles > jp.tiles_per_split_q) tiles = jp.tiles_per_split_q;
@@ -1183,13 +1033,13 @@ float predict_us(const JointPlan& jp, int k, int L_q, int L_d, int Hq) {
         while (jp.chunk * (g + 1) * (g + 2) / 2 <= slot) ++g;
         const int rem = slot - jp.chunk * g * (g + 1) / 2;
         const int unit = g * jp.chunk + rem / (g + 1), range = rem % (g + 1);
-        const int n_tiles = jp.unit_blocks * (unit + 1) < jp.n_tb_i ? jp.unit_blocks * (unit + 1) : jp.n_tb_i;
+        const int n_tiles = unit + 1 < jp.n_tb_i ? unit + 1 : jp.n_tb_i;
         run(Hq, (range + 1) * n_tiles / (g + 1) - range * n_tiles / (g + 1));
-        if (g >= 1) part_rows_i += (size_t)jp.unit_blocks * kBlockM * Hq;
+        if (g >= 1) part_rows_i += (size_t)kBlockM * Hq;
     }
     (void)k;
     const float merge_mb = (float)(jp.part_bytes_q + part_rows_i * 516) / 1e6f;
-    const bool merges = jp.n_splits_q > 1 || jp.chunk < jp.n_units_i;
+    const bool merges = jp.n_splits_q > 1 || jp.chunk < jp.n_tb_i;
     return makespan + (merges ? kCostMergeUs + kCostMergeUsPerMB * merge_mb : 0.f);
 }
 }  // namespace
@@ -1205,17 +1055,14 @@ JointPlan plan_joint(int k, int L_q, int L_d, int Hq, int G) {
         if (it != cache.end()) return it->second;
     }
     JointPlan jp;
-    jp.unit_blocks = use_pair_form() ? 2 : 1;
     jp.n_tb_i = (k + kBlockM - 1) / kBlockM;
-    jp.n_units_i = (jp.n_tb_i + jp.unit_blocks - 1) / jp.unit_blocks;
     jp.Gp_q = G > 128 ? 1 : G;
     jp.Tt_q = kBlockM / jp.Gp_q;
     jp.n_tb_q = (L_q + jp.Tt_q - 1) / jp.Tt_q;
-    jp.n_units_q = (jp.n_tb_q + jp.unit_blocks - 1) / jp.unit_blocks;
     jp.head_blocks_q = Hq / jp.Gp_q;
     const int tiles_q = (L_d + L_q + kBlockN - 1) / kBlockN;
     if (forced) {
-        set_choice(jp, g_force_chunk > 0 ? g_force_chunk : jp.n_units_i, g_force_splits_q > 0 ? g_force_splits_q : 1, L_q, L_d, Hq);
+        set_choice(jp, g_force_chunk > 0 ? g_force_chunk : jp.n_tb_i, g_force_splits_q > 0 ? g_force_splits_q : 1, L_q, L_d, Hq);
         g_last_predicted_us = predict_us(jp, k, L_q, L_d, Hq);
         return jp;
     }
@@ -1224,8 +1071,8 @@ JointPlan plan_joint(int k, int L_q, int L_d, int Hq, int G) {
     JointPlan best = jp;
     float best_us = -1.f;
     for (int m = 1; m <= 6; ++m) {
-        const int chunk = (jp.n_units_i + m - 1) / m;
-        if (m > 1 && chunk == (jp.n_units_i + m - 2) / (m - 1)) continue;   // same cut as the previous candidate
+        const int chunk = (jp.n_tb_i + m - 1) / m;
+        if (m > 1 && chunk == (jp.n_tb_i + m - 2) / (m - 1)) continue;   // same cut as the previous candidate
         int last_tps = -1;
         for (int n = 1; n <= kMaxSplits && n <= tiles_q; ++n) {
             JointPlan cand = jp;
@@ -1248,7 +1095,7 @@ extern "C" void daf_dbg_joint_force(int chunk, int n_splits_q) { g_force_chunk =
 extern "C" float daf_dbg_joint_predicted_us(void) { return g_last_predicted_us; }
 extern "C" void daf_dbg_joint_plan(int k, int L_q, int L_d, int Hq, int G, int* out) {
     const JointPlan jp = plan_joint(k, L_q, L_d, Hq, G);
-    out[0] = jp.chunk; out[1] = jp.n_units_i; out[2] = jp.n_splits_q; out[3] = jp.items_i + jp.items_q;
+    out[0] = jp.chunk; out[1] = jp.n_tb_i; out[2] = jp.n_splits_q; out[3] = jp.items_i + jp.items_q;
 }
 #endif
 
@@ -1266,8 +1113,8 @@ static void fill_problem(SegArgs* s, int n_q, int n_kv, int Hq, int G, int Gp, i
     s->lse = lse;
 }
 
-static void fill_combine(CombineSeg* c, const SegArgs& s, int unit_blocks) {
-    const int unit_tokens = unit_blocks * kBlockM;   // packed causal attention has one head per tile: 128 tokens per token block
+static void fill_combine(CombineSeg* c, const SegArgs& s) {
+    const int unit_tokens = kBlockM;   // packed causal attention has one head per tile: a unit is 128 tokens
     c->part_o = s.part_o; c->part_lse = s.part_lse;
     c->n_q = s.n_q; c->Hq = s.Hq;
     c->n_splits = s.chunk == 0 ? s.n_splits : 0;
@@ -1299,11 +1146,9 @@ int launch_attention(const void* q, const void* k, const void* v, int n_q, int n
     const size_t need = attn_partial_bytes(n_q, Hq, pl.n_splits);
     if (need > scratch_bytes) return DAF_ERR_WORKSPACE;
 
-    const bool pair = use_pair_form();
     CUtensorMap tq, tk, tv;
     if (int rc = make_tmap(&tq, q, n_q, Hq, pl.Gp, pl.Tt)) return rc;
-    // pair form: a CTA loads 32 of a sub-step's 64 keys (all columns) and 64 of V's 128 columns (all keys)
-    if (int rc = make_tmap(&tk, k, n_kv, Hkv, 1, pair ? kSubN / 2 : kSubN)) return rc;
+    if (int rc = make_tmap(&tk, k, n_kv, Hkv, 1, kSubN)) return rc;
     if (int rc = make_tmap(&tv, v, n_kv, Hkv, 1, kSubN)) return rc;
     // rows in token order leave by tiled stores: the output as a [n_q, Hq, 128] tensor with the caller's row stride
     const bool out_tiled = dst_rows == nullptr;
@@ -1317,24 +1162,25 @@ int launch_attention(const void* q, const void* k, const void* v, int n_q, int n
     SegArgs& s = a.seg[0];
     fill_problem(&s, n_q, n_kv, Hq, G, pl.Gp, causal_off, q_pos, scale, out, out_row_stride_bytes, dst_rows, lse);
     s.out_tiled = out_tiled ? 1 : 0;
-    s.n_units = pair ? (pl.n_tb + 1) / 2 : pl.n_tb;
+    s.n_units = pl.n_tb;
     s.n_splits = pl.n_splits; s.tiles_per_split = pl.tiles_per_split;
     s.chunk = 0; s.n_slots = 0;
-    s.n_items = pl.head_blocks * s.n_units * pl.n_splits;
+    s.n_items = pl.head_blocks * pl.n_tb * pl.n_splits;
     s.part_o = reinterpret_cast<float*>(scratch);
     s.part_lse = pl.n_splits > 1 ? reinterpret_cast<float*>(reinterpret_cast<char*>(scratch) +
                                                             (size_t)pl.n_splits * n_q * Hq * kD * sizeof(float))
                                  : nullptr;
-    a.joint = pair ? 1 : 0;     // the pair form always walks a 1-D list of items (here: those of one problem)
+    a.joint = 0;
     a.status = status;
-    const dim3 grid = pair ? dim3((unsigned)(2 * s.n_items)) : dim3((unsigned)pl.head_blocks, (unsigned)pl.n_tb, (unsigned)pl.n_splits);
-    cudaError_t e = launch_attn_kernel(pair, grid, stream, after_kernel, tq, tk, tv, tq, tk, tv, to, to, a);
+    dim3 grid((unsigned)pl.head_blocks, (unsigned)pl.n_tb, (unsigned)pl.n_splits);
+    cudaError_t e = launch_kernel(attn_fwd_kernel, grid, dim3(kAttnThreads), kAttnSmemBytes, stream, after_kernel, tq, tk, tv, tq, tk, tv,
+                                  to, to, a);
     count_launch();
     if (e != cudaSuccess) { set_cuda_error(e); return DAF_ERR_CUDA; }
     if (int rc = check_launch()) return rc;
     if (pl.n_splits > 1) {
         CombineSeg c0, c1;
-        fill_combine(&c0, s, pair ? 2 : 1);
+        fill_combine(&c0, s);
         memset(&c1, 0, sizeof(c1));
         return launch_combine(c0, c1, stream);
     }
@@ -1379,12 +1225,10 @@ int launch_attention_joint(const void* q_imp, const void* q_fresh, const int32_t
     const bool gather_q = q_imp == nullptr;
     if (gather_q && (q_fresh == nullptr || idx == nullptr)) return DAF_ERR_INVALID_ARG;
     if (int rc = make_tmap(&tq0, gather_q ? q_question : q_imp, gather_q ? L_q : k, Hq, 1, kBlockM)) return rc;
-    const bool pair = jp.unit_blocks == 2;
-    const int k_box = pair ? kSubN / 2 : kSubN;    // pair form: a CTA loads 32 of a sub-step's 64 keys
-    if (int rc = make_tmap(&tk0, k_imp, k, Hkv, 1, k_box)) return rc;
+    if (int rc = make_tmap(&tk0, k_imp, k, Hkv, 1, kSubN)) return rc;
     if (int rc = make_tmap(&tv0, v_imp, k, Hkv, 1, kSubN)) return rc;
     if (int rc = make_tmap(&tq1, q_question, L_q, Hq, jp.Gp_q, jp.Tt_q)) return rc;
-    if (int rc = make_tmap(&tk1, kv_k, N, Hkv, 1, k_box)) return rc;
+    if (int rc = make_tmap(&tk1, kv_k, N, Hkv, 1, kSubN)) return rc;
     if (int rc = make_tmap(&tv1, kv_v, N, Hkv, 1, kSubN)) return rc;
     // final rows in token order (the compact layout) leave by tiled stores
     CUtensorMap to0 = tq1, to1 = tq1;
@@ -1401,7 +1245,7 @@ int launch_attention_joint(const void* q_imp, const void* q_fresh, const int32_t
     SegArgs& sq = a.seg[1];
     fill_problem(&sq, L_q, N, Hq, G, jp.Gp_q, L_d, nullptr, scale, out_question, out_row_stride_bytes, nullptr, nullptr);
     sq.out_tiled = 1;
-    sq.n_units = jp.n_units_q;
+    sq.n_units = jp.n_tb_q;
     sq.n_splits = jp.n_splits_q; sq.tiles_per_split = jp.tiles_per_split_q;
     sq.chunk = 0; sq.n_slots = 0;
     sq.n_items = jp.items_q;
@@ -1416,11 +1260,11 @@ int launch_attention_joint(const void* q_imp, const void* q_fresh, const int32_t
         si.q_src_rows = L_d;
     }
     si.out_tiled = imp_tiled ? 1 : 0;
-    si.n_units = jp.n_units_i;
+    si.n_units = jp.n_tb_i;
     si.n_splits = 1; si.tiles_per_split = jp.n_tb_i;
     si.chunk = jp.chunk; si.n_slots = jp.n_slots;
     si.n_items = jp.items_i;
-    const size_t rows_i = (size_t)jp.n_slots * jp.unit_blocks * kBlockM * Hq;
+    const size_t rows_i = (size_t)jp.n_slots * kBlockM * Hq;
     si.part_o = reinterpret_cast<float*>(sc + jp.part_bytes_q);
     si.part_lse = reinterpret_cast<float*>(sc + jp.part_bytes_q + rows_i * kD * sizeof(float));
     a.joint = 1;
@@ -1428,16 +1272,16 @@ int launch_attention_joint(const void* q_imp, const void* q_fresh, const int32_t
 
     const int items = jp.items_q + jp.items_i;
     if (launches & 1) {
-        const cudaError_t e = launch_attn_kernel(pair, dim3((unsigned)(pair ? 2 * items : items)), stream, after_kernel,
-                                                 tq0, tk0, tv0, tq1, tk1, tv1, to0, to1, a);
+        const cudaError_t e = launch_kernel(attn_fwd_kernel, dim3((unsigned)items), dim3(kAttnThreads), kAttnSmemBytes, stream,
+                                            after_kernel, tq0, tk0, tv0, tq1, tk1, tv1, to0, to1, a);
         count_launch();
         if (e != cudaSuccess) { set_cuda_error(e); return DAF_ERR_CUDA; }
         if (int rc = check_launch()) return rc;
     }
     if (!(launches & 2)) return DAF_OK;
     CombineSeg ci, cq;
-    fill_combine(&ci, si, jp.unit_blocks);
-    fill_combine(&cq, sq, jp.unit_blocks);
+    fill_combine(&ci, si);
+    fill_combine(&cq, sq);
     return launch_combine(ci, cq, stream);
 }
 
