@@ -409,9 +409,23 @@ def measure_config(env: Env, w: W.Workload, primary: bool):
         api.check(api.daf_deviation_scores(p, b.L["k_fresh"], b.L["v_fresh"], b.L["k_cached"], b.L["v_cached"],
                                            dev_scores), "daf_deviation_scores")
 
+    # the signal of three layers aggregated in one pass (what daf_select_from_kv runs ahead of the top-k): timed
+    # alone through that entry point with r = 0 and no question rows, so that nothing else is launched
+    n_sig_layers = min(3, len(bufs))
+    p_sig = api.make_params(w.L_d, 0, 0.0, w.n_q_heads, w.n_kv_heads)
+    ws_sig = api.alloc_workspace(p_sig, dev)
+
+    def st_dev_sum(b):
+        i = bufs.index(b)
+        grp = [bufs[(i + j) % len(bufs)].L for j in range(n_sig_layers)]
+        api.check(api.daf_select_from_kv(p_sig, [g["k_fresh"] for g in grp], [g["v_fresh"] for g in grp],
+                                         [g["k_cached"] for g in grp], [g["v_cached"] for g in grp], None, None, None, None,
+                                         None, None, None, None, None, dev_scores, ws_sig), "daf_select_from_kv (signal only)")
+
     for b in bufs:                       # the stand-alone important-token stage below reads packed Q rows
         st_select(b, pack_q=True)
     us_dev = time_stage(st_dev, bufs)
+    us_dev_sum = time_stage(st_dev_sum, bufs)
     us_select = time_stage(st_select, bufs)
     us_imp = time_stage(st_imp, bufs) if w.k > 0 else 0.0
     us_qd = time_stage(st_qd, bufs) if w.L_q > 0 else 0.0
@@ -544,7 +558,11 @@ def measure_config(env: Env, w: W.Workload, primary: bool):
                               "kv_gbs": 2 * w.N * w.n_kv_heads * 256 / (us_qd * 1e-6) / 1e9 if us_qd else None},
             "deviation_scores": {"bound": "hbm", "us": us_dev, "gbs": dev_bytes / (us_dev * 1e-6) / 1e9,
                                  "frac": dev_bytes / (us_dev * 1e-6) / 1e9 / peaks["hbm_gbs"],
-                                 "note": "signal layers only; not part of the per-layer step"},
+                                 "note": "one signal layer; not part of the per-layer step"},
+            "deviation_sum": {"bound": "hbm", "us": us_dev_sum, "signal_layers": n_sig_layers,
+                              "gbs": (n_sig_layers * (dev_bytes - 4 * w.L_d) + 4 * w.L_d) / (us_dev_sum * 1e-6) / 1e9,
+                              "frac": (n_sig_layers * (dev_bytes - 4 * w.L_d) + 4 * w.L_d) / (us_dev_sum * 1e-6) / 1e9 / peaks["hbm_gbs"],
+                              "note": "signal of several layers aggregated in one pass (first kernel of daf_select_from_kv)"},
             "select_gather_update": {"bound": "hbm", "gbs": gather_bytes / (us_select * 1e-6) / 1e9,
                                      "frac": gather_bytes / (us_select * 1e-6) / 1e9 / peaks["hbm_gbs"],
                                      "note": "includes the latency-bound top-k kernel"},

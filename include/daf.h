@@ -119,6 +119,24 @@ int daf_select(const daf_params* p, const float* scores, int32_t n_sig, const in
                int32_t* idx_out, void* q_pack, void* k_pack, void* v_pack,
                void* workspace, size_t workspace_bytes, void* stream);
 
+/* Step 1 starting from K/V instead of from scores (Methods item 1: the deviation signals of several layers,
+ * typically the 2nd to 4th, are aggregated and the tokens ranked by the aggregate).  The signal of layer l is
+ * the one daf_deviation_scores computes; the layers are added in ascending order in fp32, exactly as daf_select
+ * adds the rows of a score matrix, and the k highest sums are selected.  The per-layer score matrix is never
+ * written: one kernel streams the signal layers' K/V once and leaves one fp32 sum per document token.
+ *   n_sig           number of signal layers, 1..8
+ *   sig_k_fresh, sig_v_fresh, sig_k_cached, sig_v_cached
+ *                   HOST arrays of n_sig DEVICE pointers: fresh and offline K/V of each signal layer,
+ *                   [>= L_d, n_kv_heads, 128] each (the arrays are read before the call returns)
+ *   q_fresh ... v_pack   the layer being processed, exactly as in daf_select (gather and cache update)
+ *   signal_sum_out  optional fp32 [L_d] (device): receives the aggregated signal; NULL keeps it in the workspace
+ */
+int daf_select_from_kv(const daf_params* p, int32_t n_sig, const void* const* sig_k_fresh, const void* const* sig_v_fresh,
+                       const void* const* sig_k_cached, const void* const* sig_v_cached,
+                       const void* q_fresh, const void* k_fresh, const void* v_fresh, void* kv_k, void* kv_v,
+                       int32_t* idx_out, void* q_pack, void* k_pack, void* v_pack, float* signal_sum_out,
+                       void* workspace, size_t workspace_bytes, void* stream);
+
 /* Step 2 (Methods item 1; the r^2 L_d^2 term of the complexity analysis): causal
  * softmax attention among the k packed rows, query head h reading KV head
  * h / (n_q_heads / n_kv_heads).  bf16 operands, fp32 accumulation and softmax.

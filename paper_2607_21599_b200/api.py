@@ -32,7 +32,7 @@ EXPORTS = [
     "daf_layer_host", "daf_poll_status", "daf_strerror", "daf_last_cuda_error", "daf_launch_count",
     "daf_qd_attn_static", "daf_qd_attn_static_max_bytes", "daf_deviation_scores", "daf_blend_attn",
     "daf_imp_qd_attn", "daf_selftest_bounded_wait", "daf_qd_attn_static_poll_status",
-    "daf_imp_qd_attn_launches",
+    "daf_imp_qd_attn_launches", "daf_select_from_kv",
 ]
 
 
@@ -83,6 +83,8 @@ def lib() -> ctypes.CDLL:
         L.daf_workspace_init.argtypes = [vp, sz, vp]
         L.daf_select.restype = ctypes.c_int
         L.daf_select.argtypes = [pp, vp, i32, vp] + [vp] * 3 + [vp] * 2 + [vp] * 4 + [vp, sz, vp]
+        L.daf_select_from_kv.restype = ctypes.c_int
+        L.daf_select_from_kv.argtypes = [pp, i32, vp, vp, vp, vp] + [vp] * 3 + [vp] * 2 + [vp] * 4 + [vp] + [vp, sz, vp]
         L.daf_important_attn.restype = ctypes.c_int
         L.daf_important_attn.argtypes = [pp, i32, vp, vp, vp, vp, i64, vp, vp, vp, sz, vp]
         L.daf_qd_attn.restype = ctypes.c_int
@@ -184,6 +186,24 @@ def daf_select(p, scores, n_sig, idx_in, q_fresh, k_fresh, v_fresh, kv_k, kv_v, 
     return lib().daf_select(ctypes.byref(p), _ptr(scores), int(n_sig), _ptr(idx_in), _ptr(q_fresh), _ptr(k_fresh),
                             _ptr(v_fresh), _ptr(kv_k), _ptr(kv_v), _ptr(idx_out), _ptr(q_pack), _ptr(k_pack),
                             _ptr(v_pack), _ptr(workspace), _nbytes(workspace), _stream(stream))
+
+
+def _ptr_array(tensors):
+    """A host array of device pointers (one per signal layer)."""
+    arr = (ctypes.c_void_p * len(tensors))()
+    for i, t in enumerate(tensors):
+        arr[i] = _ptr(t)
+    return arr
+
+
+def daf_select_from_kv(p, sig_k_fresh, sig_v_fresh, sig_k_cached, sig_v_cached, q_fresh, k_fresh, v_fresh, kv_k, kv_v,
+                       idx_out, q_pack, k_pack, v_pack, signal_sum_out, workspace, stream=None) -> int:
+    """sig_*: lists of n_sig device tensors (the signal layers' fresh and offline K/V)."""
+    n_sig = len(sig_k_fresh)
+    arrays = [_ptr_array(x) for x in (sig_k_fresh, sig_v_fresh, sig_k_cached, sig_v_cached)]
+    return lib().daf_select_from_kv(ctypes.byref(p), n_sig, *arrays, _ptr(q_fresh), _ptr(k_fresh), _ptr(v_fresh),
+                                    _ptr(kv_k), _ptr(kv_v), _ptr(idx_out), _ptr(q_pack), _ptr(k_pack), _ptr(v_pack),
+                                    _ptr(signal_sum_out), _ptr(workspace), _nbytes(workspace), _stream(stream))
 
 
 def daf_important_attn(p, k, q_pack, k_pack, v_pack, out, out_row_stride_bytes, dst_rows, lse, workspace,

@@ -51,6 +51,7 @@ int resolve_params(const daf_params* p, ResolvedParams* out) {
 
 struct Workspace {
     DeviceStatus* status;
+    float* signal_sums;       // [L_d] aggregated importance signal (daf_select_from_kv)
     void* select_scratch;
     void* attn_scratch;
     size_t attn_bytes;
@@ -72,8 +73,10 @@ static size_t attn_scratch_bytes(const ResolvedParams& rp) {
     return need;
 }
 
+static size_t signal_sum_bytes(const ResolvedParams& rp) { return ((size_t)rp.L_d * sizeof(float) + 255) / 256 * 256; }
+
 static size_t workspace_bytes(const ResolvedParams& rp) {
-    return kStatusBytes + select_scratch_bytes(rp.L_d) + attn_scratch_bytes(rp);
+    return kStatusBytes + signal_sum_bytes(rp) + select_scratch_bytes(rp.L_d) + attn_scratch_bytes(rp);
 }
 
 static int carve_workspace(const ResolvedParams& rp, void* workspace, size_t bytes, Workspace* ws) {
@@ -81,15 +84,17 @@ static int carve_workspace(const ResolvedParams& rp, void* workspace, size_t byt
     if (!aligned16(workspace)) return DAF_ERR_ALIGNMENT;
     char* base = reinterpret_cast<char*>(workspace);
     ws->status = reinterpret_cast<DeviceStatus*>(base);
-    ws->select_scratch = base + kStatusBytes;
-    ws->attn_scratch = base + kStatusBytes + select_scratch_bytes(rp.L_d);
-    ws->attn_bytes = bytes - kStatusBytes - select_scratch_bytes(rp.L_d);
+    ws->signal_sums = reinterpret_cast<float*>(base + kStatusBytes);
+    ws->select_scratch = base + kStatusBytes + signal_sum_bytes(rp);
+    ws->attn_scratch = base + kStatusBytes + signal_sum_bytes(rp) + select_scratch_bytes(rp.L_d);
+    ws->attn_bytes = bytes - kStatusBytes - signal_sum_bytes(rp) - select_scratch_bytes(rp.L_d);
     return DAF_OK;
 }
 
 static int do_select(const ResolvedParams& rp, const float* scores, int32_t n_sig, const int32_t* idx_in,
                      const void* q_fresh, const void* k_fresh, const void* v_fresh, void* kv_k, void* kv_v,
-                     int32_t* idx_out, void* q_pack, void* k_pack, void* v_pack, const Workspace& ws, cudaStream_t st) {
+                     int32_t* idx_out, void* q_pack, void* k_pack, void* v_pack, const Workspace& ws, cudaStream_t st,
+                     bool scores_from_previous_kernel = false) {
     if (scores != nullptr && n_sig < 1) return DAF_ERR_INVALID_ARG;
     if (rp.k > 0) {
         if (scores == nullptr && idx_in == nullptr) return DAF_ERR_INVALID_ARG;
@@ -103,7 +108,7 @@ static int do_select(const ResolvedParams& rp, const float* scores, int32_t n_si
     for (const void* ptr : ptrs)
         if (ptr != nullptr && !aligned16(ptr)) return DAF_ERR_ALIGNMENT;
     return launch_select(rp, scores, n_sig, idx_in, q_fresh, k_fresh, v_fresh, kv_k, kv_v, idx_out, q_pack, k_pack,
-                         v_pack, ws.status, ws.select_scratch, st);
+                         v_pack, ws.status, ws.select_scratch, st, scores_from_previous_kernel);
 }
 
 static int check_out(const void* out, int64_t stride_bytes, int Hq) {
@@ -143,6 +148,35 @@ int daf_select(const daf_params* p, const float* scores, int32_t n_sig, const in
     if (int rc = carve_workspace(rp, workspace, workspace_bytes_, &ws)) return rc;
     return do_select(rp, scores, n_sig, idx_in, q_fresh, k_fresh, v_fresh, kv_k, kv_v, idx_out, q_pack, k_pack, v_pack,
                      ws, (cudaStream_t)stream);
+}
+
+int daf_select_from_kv(const daf_params* p, int32_t n_sig, const void* const* sig_k_fresh, const void* const* sig_v_fresh,
+                       const void* const* sig_k_cached, const void* const* sig_v_cached,
+                       const void* q_fresh, const void* k_fresh, const void* v_fresh, void* kv_k, void* kv_v,
+                       int32_t* idx_out, void* q_pack, void* k_pack, void* v_pack, float* signal_sum_out,
+                       void* workspace, size_t workspace_bytes_, void* stream) {
+    ResolvedParams rp;
+    if (int rc = resolve_params(p, &rp)) return rc;
+    Workspace ws;
+    if (int rc = carve_workspace(rp, workspace, workspace_bytes_, &ws)) return rc;
+    if (n_sig < 1 || n_sig > kMaxSignalLayersHost) return DAF_ERR_INVALID_ARG;
+    if (!sig_k_fresh || !sig_v_fresh || !sig_k_cached || !sig_v_cached) return DAF_ERR_INVALID_ARG;
+    for (int l = 0; l < n_sig; ++l) {
+        const void* ptrs[] = {sig_k_fresh[l], sig_v_fresh[l], sig_k_cached[l], sig_v_cached[l]};
+        for (const void* ptr : ptrs) {
+            if (ptr == nullptr) return DAF_ERR_INVALID_ARG;
+            if (!aligned16(ptr)) return DAF_ERR_ALIGNMENT;
+        }
+    }
+    if (signal_sum_out != nullptr && (reinterpret_cast<uintptr_t>(signal_sum_out) & 15u) != 0) return DAF_ERR_ALIGNMENT;
+    if (rp.k > 0 && idx_out == nullptr) return DAF_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    float* sums = signal_sum_out != nullptr ? signal_sum_out : ws.signal_sums;
+    if (rp.L_d > 0)
+        if (int rc = launch_deviation_sum(rp, n_sig, sig_k_fresh, sig_v_fresh, sig_k_cached, sig_v_cached, sums, st)) return rc;
+    // the sums are one signal row: from here on this is daf_select, launched right behind the signal kernel
+    return do_select(rp, rp.L_d > 0 ? sums : nullptr, 1, nullptr, q_fresh, k_fresh, v_fresh, kv_k, kv_v, idx_out, q_pack, k_pack,
+                     v_pack, ws, st, /*scores_from_previous_kernel=*/true);
 }
 
 int daf_important_attn(const daf_params* p, int32_t k, const void* q_pack, const void* k_pack, const void* v_pack,

@@ -66,6 +66,7 @@ select_topk_kernel(const float* __restrict__ scores, int n_sig, int L_d, int k,
     namespace cg = cooperative_groups;
     cg::cluster_group cluster = cg::this_cluster();
     DAF_KT_BEGIN(0);
+    pdl_wait();                // the scores may come from the signal kernel launched just before
     pdl_launch_dependents();   // the gather kernel may start launching; it waits for this grid before reading idx
     extern __shared__ __align__(16) unsigned char sel_smem[];
     SelShared* sh = reinterpret_cast<SelShared*>(sel_smem);
@@ -291,6 +292,7 @@ select_topk_cta_kernel(const float* __restrict__ scores, int n_sig, int L_d, int
     uint32_t* cand = keys + padded(L_d);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     DAF_KT_BEGIN(0);
+    pdl_wait();                // the scores may come from the signal kernel launched just before
     pdl_launch_dependents();   // the gather kernel may start launching; it waits for this grid before reading idx
 
     // aggregate the signal rows in ascending row order (fp32 adds, no fusing), build keys, find their range
@@ -528,6 +530,45 @@ deviation_scores_kernel(const int4* __restrict__ k_fresh, const int4* __restrict
     }
 }
 
+// The same signal for several layers at once, aggregated on the fly (Methods, item 1: the signals of several
+// layers, typically the 2nd to 4th, are aggregated before the tokens are ranked).  One warp per token walks
+// the signal layers in ascending order: each layer's value is computed exactly as deviation_scores_kernel
+// computes it (same chunk order, same shuffle tree) and added to the running fp32 sum with a plain
+// round-to-nearest add, subnormals kept -- the order and arithmetic in which the selection kernels
+// aggregate the rows of a score matrix -- so ranking the sums gives the positions that the two-step route
+// (one daf_deviation_scores call per layer, then daf_select on the [n_sig, L_d] matrix) would give, without
+// that matrix ever being written.
+constexpr int kMaxSignalLayers = 8;
+struct SignalLayers {
+    const int4* k_fresh[kMaxSignalLayers]; const int4* v_fresh[kMaxSignalLayers];
+    const int4* k_cached[kMaxSignalLayers]; const int4* v_cached[kMaxSignalLayers];
+    int n;
+};
+
+__global__ void __launch_bounds__(256)
+deviation_sum_kernel(const SignalLayers layers, int L_d, int chunks_per_row, float* __restrict__ sums) {
+    pdl_launch_dependents();   // the selection kernel may start launching; it waits for this grid before reading sums
+    const int lane = threadIdx.x & 31;
+    const int warps_per_grid = (int)(gridDim.x * (blockDim.x >> 5));
+    for (int tok = (int)(blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)); tok < L_d; tok += warps_per_grid) {
+        const size_t base = (size_t)tok * chunks_per_row;
+        float total = 0.f;
+        for (int l = 0; l < layers.n; ++l) {
+            const int4* kf = layers.k_fresh[l]; const int4* vf = layers.v_fresh[l];
+            const int4* kc = layers.k_cached[l]; const int4* vc = layers.v_cached[l];
+            float acc = 0.f;
+            for (int c = lane; c < chunks_per_row; c += 32) {
+                acc += sq_dev8(__ldg(kf + base + c), __ldg(kc + base + c));
+                acc += sq_dev8(__ldg(vf + base + c), __ldg(vc + base + c));
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+            total = l == 0 ? acc : add_rn_keep_subnormals(total, acc);
+        }
+        if (lane == 0) sums[tok] = total;
+    }
+}
+
 // ----------------------------------------------------------------- host side
 // Measured on B200 (selection alone): one CTA 4.9 / 5.3 / 8.1 us at 6K / 8K / 16K tokens, the cluster of eight
 // 7.0 / 5.8 / 7.6 us: one CTA up to 8K tokens, the cluster beyond.
@@ -549,9 +590,9 @@ static size_t select_smem_bytes(int L_d) {
 int launch_select(const ResolvedParams& rp, const float* scores, int n_sig, const int32_t* idx_in,
                   const void* q_fresh, const void* k_fresh, const void* v_fresh, void* kv_k, void* kv_v,
                   int32_t* idx_out, void* q_pack, void* k_pack, void* v_pack,
-                  DeviceStatus* status, void* scratch, cudaStream_t stream) {
+                  DeviceStatus* status, void* scratch, cudaStream_t stream, bool scores_from_previous_kernel) {
     const int32_t* idx_src = idx_in;
-    if (scores != nullptr && rp.L_d > 0) {
+    if (scores != nullptr && rp.L_d > 0 && rp.k > 0) {
         static std::atomic<bool> attr_done[64];   // per device; a concurrent first call sets the same values
         int dev = 0;
         cudaGetDevice(&dev);
@@ -566,11 +607,15 @@ int launch_select(const ResolvedParams& rp, const float* scores, int n_sig, cons
         }
         if (rp.L_d <= g_sel1_max_keys) {
             const size_t smem1 = sizeof(Sel1Shared) + ((size_t)padded(rp.L_d) + rp.L_d) * sizeof(uint32_t);   // keys and candidate list
-            select_topk_cta_kernel<<<1, kSel1Threads, smem1, stream>>>(scores, n_sig, rp.L_d, rp.k, idx_out);
+            const cudaError_t e = launch_kernel(select_topk_cta_kernel, dim3(1), dim3(kSel1Threads), smem1, stream,
+                                                scores_from_previous_kernel, scores, n_sig, rp.L_d, rp.k, idx_out);
+            if (e != cudaSuccess) { set_cuda_error(e); return DAF_ERR_CUDA; }
         } else {
             const size_t smem = select_smem_bytes(rp.L_d);
-            select_topk_kernel<<<kSelCluster, kSelThreads, smem, stream>>>(scores, n_sig, rp.L_d, rp.k,
-                                                                reinterpret_cast<uint32_t*>(scratch), idx_out);
+            const cudaError_t e = launch_kernel(select_topk_kernel, dim3(kSelCluster), dim3(kSelThreads), smem, stream,
+                                                scores_from_previous_kernel, scores, n_sig, rp.L_d, rp.k,
+                                                reinterpret_cast<uint32_t*>(scratch), idx_out);
+            if (e != cudaSuccess) { set_cuda_error(e); return DAF_ERR_CUDA; }
         }
         count_launch();
         if (int rc = check_launch()) return rc;
@@ -612,6 +657,28 @@ int launch_deviation_scores(const ResolvedParams& rp, const void* k_fresh, const
     deviation_scores_kernel<<<blocks, warps * 32, 0, stream>>>(
         reinterpret_cast<const int4*>(k_fresh), reinterpret_cast<const int4*>(v_fresh),
         reinterpret_cast<const int4*>(k_cached), reinterpret_cast<const int4*>(v_cached), rp.L_d, rp.Hkv * 16, scores);
+    count_launch();
+    return check_launch();
+}
+
+int launch_deviation_sum(const ResolvedParams& rp, int n_sig, const void* const* k_fresh, const void* const* v_fresh,
+                         const void* const* k_cached, const void* const* v_cached, float* sums, cudaStream_t stream) {
+    if (rp.L_d == 0) return DAF_OK;
+    if (n_sig < 1 || n_sig > kMaxSignalLayers) return DAF_ERR_INVALID_ARG;
+    SignalLayers layers;
+    layers.n = n_sig;
+    for (int l = 0; l < kMaxSignalLayers; ++l) {
+        const int j = l < n_sig ? l : 0;
+        layers.k_fresh[l] = reinterpret_cast<const int4*>(k_fresh[j]);
+        layers.v_fresh[l] = reinterpret_cast<const int4*>(v_fresh[j]);
+        layers.k_cached[l] = reinterpret_cast<const int4*>(k_cached[j]);
+        layers.v_cached[l] = reinterpret_cast<const int4*>(v_cached[j]);
+    }
+    const int warps = 8;
+    int blocks = (rp.L_d + warps - 1) / warps;
+    const int max_blocks = 148 * 8;
+    if (blocks > max_blocks) blocks = max_blocks;
+    deviation_sum_kernel<<<blocks, warps * 32, 0, stream>>>(layers, rp.L_d, rp.Hkv * 16, sums);
     count_launch();
     return check_launch();
 }

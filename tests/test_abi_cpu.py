@@ -107,6 +107,14 @@ def test_host_side_argument_validation(lib):
     assert api.daf_layer(r0, None, 0, None, buf, buf, buf, None, buf, None, None, None, None, buf, None, ws) == api.DAF_ERR_INVALID_ARG
     # important rows without packed K/V buffers
     assert api.daf_layer(ok, buf, 1, None, buf, buf, buf, buf, buf, buf, buf, None, buf, buf, None, ws) == api.DAF_ERR_INVALID_ARG
+    # selection straight from the signal layers' K/V: the number of layers and every pointer are checked first
+    sig = lambda n: [buf] * n  # noqa: E731
+    skv = lambda n, kf=None, wsp=ws: api.daf_select_from_kv(ok, kf if kf is not None else sig(n), sig(n), sig(n), sig(n), buf, buf, buf,  # noqa: E731
+                                                           buf, buf, buf, buf, buf, buf, None, wsp)
+    assert skv(0) == api.DAF_ERR_INVALID_ARG and skv(9) == api.DAF_ERR_INVALID_ARG
+    assert skv(2, kf=[buf, None]) == api.DAF_ERR_INVALID_ARG
+    assert skv(2, kf=[buf, buf[8:]]) == api.DAF_ERR_ALIGNMENT
+    assert skv(2, wsp=None) == api.DAF_ERR_WORKSPACE
     # the self-test of the bounded wait checks its arguments before it launches anything
     assert api.daf_selftest_bounded_wait(None, 50) == api.DAF_ERR_WORKSPACE
     assert api.daf_selftest_bounded_wait(ws[:64], 50) == api.DAF_ERR_WORKSPACE

@@ -141,6 +141,67 @@ def test_deviation_scores_match_oracle(L_d, L_q, Hkv):
         assert ref[sel].min() >= ref[~sel].max() * (1 - 1e-4)
 
 
+@pytest.mark.parametrize("L_d,L_q,Hkv,n_sig,r", [(1024, 32, 4, 3, 0.15), (6144, 64, 4, 3, 0.15), (777, 0, 8, 1, 0.3),
+                                                 (20000, 16, 8, 2, 0.1), (40, 3, 1, 8, 0.5)])
+def test_selection_straight_from_the_signal_layers_kv(L_d, L_q, Hkv, n_sig, r):
+    """daf_select_from_kv: the aggregated signal equals the per-layer signals of daf_deviation_scores added in
+    ascending layer order in fp32 (bit for bit), agrees with the fp64 oracle within the signal's tolerance, and the
+    selected positions are exactly what the oracle's selection gives on those fp32 sums; gather and cache update
+    as in daf_select."""
+    dev = "cuda"
+    N, Hq = L_d + L_q, 2 * Hkv
+    layers = []
+    for l in range(n_sig):
+        kf, vf = _normal((N, Hkv, 128), 500 + 10 * l).to(dev), _normal((N, Hkv, 128), 501 + 10 * l).to(dev)
+        # offline rows: the fresh ones plus a perturbation whose size varies from token to token
+        g = W.standard_normal(L_d, 600 + l).float().abs().view(L_d, 1, 1).to(dev)
+        kc = (kf[:L_d].float() + 0.2 * g * _normal((L_d, Hkv, 128), 502 + 10 * l).to(dev).float()).to(torch.bfloat16)
+        vc = (vf[:L_d].float() + 0.1 * g * _normal((L_d, Hkv, 128), 503 + 10 * l).to(dev).float()).to(torch.bfloat16)
+        layers.append((kf, vf, kc, vc))
+    p = api.make_params(L_d, L_q, r, Hq, Hkv)
+    k = api.daf_num_important(L_d, r)
+    ws = api.alloc_workspace(p)
+    # the layer being processed
+    q_fresh, k_fresh, v_fresh = _normal((N, Hq, 128), 700).to(dev), _normal((N, Hkv, 128), 701).to(dev), _normal((N, Hkv, 128), 702).to(dev)
+    k_cached, v_cached = _normal((L_d, Hkv, 128), 703).to(dev), _normal((L_d, Hkv, 128), 704).to(dev)
+    kv_k = torch.cat([k_cached, torch.zeros(L_q, Hkv, 128, dtype=torch.bfloat16, device=dev)])
+    kv_v = torch.cat([v_cached, torch.zeros(L_q, Hkv, 128, dtype=torch.bfloat16, device=dev)])
+    idx_out = torch.full((max(k, 1),), -1, dtype=torch.int32, device=dev)
+    qp = torch.zeros(max(k, 1), Hq, 128, dtype=torch.bfloat16, device=dev)
+    kp = torch.zeros(max(k, 1), Hkv, 128, dtype=torch.bfloat16, device=dev)
+    vp = torch.zeros_like(kp)
+    sums = torch.full((L_d + 4,), -1.0, dtype=torch.float32, device=dev)
+    _ok(api.daf_select_from_kv(p, [x[0] for x in layers], [x[1] for x in layers], [x[2] for x in layers],
+                               [x[3] for x in layers], q_fresh, k_fresh, v_fresh, kv_k, kv_v, idx_out, qp, kp, vp, sums, ws),
+        ws, "daf_select_from_kv")
+    assert torch.all(sums[L_d:] == -1.0), "wrote past the end of the sums"
+    got = sums[:L_d].cpu().numpy()
+    # (1) per-layer signals from the stand-alone kernel, added in ascending order in fp32
+    rows = []
+    for kf, vf, kc, vc in layers:
+        row = torch.zeros(L_d, dtype=torch.float32, device=dev)
+        api.check(api.daf_deviation_scores(p, kf, vf, kc, vc, row), "daf_deviation_scores")
+        rows.append(row.cpu().numpy())
+    acc = rows[0].copy()
+    for row in rows[1:]:
+        acc = (acc + row).astype(np.float32)
+    assert np.array_equal(got.view(np.uint32), acc.view(np.uint32)), "aggregate differs from the per-layer rows added in order"
+    # (2) against the oracle's fp64 signal
+    ref = sum(oracle.deviation_scores(_f(kf), _f(vf), _f(kc), _f(vc), L_d) for kf, vf, kc, vc in layers)
+    np.testing.assert_allclose(got.astype(np.float64), ref, rtol=2e-5, atol=0)
+    # (3) positions: the oracle's selection on the same fp32 sums, bit-exact; and the oracle's aggregation of
+    #     the per-layer rows gives the same sums
+    assert np.array_equal(oracle.aggregate(np.stack(rows)).view(np.uint32), got.view(np.uint32))
+    idx = oracle.select(got[None, :], k)
+    assert np.array_equal(idx_out[:k].cpu().numpy(), idx)
+    # (4) gather and hybrid cache, byte-exact
+    it = torch.from_numpy(idx).long().to(dev)
+    assert torch.equal(qp[:k], q_fresh[it]) and torch.equal(kp[:k], k_fresh[it]) and torch.equal(vp[:k], v_fresh[it])
+    exp_k = torch.cat([k_cached, k_fresh[L_d:]]); exp_k[it] = k_fresh[it]
+    exp_v = torch.cat([v_cached, v_fresh[L_d:]]); exp_v[it] = v_fresh[it]
+    assert torch.equal(kv_k, exp_k) and torch.equal(kv_v, exp_v)
+
+
 # --------------------------------------------------------------------------- gather / hybrid cache / fusion
 @pytest.mark.parametrize("name,Hq,Hkv,L_d,L_q,r", [("c0", 28, 4, 1024, 32, 0.15), ("x", 8, 8, 300, 7, 0.4),
                                                   ("y", 40, 8, 513, 0, 0.2), ("z", 4, 1, 64, 5, 0.0)])
