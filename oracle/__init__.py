@@ -17,6 +17,8 @@ from .daf_oracle import (  # noqa: F401
     fuse,
     deviation_scores,
     blend_attn,
+    e4m3_decode,
+    dequant_fp8,
     daf_layer,
     num_threads,
 )

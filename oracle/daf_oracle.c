@@ -31,6 +31,8 @@
  * hand-worked rational example in tests/golden/), against a brute-force masked
  * N x N attention over the concatenated context, and the selection against a
  * library stable argsort and an O(L_d^2) rank count.
+ * The fp8 decode is pinned against a library conversion of all 256 byte values and stated values of the
+ * format (largest finite 448, smallest subnormal 2^-9), the expansion by "scale 1 == widening".
  * Parity unpinned: the *formula* of the per-layer deviation signal (the paper names
  * the signal but gives no formula; daf_oracle_deviation_scores states the reading
  * taken).  The selection rule applied to given scores is pinned, and so is the
@@ -255,6 +257,55 @@ void daf_oracle_deviation_scores(const float *k_fresh, const float *v_fresh, con
         }
         s_out[i] = acc;
     }
+}
+
+/* ------------------------------------------------- offline cache stored in fp8
+ * (Preliminary Results, Limitations: the storage of the offline KV caches is the
+ * industrial bottleneck.)  Reading taken for the stored-in-fp8 variant: an offline
+ * K or V element is one byte in the 8-bit floating-point format with 1 sign bit,
+ * 4 exponent bits (bias 7) and 3 mantissa bits, no infinities, and the single
+ * NaN pattern S.1111.111 ("e4m3"); every KV head has one fp32 scale.  The value
+ * the attention sees is   bf16( scale * decode(byte) )   with the product taken in
+ * fp32 and both roundings to nearest-even: the cache is expanded to the bf16
+ * working precision of the rest of the path, after which nothing differs from the
+ * bf16 path.  With scale = 1 the expansion is exact (every e4m3 value is a bf16
+ * value).
+ */
+float daf_oracle_e4m3_decode(uint8_t byte)
+{
+    const int sign = byte >> 7, e = (byte >> 3) & 0xF, m = byte & 0x7;
+    float v;
+    if (e == 0xF && m == 0x7) return NAN;
+    if (e == 0) v = ldexpf((float)m, -9);                 /* subnormal: m/8 * 2^-6 */
+    else v = ldexpf(1.0f + (float)m / 8.0f, e - 7);
+    return sign ? -v : v;
+}
+
+static float round_to_bf16(float x)
+{
+    uint32_t u;
+    memcpy(&u, &x, 4);
+    if ((u & 0x7FFFFFFFu) > 0x7F800000u) return x;        /* NaN stays NaN */
+    u += 0x7FFFu + ((u >> 16) & 1u);                      /* round to nearest, ties to even */
+    u &= 0xFFFF0000u;
+    memcpy(&x, &u, 4);
+    return x;
+}
+
+/* bytes: [tokens, heads, D] e4m3; scale: [heads] or NULL (all 1); out: fp32 [tokens, heads, D]
+ * holding bf16-representable values. */
+void daf_oracle_dequant_fp8(const uint8_t *bytes, const float *scale, int64_t tokens, int32_t heads, int32_t D,
+                            float *out)
+{
+    for (int64_t t = 0; t < tokens; ++t)
+        for (int32_t h = 0; h < heads; ++h) {
+            const float s = scale ? scale[h] : 1.0f;
+            for (int32_t d = 0; d < D; ++d) {
+                const int64_t i = (t * heads + h) * D + d;
+                const float prod = s * daf_oracle_e4m3_decode(bytes[i]);    /* fp32 product, rounded once */
+                out[i] = round_to_bf16(prod);
+            }
+        }
 }
 
 /* State fusion (Methods, item 3).  mode 0: compact concatenation, important rows

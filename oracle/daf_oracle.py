@@ -62,6 +62,10 @@ def _load():
         lib.daf_oracle_deviation_scores.argtypes = [c_f, c_f, c_f, c_f, i32, i64, c_d]
         lib.daf_oracle_fuse.restype = None
         lib.daf_oracle_fuse.argtypes = [c_d, c_d, c_i, i32, i32, i32, i64, i32, c_d, c_i]
+        lib.daf_oracle_e4m3_decode.restype = ctypes.c_float
+        lib.daf_oracle_e4m3_decode.argtypes = [ctypes.c_uint8]
+        lib.daf_oracle_dequant_fp8.restype = None
+        lib.daf_oracle_dequant_fp8.argtypes = [ctypes.POINTER(ctypes.c_uint8), c_f, i64, i32, i32, c_f]
         lib.daf_oracle_num_threads.restype = i32
         lib.daf_oracle_num_threads.argtypes = []
         _lib = lib
@@ -209,6 +213,23 @@ def deviation_scores(k_fresh, v_fresh, k_cached, v_cached, L_d: int) -> np.ndarr
     out = np.zeros(L_d, dtype=np.float64)
     _load().daf_oracle_deviation_scores(_p(kf, ctypes.c_float), _p(vf, ctypes.c_float), _p(kc, ctypes.c_float),
                                         _p(vc, ctypes.c_float), int(L_d), row_elems, _p(out, ctypes.c_double))
+    return out
+
+
+def e4m3_decode(byte: int) -> float:
+    """Value of one byte of the 8-bit floating-point format (1 sign, 4 exponent, 3 mantissa bits; no infinities)."""
+    return float(_load().daf_oracle_e4m3_decode(int(byte) & 0xFF))
+
+
+def dequant_fp8(cache_bytes, scale=None) -> np.ndarray:
+    """uint8 [tokens, heads, D] e4m3 bytes (+ optional fp32 [heads] scales) -> fp32 [tokens, heads, D] holding
+    bf16(scale * decode(byte)): the offline cache as the rest of the path sees it."""
+    b = np.ascontiguousarray(cache_bytes, dtype=np.uint8)
+    tokens, heads, D = b.shape
+    sc = None if scale is None else _f32(scale)
+    out = np.empty(b.shape, dtype=np.float32)
+    _load().daf_oracle_dequant_fp8(b.ctypes.data_as(ctypes.POINTER(ctypes.c_uint8)), _p(sc, ctypes.c_float), tokens, heads, D,
+                                   _p(out, ctypes.c_float))
     return out
 
 
