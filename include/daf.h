@@ -247,6 +247,28 @@ int daf_layer(const daf_params* p, const float* scores, int32_t n_sig, const int
               void* hidden, int32_t* row_pos_out,
               void* workspace, size_t workspace_bytes, void* stream);
 
+/* Offline cache stored in fp8 (no counterpart in the paper beyond its remark, under Limitations, that storing the
+ * offline KV caches is the bottleneck at scale).  The document rows of a layer's offline cache are kept as one byte per
+ * element in the 8-bit floating-point format with 1 sign, 4 exponent (bias 7) and 3 mantissa bits (no infinities,
+ * S.1111.111 = NaN), with one fp32 scale per KV head; only the layer being processed is expanded to bf16:
+ *     kv[t, h, d] = bf16( scale[h] * value(byte[t, h, d]) )      fp32 product, both roundings to nearest-even
+ * into rows [0, L_d) of the hybrid-cache buffer, after which the path is the bf16 path: the important rows are
+ * overwritten with fresh bf16 K/V and the question rows appended, exactly as in daf_select.  The fp8 cache itself
+ * is read-only, so a resident offline cache costs half the bytes and one [N, n_kv_heads, 128] bf16 buffer pair is
+ * reused from layer to layer.
+ *   k_cached_fp8, v_cached_fp8  [L_d, n_kv_heads, 128] bytes (device)
+ *   k_scale, v_scale            fp32 [n_kv_heads] (device), or NULL for 1
+ *   kv_k, kv_v                  [N, n_kv_heads, 128] bf16 OUT
+ * daf_layer_fp8 = this expansion followed by daf_layer (same remaining arguments); the selection kernel runs
+ * beside the expansion, which it does not depend on. */
+int daf_expand_fp8_cache(const daf_params* p, const void* k_cached_fp8, const void* v_cached_fp8, const float* k_scale,
+                         const float* v_scale, void* kv_k, void* kv_v, void* stream);
+int daf_layer_fp8(const daf_params* p, const float* scores, int32_t n_sig, const int32_t* idx_in,
+                  const void* q_fresh, const void* k_fresh, const void* v_fresh,
+                  const void* k_cached_fp8, const void* v_cached_fp8, const float* k_scale, const float* v_scale,
+                  void* kv_k, void* kv_v, int32_t* idx_out, void* q_pack, void* k_pack, void* v_pack,
+                  void* hidden, int32_t* row_pos_out, void* workspace, size_t workspace_bytes, void* stream);
+
 /* The same layer for callers whose tensors live in HOST memory (pinned memory
  * makes the copies asynchronous).  h_* are host pointers; every copy to and from
  * the device is part of the call.  `arena` is caller-owned device memory of at

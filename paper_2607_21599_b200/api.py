@@ -32,7 +32,7 @@ EXPORTS = [
     "daf_layer_host", "daf_poll_status", "daf_strerror", "daf_last_cuda_error", "daf_launch_count",
     "daf_qd_attn_static", "daf_qd_attn_static_max_bytes", "daf_deviation_scores", "daf_blend_attn",
     "daf_imp_qd_attn", "daf_selftest_bounded_wait", "daf_qd_attn_static_poll_status",
-    "daf_imp_qd_attn_launches", "daf_select_from_kv",
+    "daf_imp_qd_attn_launches", "daf_select_from_kv", "daf_expand_fp8_cache", "daf_layer_fp8",
 ]
 
 
@@ -109,6 +109,10 @@ def lib() -> ctypes.CDLL:
         L.daf_full_causal_attn.argtypes = [pp, i32, vp, vp, vp, vp, vp, vp, sz, vp]
         L.daf_layer.restype = ctypes.c_int
         L.daf_layer.argtypes = [pp, vp, i32, vp] + [vp] * 3 + [vp] * 2 + [vp] * 4 + [vp, vp] + [vp, sz, vp]
+        L.daf_layer_fp8.restype = ctypes.c_int
+        L.daf_layer_fp8.argtypes = [pp, vp, i32, vp] + [vp] * 3 + [vp] * 4 + [vp] * 2 + [vp] * 4 + [vp, vp] + [vp, sz, vp]
+        L.daf_expand_fp8_cache.restype = ctypes.c_int
+        L.daf_expand_fp8_cache.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp]
         L.daf_layer_host_arena_bytes.restype = sz
         L.daf_layer_host_arena_bytes.argtypes = [pp]
         L.daf_layer_host.restype = ctypes.c_int
@@ -278,6 +282,19 @@ def daf_layer(p, scores, n_sig, idx_in, q_fresh, k_fresh, v_fresh, kv_k, kv_v, i
                            _ptr(v_fresh), _ptr(kv_k), _ptr(kv_v), _ptr(idx_out), _ptr(q_pack), _ptr(k_pack),
                            _ptr(v_pack), _ptr(hidden), _ptr(row_pos_out), _ptr(workspace), _nbytes(workspace),
                            _stream(stream))
+
+
+def daf_layer_fp8(p, scores, n_sig, idx_in, q_fresh, k_fresh, v_fresh, k_cached_fp8, v_cached_fp8, k_scale, v_scale, kv_k, kv_v,
+                  idx_out, q_pack, k_pack, v_pack, hidden, row_pos_out, workspace, stream=None) -> int:
+    return lib().daf_layer_fp8(ctypes.byref(p), _ptr(scores), int(n_sig), _ptr(idx_in), _ptr(q_fresh), _ptr(k_fresh),
+                               _ptr(v_fresh), _ptr(k_cached_fp8), _ptr(v_cached_fp8), _ptr(k_scale), _ptr(v_scale),
+                               _ptr(kv_k), _ptr(kv_v), _ptr(idx_out), _ptr(q_pack), _ptr(k_pack), _ptr(v_pack), _ptr(hidden),
+                               _ptr(row_pos_out), _ptr(workspace), _nbytes(workspace), _stream(stream))
+
+
+def daf_expand_fp8_cache(p, k_cached_fp8, v_cached_fp8, k_scale, v_scale, kv_k, kv_v, stream=None) -> int:
+    return lib().daf_expand_fp8_cache(ctypes.byref(p), _ptr(k_cached_fp8), _ptr(v_cached_fp8), _ptr(k_scale), _ptr(v_scale),
+                                      _ptr(kv_k), _ptr(kv_v), _stream(stream))
 
 
 def daf_layer_host_arena_bytes(p: daf_params) -> int:

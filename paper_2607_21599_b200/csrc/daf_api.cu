@@ -94,7 +94,7 @@ static int carve_workspace(const ResolvedParams& rp, void* workspace, size_t byt
 static int do_select(const ResolvedParams& rp, const float* scores, int32_t n_sig, const int32_t* idx_in,
                      const void* q_fresh, const void* k_fresh, const void* v_fresh, void* kv_k, void* kv_v,
                      int32_t* idx_out, void* q_pack, void* k_pack, void* v_pack, const Workspace& ws, cudaStream_t st,
-                     bool scores_from_previous_kernel = false) {
+                     bool scores_from_previous_kernel = false, bool beside_previous_kernel = false) {
     if (scores != nullptr && n_sig < 1) return DAF_ERR_INVALID_ARG;
     if (rp.k > 0) {
         if (scores == nullptr && idx_in == nullptr) return DAF_ERR_INVALID_ARG;
@@ -108,7 +108,7 @@ static int do_select(const ResolvedParams& rp, const float* scores, int32_t n_si
     for (const void* ptr : ptrs)
         if (ptr != nullptr && !aligned16(ptr)) return DAF_ERR_ALIGNMENT;
     return launch_select(rp, scores, n_sig, idx_in, q_fresh, k_fresh, v_fresh, kv_k, kv_v, idx_out, q_pack, k_pack,
-                         v_pack, ws.status, ws.select_scratch, st, scores_from_previous_kernel);
+                         v_pack, ws.status, ws.select_scratch, st, scores_from_previous_kernel, beside_previous_kernel);
 }
 
 static int check_out(const void* out, int64_t stride_bytes, int Hq) {
@@ -301,17 +301,27 @@ int daf_full_causal_attn(const daf_params* p, int32_t n_tokens, const void* q, c
                             (cudaStream_t)stream);
 }
 
-int daf_layer(const daf_params* p, const float* scores, int32_t n_sig, const int32_t* idx_in,
-              const void* q_fresh, const void* k_fresh, const void* v_fresh, void* kv_k, void* kv_v,
-              int32_t* idx_out, void* q_pack, void* k_pack, void* v_pack,
-              void* hidden, int32_t* row_pos_out,
-              void* workspace, size_t workspace_bytes_, void* stream) {
+}  // extern "C"
+
+namespace {
+// Offline cache of one layer kept in fp8 (daf_layer_fp8): expanded into kv_k / kv_v ahead of everything else.
+struct Fp8Cache { const void* k8; const void* v8; const float* k_scale; const float* v_scale; };
+
+int layer_impl(const daf_params* p, const Fp8Cache* fp8, const float* scores, int32_t n_sig, const int32_t* idx_in,
+               const void* q_fresh, const void* k_fresh, const void* v_fresh, void* kv_k, void* kv_v,
+               int32_t* idx_out, void* q_pack, void* k_pack, void* v_pack,
+               void* hidden, int32_t* row_pos_out,
+               void* workspace, size_t workspace_bytes_, void* stream) {
     ResolvedParams rp;
     if (int rc = resolve_params(p, &rp)) return rc;
     Workspace ws;
     if (int rc = carve_workspace(rp, workspace, workspace_bytes_, &ws)) return rc;
     cudaStream_t st = (cudaStream_t)stream;
     if (rp.k + rp.L_q == 0) return DAF_OK;
+    if (fp8 != nullptr) {
+        if (rp.L_d > 0 && (!fp8->k8 || !fp8->v8 || !kv_k || !kv_v)) return DAF_ERR_INVALID_ARG;
+        if (!aligned16(fp8->k8) || !aligned16(fp8->v8) || !aligned16(kv_k) || !aligned16(kv_v)) return DAF_ERR_ALIGNMENT;
+    }
     if (rp.k > 0 && idx_out == nullptr) return DAF_ERR_INVALID_ARG;
     if (rp.k > 0 && rp.L_q == 0 && q_pack == nullptr) return DAF_ERR_INVALID_ARG;   // only the joint launch reads Q in place
     // the question rows are read from q_fresh even when nothing is selected (r = 0)
@@ -320,8 +330,13 @@ int daf_layer(const daf_params* p, const float* scores, int32_t n_sig, const int
     if (q_fresh != nullptr && !aligned16(q_fresh)) return DAF_ERR_ALIGNMENT;
     const int64_t row_bytes = (int64_t)rp.Hq * 256;
     if (int rc = check_out(hidden, row_bytes, rp.Hq)) return rc;
+    // An fp8 offline cache is expanded into the hybrid-cache buffer first.  The selection does not depend on it,
+    // so the selection kernel is launched beside it; the gather kernel (which overwrites the important rows of
+    // the expanded cache) runs behind both.
+    if (fp8 != nullptr)
+        if (int rc = launch_expand_fp8(rp, fp8->k8, fp8->v8, fp8->k_scale, fp8->v_scale, kv_k, kv_v, st)) return rc;
     if (int rc = do_select(rp, scores, n_sig, idx_in, q_fresh, k_fresh, v_fresh, kv_k, kv_v, idx_out, q_pack, k_pack,
-                           v_pack, ws, st)) return rc;
+                           v_pack, ws, st, false, /*beside_previous_kernel=*/fp8 != nullptr && rp.L_d > 0)) return rc;
     char* h = reinterpret_cast<char*>(hidden);
     // State fusion is done by the attention epilogues: each stage writes its final rows.  When both
     // stages have rows they run as one list of work items in one launch, right behind the gather
@@ -346,6 +361,38 @@ int daf_layer(const daf_params* p, const float* scores, int32_t n_sig, const int
         if (int rc = launch_fuse(rp, idx_out, nullptr, nullptr, nullptr, row_pos_out, st)) return rc;
     }
     return DAF_OK;
+}
+}  // namespace
+
+extern "C" {
+
+int daf_layer(const daf_params* p, const float* scores, int32_t n_sig, const int32_t* idx_in,
+              const void* q_fresh, const void* k_fresh, const void* v_fresh, void* kv_k, void* kv_v,
+              int32_t* idx_out, void* q_pack, void* k_pack, void* v_pack,
+              void* hidden, int32_t* row_pos_out,
+              void* workspace, size_t workspace_bytes_, void* stream) {
+    return layer_impl(p, nullptr, scores, n_sig, idx_in, q_fresh, k_fresh, v_fresh, kv_k, kv_v, idx_out, q_pack, k_pack, v_pack,
+                      hidden, row_pos_out, workspace, workspace_bytes_, stream);
+}
+
+int daf_layer_fp8(const daf_params* p, const float* scores, int32_t n_sig, const int32_t* idx_in,
+                  const void* q_fresh, const void* k_fresh, const void* v_fresh,
+                  const void* k_cached_fp8, const void* v_cached_fp8, const float* k_scale, const float* v_scale,
+                  void* kv_k, void* kv_v, int32_t* idx_out, void* q_pack, void* k_pack, void* v_pack,
+                  void* hidden, int32_t* row_pos_out, void* workspace, size_t workspace_bytes_, void* stream) {
+    const Fp8Cache fp8{k_cached_fp8, v_cached_fp8, k_scale, v_scale};
+    return layer_impl(p, &fp8, scores, n_sig, idx_in, q_fresh, k_fresh, v_fresh, kv_k, kv_v, idx_out, q_pack, k_pack, v_pack,
+                      hidden, row_pos_out, workspace, workspace_bytes_, stream);
+}
+
+int daf_expand_fp8_cache(const daf_params* p, const void* k_cached_fp8, const void* v_cached_fp8, const float* k_scale,
+                         const float* v_scale, void* kv_k, void* kv_v, void* stream) {
+    ResolvedParams rp;
+    if (int rc = resolve_params(p, &rp)) return rc;
+    if (rp.L_d == 0) return DAF_OK;
+    if (!k_cached_fp8 || !v_cached_fp8 || !kv_k || !kv_v) return DAF_ERR_INVALID_ARG;
+    if (!aligned16(k_cached_fp8) || !aligned16(v_cached_fp8) || !aligned16(kv_k) || !aligned16(kv_v)) return DAF_ERR_ALIGNMENT;
+    return launch_expand_fp8(rp, k_cached_fp8, v_cached_fp8, k_scale, v_scale, kv_k, kv_v, (cudaStream_t)stream);
 }
 
 // ---- host-buffer form

@@ -40,7 +40,10 @@ size_t select_scratch_bytes(int L_d);
 int launch_select(const ResolvedParams& rp, const float* scores, int n_sig, const int32_t* idx_in,
                   const void* q_fresh, const void* k_fresh, const void* v_fresh, void* kv_k, void* kv_v,
                   int32_t* idx_out, void* q_pack, void* k_pack, void* v_pack,
-                  DeviceStatus* status, void* scratch, cudaStream_t stream, bool scores_from_previous_kernel = false);
+                  DeviceStatus* status, void* scratch, cudaStream_t stream, bool scores_from_previous_kernel = false,
+                  bool beside_previous_kernel = false);
+int launch_expand_fp8(const ResolvedParams& rp, const void* k8, const void* v8, const float* k_scale, const float* v_scale,
+                      void* kv_k, void* kv_v, cudaStream_t stream);
 constexpr int kMaxSignalLayersHost = 8;
 int launch_deviation_sum(const ResolvedParams& rp, int n_sig, const void* const* k_fresh, const void* const* v_fresh,
                          const void* const* k_cached, const void* const* v_cached, float* sums, cudaStream_t stream);

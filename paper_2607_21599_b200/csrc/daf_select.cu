@@ -5,6 +5,7 @@
 // and launch latency, not by arithmetic, so they are plain coalesced 16-byte
 // kernels with no tensor-core work.
 #include <cooperative_groups.h>
+#include <cuda_fp8.h>
 
 #include <atomic>
 
@@ -62,11 +63,14 @@ struct SelShared {
 
 __global__ void __cluster_dims__(kSelCluster, 1, 1) __launch_bounds__(kSelThreads, 1)
 select_topk_kernel(const float* __restrict__ scores, int n_sig, int L_d, int k,
-                   uint32_t* __restrict__ gkeys, int32_t* __restrict__ idx_out) {
+                   uint32_t* __restrict__ gkeys, int32_t* __restrict__ idx_out, int wait_at_end) {
     namespace cg = cooperative_groups;
     cg::cluster_group cluster = cg::this_cluster();
     DAF_KT_BEGIN(0);
-    pdl_wait();                // the scores may come from the signal kernel launched just before
+    // The kernel launched just before this one is either the one that wrote the scores (wait for it now) or one
+    // this kernel does not depend on (the expansion of an fp8 cache: run beside it and wait for it only at the
+    // end, so that the kernel behind this one finds both finished).
+    if (!wait_at_end) pdl_wait();
     pdl_launch_dependents();   // the gather kernel may start launching; it waits for this grid before reading idx
     extern __shared__ __align__(16) unsigned char sel_smem[];
     SelShared* sh = reinterpret_cast<SelShared*>(sel_smem);
@@ -207,6 +211,7 @@ select_topk_kernel(const float* __restrict__ scores, int n_sig, int L_d, int k,
         }
     }
     cluster.sync();   // no CTA may retire while a peer can still read its shared memory
+    if (wait_at_end) pdl_wait();
     DAF_KT_END(0);
 }
 
@@ -285,14 +290,15 @@ __device__ __forceinline__ void pick_bin(Sel1Shared* sh, int n_bins, int per) {
 }
 
 __global__ void __launch_bounds__(kSel1Threads, 1)
-select_topk_cta_kernel(const float* __restrict__ scores, int n_sig, int L_d, int k, int32_t* __restrict__ idx_out) {
+select_topk_cta_kernel(const float* __restrict__ scores, int n_sig, int L_d, int k, int32_t* __restrict__ idx_out,
+                       int wait_at_end) {
     extern __shared__ __align__(16) unsigned char sel_smem[];
     Sel1Shared* sh = reinterpret_cast<Sel1Shared*>(sel_smem);
     uint32_t* keys = reinterpret_cast<uint32_t*>(sel_smem + sizeof(Sel1Shared));
     uint32_t* cand = keys + padded(L_d);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     DAF_KT_BEGIN(0);
-    pdl_wait();                // the scores may come from the signal kernel launched just before
+    if (!wait_at_end) pdl_wait();   // see select_topk_kernel
     pdl_launch_dependents();   // the gather kernel may start launching; it waits for this grid before reading idx
 
     // aggregate the signal rows in ascending row order (fp32 adds, no fusing), build keys, find their range
@@ -409,6 +415,7 @@ select_topk_cta_kernel(const float* __restrict__ scores, int n_sig, int L_d, int
             if (take) idx_out[pos++] = i;
         }
     }
+    if (wait_at_end) pdl_wait();
     DAF_KT_END(0);
 }
 
@@ -590,7 +597,12 @@ static size_t select_smem_bytes(int L_d) {
 int launch_select(const ResolvedParams& rp, const float* scores, int n_sig, const int32_t* idx_in,
                   const void* q_fresh, const void* k_fresh, const void* v_fresh, void* kv_k, void* kv_v,
                   int32_t* idx_out, void* q_pack, void* k_pack, void* v_pack,
-                  DeviceStatus* status, void* scratch, cudaStream_t stream, bool scores_from_previous_kernel) {
+                  DeviceStatus* status, void* scratch, cudaStream_t stream, bool scores_from_previous_kernel,
+                  bool beside_previous_kernel) {
+    // beside_previous_kernel: the kernel launched just before (the fp8 cache expansion) is independent of the
+    // selection; the selection kernel starts while it runs and only waits for it before it retires
+    const bool dependent = scores_from_previous_kernel || beside_previous_kernel;
+    const int wait_at_end = beside_previous_kernel ? 1 : 0;
     const int32_t* idx_src = idx_in;
     if (scores != nullptr && rp.L_d > 0 && rp.k > 0) {
         static std::atomic<bool> attr_done[64];   // per device; a concurrent first call sets the same values
@@ -608,13 +620,13 @@ int launch_select(const ResolvedParams& rp, const float* scores, int n_sig, cons
         if (rp.L_d <= g_sel1_max_keys) {
             const size_t smem1 = sizeof(Sel1Shared) + ((size_t)padded(rp.L_d) + rp.L_d) * sizeof(uint32_t);   // keys and candidate list
             const cudaError_t e = launch_kernel(select_topk_cta_kernel, dim3(1), dim3(kSel1Threads), smem1, stream,
-                                                scores_from_previous_kernel, scores, n_sig, rp.L_d, rp.k, idx_out);
+                                                dependent, scores, n_sig, rp.L_d, rp.k, idx_out, wait_at_end);
             if (e != cudaSuccess) { set_cuda_error(e); return DAF_ERR_CUDA; }
         } else {
             const size_t smem = select_smem_bytes(rp.L_d);
             const cudaError_t e = launch_kernel(select_topk_kernel, dim3(kSelCluster), dim3(kSelThreads), smem, stream,
-                                                scores_from_previous_kernel, scores, n_sig, rp.L_d, rp.k,
-                                                reinterpret_cast<uint32_t*>(scratch), idx_out);
+                                                dependent, scores, n_sig, rp.L_d, rp.k,
+                                                reinterpret_cast<uint32_t*>(scratch), idx_out, wait_at_end);
             if (e != cudaSuccess) { set_cuda_error(e); return DAF_ERR_CUDA; }
         }
         count_launch();
@@ -679,6 +691,61 @@ int launch_deviation_sum(const ResolvedParams& rp, int n_sig, const void* const*
     const int max_blocks = 148 * 8;
     if (blocks > max_blocks) blocks = max_blocks;
     deviation_sum_kernel<<<blocks, warps * 32, 0, stream>>>(layers, rp.L_d, rp.Hkv * 16, sums);
+    count_launch();
+    return check_launch();
+}
+
+// ------------------------------------------------ offline cache stored in fp8
+// Expands the document rows of an offline cache kept as 8-bit floating point (1 sign, 4 exponent, 3 mantissa
+// bits, bias 7, no infinities) into the bf16 hybrid-cache buffer: element = bf16(scale[head] * value), the product in
+// fp32, both roundings to nearest-even.  A streaming pass (1 byte read, 2 written per element); each thread
+// takes 16 elements.
+__device__ __forceinline__ float mul_rn_keep_subnormals(float a, float b) {
+    float d;
+    asm("mul.rn.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
+    return d;
+}
+__device__ __forceinline__ uint4 expand8(uint2 bytes, float scale) {
+    const __nv_fp8x2_storage_t* pr = reinterpret_cast<const __nv_fp8x2_storage_t*>(&bytes);
+    uint32_t w[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const __half2_raw h2 = __nv_cvt_fp8x2_to_halfraw2(pr[i], __NV_E4M3);    // exact: every value is an fp16 value
+        const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&h2));
+        w[i] = pack_bf16(mul_rn_keep_subnormals(f.x, scale), mul_rn_keep_subnormals(f.y, scale));
+    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+__global__ void __launch_bounds__(256)
+expand_fp8_cache_kernel(const uint4* __restrict__ k8, const uint4* __restrict__ v8, const float* __restrict__ k_scale,
+                        const float* __restrict__ v_scale, uint4* __restrict__ kv_k, uint4* __restrict__ kv_v,
+                        long long n_chunks, int Hkv) {
+    pdl_launch_dependents();   // the selection kernel does not depend on this grid and may run beside it
+    // chunk c = 16 consecutive elements; a head is 128 elements = 8 chunks
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long c = (long long)blockIdx.x * blockDim.x + threadIdx.x; c < 2 * n_chunks; c += stride) {
+        const bool is_v = c >= n_chunks;
+        const long long cc = is_v ? c - n_chunks : c;
+        const int head = (int)((cc >> 3) % Hkv);
+        const float* sc = is_v ? v_scale : k_scale;
+        const float scale = sc != nullptr ? __ldg(sc + head) : 1.0f;
+        const uint4 in = __ldcs((is_v ? v8 : k8) + cc);
+        uint4* out = (is_v ? kv_v : kv_k) + 2 * cc;
+        out[0] = expand8(make_uint2(in.x, in.y), scale);
+        out[1] = expand8(make_uint2(in.z, in.w), scale);
+    }
+}
+
+int launch_expand_fp8(const ResolvedParams& rp, const void* k8, const void* v8, const float* k_scale, const float* v_scale,
+                      void* kv_k, void* kv_v, cudaStream_t stream) {
+    const long long n_chunks = (long long)rp.L_d * rp.Hkv * 8;     // 16-element chunks per tensor
+    if (n_chunks == 0) return DAF_OK;
+    long long blocks = (2 * n_chunks + 255) / 256;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    expand_fp8_cache_kernel<<<(unsigned)blocks, 256, 0, stream>>>(
+        reinterpret_cast<const uint4*>(k8), reinterpret_cast<const uint4*>(v8), k_scale, v_scale,
+        reinterpret_cast<uint4*>(kv_k), reinterpret_cast<uint4*>(kv_v), n_chunks, rp.Hkv);
     count_launch();
     return check_launch();
 }

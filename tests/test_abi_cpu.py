@@ -19,7 +19,7 @@ def lib():
 def test_header_symbols_are_exported(lib, repo_root):
     header = open(os.path.join(repo_root, "include", "daf.h")).read()
     header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
-    declared = set(re.findall(r"\b(daf_[a-z_]+)\s*\(", header))
+    declared = set(re.findall(r"\b(daf_[a-z0-9_]+)\s*\(", header))
     assert declared, "no declarations found"
     assert declared == set(api.EXPORTS)
     for name in declared:
