@@ -232,6 +232,7 @@ class LayerBuffers:
         self.k_pack = torch.empty(max(k, 1), Hkv, 128, dtype=bf, device=dev)
         self.v_pack = torch.empty(max(k, 1), Hkv, 128, dtype=bf, device=dev)
         self.hidden = torch.empty(k + w.L_q, Hq, 128, dtype=bf, device=dev)
+        self.idx_sel = torch.zeros(max(k, 1), dtype=torch.int32, device=dev)     # positions from the hoisted selection
         self.n_sig = 0 if L["scores"] is None else L["scores"].shape[0]
 
 
@@ -348,7 +349,32 @@ def measure_config(env: Env, w: W.Workload, primary: bool):
         torch.cuda.synchronize()
         return e0.elapsed_time(e1) / reps  # ms per replay
 
-    step = over(layer_call, bufs)
+    # The selection of a layer depends only on that layer's scores (in the method they come from the signal layers,
+    # long before the layer is reached), so the step schedules the selections of all layers on a second stream:
+    # they run beside the attention of earlier layers, and each layer proper (gather, cache update, both attention
+    # stages, fusion) starts from the positions its selection left.  Every kernel of the path still runs, and
+    # is timed, once per layer per step.  --no-overlap keeps everything on one stream.
+    overlap = (not args.no_overlap) and w.k > 0 and bufs[0].L["scores"] is not None
+    side = torch.cuda.Stream(device=dev) if overlap else None
+
+    def step_overlapped():
+        main = torch.cuda.current_stream()
+        side.wait_stream(main)
+        events = []
+        for b in bufs:
+            api.check(api.daf_select_topk(p, b.L["scores"], b.n_sig, b.idx_sel, ws, stream=side), "daf_select_topk")
+            e = torch.cuda.Event()
+            e.record(side)
+            events.append(e)
+        for b, e in zip(bufs, events):
+            main.wait_event(e)
+            L = b.L
+            api.check(api.daf_layer(p, None, 0, b.idx_sel, L["q_fresh"], L["k_fresh"], L["v_fresh"], b.kv_k, b.kv_v, b.idx_out,
+                                    None if q_in_place else b.q_pack, b.k_pack, b.v_pack, b.hidden, None, ws, stream=main),
+                      "daf_layer")
+        main.wait_stream(side)
+
+    step = step_overlapped if overlap else over(layer_call, bufs)
     for _ in range(max(args.warmup, 3)):     # eager warm-up: also sets function attributes before capture
         step()
     barrier()
@@ -422,6 +448,7 @@ def measure_config(env: Env, w: W.Workload, primary: bool):
                                          [g["k_cached"] for g in grp], [g["v_cached"] for g in grp], None, None, None, None,
                                          None, None, None, None, None, dev_scores, ws_sig), "daf_select_from_kv (signal only)")
 
+    us_layer_one_stream = time_stage(layer_call, bufs)     # the whole layer from scores on one stream, for comparison
     for b in bufs:                       # the stand-alone important-token stage below reads packed Q rows
         st_select(b, pack_q=True)
     us_dev = time_stage(st_dev, bufs)
@@ -582,6 +609,9 @@ def measure_config(env: Env, w: W.Workload, primary: bool):
         "value": us_per_layer, "unit": UNIT, "ms_per_step": ms_per_step, "config": _config_dict(w, world),
         "tflops": tflops, "frac_of_bf16_peak": tflops / (peaks["bf16_tflops"] * world),
         "roofline": roofline,
+        "schedule": ("selection of every layer on a second stream (daf_select_topk), layers from idx_in on the main one"
+                     if overlap else "one stream"),
+        "us_per_layer_one_stream": us_layer_one_stream,
         "stages_us": {"select_gather_update": us_select, "imp_qd_attn": us_both, "imp_qd_attn_kernel_only": us_kernel,
                       "merge_only": us_merge, "important_attn_alone": us_imp, "question_attn_alone": us_qd},
         "stages": {
@@ -668,6 +698,7 @@ def main():
                          f"default: {DEFAULT_PRIMARY} as the headline with {', '.join(DEFAULT_OTHERS)} under by_config")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying a CUDA graph")
+    ap.add_argument("--no-overlap", action="store_true", help="keep the selection kernels on the layer's own stream")
     ap.add_argument("--layers", type=int, default=0, help="use only the first LAYERS layers (profiling captures)")
     args = ap.parse_args()
     import dataclasses

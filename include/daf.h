@@ -119,6 +119,13 @@ int daf_select(const daf_params* p, const float* scores, int32_t n_sig, const in
                int32_t* idx_out, void* q_pack, void* k_pack, void* v_pack,
                void* workspace, size_t workspace_bytes, void* stream);
 
+/* The selection of step 1 alone: aggregates the score rows and writes the k selected positions, ascending, to
+ * idx_out; nothing is gathered.  For callers that schedule the selection apart from the rest of the layer -- it
+ * depends only on the scores, so it can run on another stream while an earlier layer's attention is still under
+ * way -- and then pass the positions to daf_select or daf_layer as idx_in.  Same result as daf_select's idx_out. */
+int daf_select_topk(const daf_params* p, const float* scores, int32_t n_sig, int32_t* idx_out,
+                    void* workspace, size_t workspace_bytes, void* stream);
+
 /* Step 1 starting from K/V instead of from scores (Methods item 1: the deviation signals of several layers,
  * typically the 2nd to 4th, are aggregated and the tokens ranked by the aggregate).  The signal of layer l is
  * the one daf_deviation_scores computes; the layers are added in ascending order in fp32, exactly as daf_select
@@ -284,6 +291,14 @@ int daf_layer_host(const daf_params* p, const float* h_scores, int32_t n_sig, co
                    void* h_kv_k, void* h_kv_v, int32_t copy_back_kv,
                    void* h_hidden, int32_t* h_idx_out,
                    void* arena, size_t arena_bytes, void* stream);
+
+/* Validation of caller-given positions (no counterpart in the paper).  daf_select and daf_layer trust idx_in to be
+ * strictly increasing positions in [0, L_d): only then is "causal in packed order" the same as "causal by position"
+ * (out-of-range positions are skipped and reported by the gather; an unsorted list is not noticed there).  This call
+ * checks k positions on the device and records the first offence in the status word of `workspace` (at least 256
+ * bytes, e.g. the layer workspace): daf_poll_status then returns DAF_ERR_BOUNDS.  Nothing faults or traps. */
+int daf_check_indices(const daf_params* p, int32_t k, const int32_t* idx, void* workspace, size_t workspace_bytes,
+                      void* stream);
 
 /* Reads the device status word kept in `workspace` (synchronises `stream`):
  * DAF_OK, DAF_ERR_TIMEOUT or DAF_ERR_BOUNDS; the word is cleared. */

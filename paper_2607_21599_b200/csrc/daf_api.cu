@@ -385,6 +385,34 @@ int daf_layer_fp8(const daf_params* p, const float* scores, int32_t n_sig, const
                       hidden, row_pos_out, workspace, workspace_bytes_, stream);
 }
 
+int daf_select_topk(const daf_params* p, const float* scores, int32_t n_sig, int32_t* idx_out,
+                    void* workspace, size_t workspace_bytes_, void* stream) {
+    ResolvedParams rp;
+    if (int rc = resolve_params(p, &rp)) return rc;
+    Workspace ws;
+    if (int rc = carve_workspace(rp, workspace, workspace_bytes_, &ws)) return rc;
+    if (rp.k == 0) return DAF_OK;
+    if (scores == nullptr || idx_out == nullptr || n_sig < 1) return DAF_ERR_INVALID_ARG;
+    if (!aligned16(scores) || !aligned16(idx_out)) return DAF_ERR_ALIGNMENT;
+    // selection alone: no rows to gather, no question rows to append
+    ResolvedParams sel = rp;
+    sel.L_q = 0;
+    return launch_select(sel, scores, n_sig, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, idx_out, nullptr, nullptr,
+                         nullptr, ws.status, ws.select_scratch, (cudaStream_t)stream, false, false, /*select_only=*/true);
+}
+
+int daf_check_indices(const daf_params* p, int32_t k, const int32_t* idx, void* workspace, size_t workspace_bytes_,
+                      void* stream) {
+    ResolvedParams rp;
+    if (int rc = resolve_params(p, &rp)) return rc;
+    if (k < 0 || k > rp.L_d) return DAF_ERR_INVALID_ARG;
+    if (workspace == nullptr || workspace_bytes_ < kStatusBytes) return DAF_ERR_WORKSPACE;
+    if (k == 0) return DAF_OK;
+    if (idx == nullptr) return DAF_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(idx) & 3u) != 0 || !aligned16(workspace)) return DAF_ERR_ALIGNMENT;
+    return launch_check_indices(idx, k, rp.L_d, reinterpret_cast<DeviceStatus*>(workspace), (cudaStream_t)stream);
+}
+
 int daf_expand_fp8_cache(const daf_params* p, const void* k_cached_fp8, const void* v_cached_fp8, const float* k_scale,
                          const float* v_scale, void* kv_k, void* kv_v, void* stream) {
     ResolvedParams rp;

@@ -598,7 +598,7 @@ int launch_select(const ResolvedParams& rp, const float* scores, int n_sig, cons
                   const void* q_fresh, const void* k_fresh, const void* v_fresh, void* kv_k, void* kv_v,
                   int32_t* idx_out, void* q_pack, void* k_pack, void* v_pack,
                   DeviceStatus* status, void* scratch, cudaStream_t stream, bool scores_from_previous_kernel,
-                  bool beside_previous_kernel) {
+                  bool beside_previous_kernel, bool select_only) {
     // beside_previous_kernel: the kernel launched just before (the fp8 cache expansion) is independent of the
     // selection; the selection kernel starts while it runs and only waits for it before it retires
     const bool dependent = scores_from_previous_kernel || beside_previous_kernel;
@@ -633,7 +633,7 @@ int launch_select(const ResolvedParams& rp, const float* scores, int n_sig, cons
         if (int rc = check_launch()) return rc;
         idx_src = idx_out;
     }
-    const int rows = rp.k + rp.L_q;
+    const int rows = select_only ? 0 : rp.k + rp.L_q;
     if (rows > 0) {
         GatherArgs a;
         a.q_fresh = reinterpret_cast<const int4*>(q_fresh);
@@ -691,6 +691,27 @@ int launch_deviation_sum(const ResolvedParams& rp, int n_sig, const void* const*
     const int max_blocks = 148 * 8;
     if (blocks > max_blocks) blocks = max_blocks;
     deviation_sum_kernel<<<blocks, warps * 32, 0, stream>>>(layers, rp.L_d, rp.Hkv * 16, sums);
+    count_launch();
+    return check_launch();
+}
+
+// ------------------------------------------------ validation of caller-given positions
+// The important-token stage treats "causal in packed order" as "causal by position", which holds only if the
+// positions are strictly increasing; a caller who passes idx_in can have them checked on the device: each
+// position must lie in [0, L_d) and exceed the one before it.  The first offence is recorded in the status
+// word (DAF_ERR_BOUNDS; where = 2 out of range, 3 not increasing; detail = the offending index into idx).
+__global__ void __launch_bounds__(256)
+check_indices_kernel(const int32_t* __restrict__ idx, int k, int L_d, DeviceStatus* status) {
+    const int i = (int)(blockIdx.x * blockDim.x + threadIdx.x);
+    if (i >= k) return;
+    const int p = idx[i];
+    if (p < 0 || p >= L_d) report_status(status, DAF_ERR_BOUNDS, 2, i);
+    else if (i > 0 && idx[i - 1] >= p) report_status(status, DAF_ERR_BOUNDS, 3, i);
+}
+
+int launch_check_indices(const int32_t* idx, int k, int L_d, DeviceStatus* status, cudaStream_t stream) {
+    if (k <= 0) return DAF_OK;
+    check_indices_kernel<<<(unsigned)((k + 255) / 256), 256, 0, stream>>>(idx, k, L_d, status);
     count_launch();
     return check_launch();
 }

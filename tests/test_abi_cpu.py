@@ -115,6 +115,10 @@ def test_host_side_argument_validation(lib):
     assert skv(2, kf=[buf, None]) == api.DAF_ERR_INVALID_ARG
     assert skv(2, kf=[buf, buf[8:]]) == api.DAF_ERR_ALIGNMENT
     assert skv(2, wsp=None) == api.DAF_ERR_WORKSPACE
+    assert api.daf_check_indices(ok, 300, buf, ws) == api.DAF_ERR_INVALID_ARG
+    assert api.daf_check_indices(ok, 4, None, ws) == api.DAF_ERR_INVALID_ARG
+    assert api.daf_check_indices(ok, 4, buf, None) == api.DAF_ERR_WORKSPACE
+    assert api.daf_check_indices(ok, 0, None, ws) == api.DAF_OK
     # the self-test of the bounded wait checks its arguments before it launches anything
     assert api.daf_selftest_bounded_wait(None, 50) == api.DAF_ERR_WORKSPACE
     assert api.daf_selftest_bounded_wait(ws[:64], 50) == api.DAF_ERR_WORKSPACE

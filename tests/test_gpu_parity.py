@@ -592,6 +592,18 @@ def test_out_of_range_index_is_skipped_and_reported():
     assert torch.all(qp[2] == 3.0) and torch.equal(qp[0], qf[3]) and torch.equal(qp[3], qf[40])
 
 
+@pytest.mark.parametrize("idx,expect", [([3, 9, 40, 63], 0), ([3, 9, 9, 40], -7), ([3, 40, 9, 50], -7), ([0, 1, 2, 64], -7),
+                                        ([-1, 1, 2, 3], -7), (list(range(0, 64)), 0), ([5], 0)])
+def test_positions_given_by_the_caller_can_be_checked_on_the_device(idx, expect):
+    p = api.make_params(64, 2, 0.5, 4, 2)
+    ws = api.alloc_workspace(p)
+    t = torch.tensor(idx, dtype=torch.int32, device="cuda")
+    api.check(api.daf_check_indices(p, len(idx), t, ws), "daf_check_indices")
+    torch.cuda.synchronize()
+    assert api.daf_poll_status(ws) == expect
+    assert api.daf_poll_status(ws) == api.DAF_OK      # reported once
+
+
 @pytest.mark.parametrize("L_d,L_q,r,Hq,Hkv,n_sig", [(900, 300, 0.2, 4, 4, 1), (512, 40, 1.0, 16, 2, 8),
                                                      (1500, 130, 0.1, 8, 1, 2), (257, 129, 0.5, 12, 4, 3)])
 def test_layer_edge_shapes(L_d, L_q, r, Hq, Hkv, n_sig):
