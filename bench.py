@@ -547,6 +547,7 @@ def measure_config(env: Env, w: W.Workload, primary: bool):
         "unit": "TFLOP/s",
         "frac": kernel_tflops / peaks["bf16_tflops"],
         "frac_with_merge": both_tflops / peaks["bf16_tflops"],
+        "frac_of_sustained_peak": (kernel_tflops / peaks["bf16_tflops_sustained"]) if peaks.get("bf16_tflops_sustained") else None,
         "peak_source": f"{peaks['source']} bf16 burst (kernel timed alone, all layers back to back)",
         "traffic": NCU_TRAFFIC_BYTES.get(w.name),
         "clocks": clocks_attn.summary(),
