@@ -442,7 +442,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
     unsigned char* v_smem = smem + 2 * (size_t)kTileBytes;        // two sub-step slots
     AttnSmem* sm = reinterpret_cast<AttnSmem*>(smem + 3 * (size_t)kTileBytes);
 
-    pdl_launch_dependents();   // a dependent kernel (the split merge) may start launching; it waits for this grid
 
     if (threadIdx.x == 0) DAF_STAMP(0);
     DAF_KT_BEGIN(0);
@@ -732,6 +731,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
     }
 
     if (threadIdx.x == 0) DAF_STAMP(4);
+    // Only now may the dependent kernel (the merge of the key ranges) start launching: its CTAs wait for this
+    // whole grid, and while they wait they hold registers and thread slots that CTAs of this grid could use.
+    pdl_launch_dependents();
     tc_fence_before();
     __syncthreads();
     if (warp == 5) {
@@ -743,7 +745,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
     if (threadIdx.x == 0) {
         DAF_STAMP(5);
         const unsigned cta = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
-        if (cta < 65536u) g_trace[8 * cta + 6] = (unsigned long long)n_t;
+        if (cta < 65536u) {
+            g_trace[8 * cta + 6] = (unsigned long long)n_t;
+            unsigned smid; asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+            g_trace[8 * cta + 7] = ((unsigned long long)smid << 32) | (unsigned long long)sm->tmem_base;
+        }
     }
 #endif
 }
