@@ -27,7 +27,7 @@ constexpr int kD = 128;                 // head_dim
 constexpr int kTileBytes = kBlockN * kD * 2;      // 32 KB: one Q tile, or K (or V) of 128 keys
 constexpr int kHalfBytes = kTileBytes / 2;        // one 64-column half (128-byte rows)
 constexpr int kMaxSplits = 32;
-constexpr int kNumSMs = 148;
+constexpr int kNumSMsDefault = 148;    // B200; the planners ask the device (num_sms below)
 constexpr float kRescaleThreshold = 8.0f;   // in log2 units: keep a stale row maximum up to 2^8
 
 // One attention problem and how it is cut into work items.
@@ -920,6 +920,23 @@ static int set_kernel_attributes() {
     return DAF_OK;
 }
 
+// SMs of the current device (asked once per device; 148 on B200).  Planning runs on the host and also
+// without a device (workspace sizing in CPU-only processes): then the B200 figure is used.
+static int num_sms() {
+    static std::atomic<int> cached[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { (void)cudaGetLastError(); return kNumSMsDefault; }
+    int n = cached[dev].load(std::memory_order_acquire);
+    if (n == 0) {
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+            (void)cudaGetLastError();
+            n = kNumSMsDefault;
+        }
+        cached[dev].store(n, std::memory_order_release);
+    }
+    return n;
+}
+
 // How a single problem is cut into CTAs: one per (head block, token block), and for the question rows,
 // where there are few query tiles and a long KV axis, also per range of the KV axis.
 
@@ -937,7 +954,7 @@ AttnPlan plan_attention(int n_q, int n_kv, int Hq, int G, int causal_off, bool p
     pl.tiles_per_split = total_tiles > 0 ? total_tiles : 1;
     if (allow_split && total_tiles > 1) {
         const int ctas = pl.n_tb * pl.head_blocks;
-        const int slots = kNumSMs * 2;
+        const int slots = num_sms() * 2;
         int want = ctas > 0 ? slots / ctas : 1;
         if (want > kMaxSplits) want = kMaxSplits;
         if (want > total_tiles) want = total_tiles;
@@ -1010,7 +1027,7 @@ void set_choice(JointPlan& jp, int chunk, int n_splits_q, int L_q, int L_d, int 
 
 // Predicted time of the attention launch + merge for a filled plan, in microseconds.
 float predict_us(const JointPlan& jp, int k, int L_q, int L_d, int Hq) {
-    const int slots = kNumSMs * 2;
+    const int slots = num_sms() * 2;
     std::priority_queue<float, std::vector<float>, std::greater<float>> free_at;
     for (int i = 0; i < slots; ++i) free_at.push(0.f);
     float makespan = 0.f;
@@ -1055,10 +1072,15 @@ JointPlan plan_joint(int k, int L_q, int L_d, int Hq, int G) {
     static std::map<JointShape, JointPlan> cache;
     const JointShape shape{k, L_q, L_d, Hq, G};
     const bool forced = g_force_chunk > 0 || g_force_splits_q > 0;
+    // a layer loop asks for the same shape over and over: each thread keeps its last answer (no lock)
+    static thread_local bool have_last = false;
+    static thread_local JointShape last_shape;
+    static thread_local JointPlan last_plan;
+    if (!forced && have_last && !(shape < last_shape) && !(last_shape < shape)) return last_plan;
     if (!forced) {
         std::lock_guard<std::mutex> lock(mu);
         auto it = cache.find(shape);
-        if (it != cache.end()) return it->second;
+        if (it != cache.end()) { last_shape = shape; last_plan = it->second; have_last = true; return it->second; }
     }
     JointPlan jp;
     jp.n_tb_i = (k + kBlockM - 1) / kBlockM;
@@ -1093,6 +1115,7 @@ JointPlan plan_joint(int k, int L_q, int L_d, int Hq, int G) {
     g_last_predicted_us = best_us;
     std::lock_guard<std::mutex> lock(mu);
     cache[shape] = best;
+    last_shape = shape; last_plan = best; have_last = true;
     return best;
 }
 

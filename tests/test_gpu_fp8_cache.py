@@ -50,7 +50,8 @@ def test_expansion_is_bit_exact(L_d, Hkv, scaled):
 
 
 @pytest.mark.parametrize("L_d,L_q,r,Hq,Hkv,scaled,given", [(1024, 32, 0.15, 28, 4, False, False), (1500, 70, 0.3, 8, 2, True, False),
-                                                           (900, 17, 0.2, 8, 8, True, True)])
+                                                           (900, 17, 0.2, 8, 8, True, True), (640, 0, 0.25, 4, 2, True, False),
+                                                           (640, 12, 0.0, 4, 2, False, False)])
 def test_layer_from_an_fp8_cache(L_d, L_q, r, Hq, Hkv, scaled, given):
     build.build()
     dev = "cuda"

@@ -592,6 +592,41 @@ def test_out_of_range_index_is_skipped_and_reported():
     assert torch.all(qp[2] == 3.0) and torch.equal(qp[0], qf[3]) and torch.equal(qp[3], qf[40])
 
 
+@pytest.mark.parametrize("L_d,r,n_sig", [(6144, 0.15, 1), (20000, 0.1, 3), (300, 1.0, 2), (300, 0.0, 1), (8193, 0.5, 1)])
+def test_selection_alone_gives_the_positions_of_the_full_call(L_d, r, n_sig):
+    """daf_select_topk writes what daf_select writes to idx_out (and the oracle's selection), and a layer run
+    from those positions through idx_in reproduces the layer run from the scores bit for bit."""
+    dev = "cuda"
+    L_q, Hq, Hkv = 9, 4, 2
+    w = W.Workload("st", 13, Hq, Hkv, 128, 1, L_d, L_d, L_q, r, "lognormal", n_sig).with_k(api.daf_num_important)
+    L = W.make_layer(w, 0, dev)
+    p = api.make_params(L_d, L_q, r, Hq, Hkv)
+    k = w.k
+    ws = api.alloc_workspace(p)
+    idx_sel = torch.full((max(k, 1),), -1, dtype=torch.int32, device=dev)
+    _ok(api.daf_select_topk(p, L["scores"], n_sig, idx_sel, ws), ws, "daf_select_topk")
+    assert np.array_equal(idx_sel[:k].cpu().numpy(), oracle.select(L["scores"].cpu().numpy(), k))
+    if k == 0:
+        assert int(idx_sel[0]) == -1
+        return
+    bf = torch.bfloat16
+
+    def run(scores, idx_in):
+        o = dict(kv_k=torch.cat([L["k_cached"], torch.zeros(L_q, Hkv, 128, dtype=bf, device=dev)]),
+                 kv_v=torch.cat([L["v_cached"], torch.zeros(L_q, Hkv, 128, dtype=bf, device=dev)]),
+                 idx=torch.full((k,), -1, dtype=torch.int32, device=dev), qp=torch.zeros(k, Hq, 128, dtype=bf, device=dev),
+                 kp=torch.zeros(k, Hkv, 128, dtype=bf, device=dev), vp=torch.zeros(k, Hkv, 128, dtype=bf, device=dev),
+                 hidden=torch.zeros(k + L_q, Hq, 128, dtype=bf, device=dev))
+        _ok(api.daf_layer(p, scores, n_sig if scores is not None else 0, idx_in, L["q_fresh"], L["k_fresh"], L["v_fresh"],
+                          o["kv_k"], o["kv_v"], o["idx"], o["qp"], o["kp"], o["vp"], o["hidden"], None, ws), ws, "daf_layer")
+        return o
+
+    a, b = run(L["scores"], None), run(None, idx_sel)
+    for name in a:
+        x, y = a[name], b[name]
+        assert torch.equal(x.view(torch.int16) if x.dtype == bf else x, y.view(torch.int16) if y.dtype == bf else y), name
+
+
 @pytest.mark.parametrize("idx,expect", [([3, 9, 40, 63], 0), ([3, 9, 9, 40], -7), ([3, 40, 9, 50], -7), ([0, 1, 2, 64], -7),
                                         ([-1, 1, 2, 3], -7), (list(range(0, 64)), 0), ([5], 0)])
 def test_positions_given_by_the_caller_can_be_checked_on_the_device(idx, expect):
