@@ -420,7 +420,7 @@ constexpr int kAttnTmemCols = 256;                     // S (two halves of 64) a
 
 struct AttnSmem {
     uint64_t q_full;
-    uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2];
+    uint64_t k_full[2], v_full[2];
     uint64_t s_full[2], p_full[2];
     uint64_t pv_done[2];      // O += P_t V_t has completed: sub-steps alternate between the two barriers
     uint64_t rows_parked;     // epilogue: the four softmax warps have parked their rows for the tiled store
@@ -483,8 +483,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
     if (warp == 4 && lane == 0) {
         mbar_init(&sm->q_full, q_idx != nullptr ? 4 : 1);
         for (int s = 0; s < 2; ++s) {
-            mbar_init(&sm->k_full[s], 1); mbar_init(&sm->k_empty[s], 1);
-            mbar_init(&sm->v_full[s], 1); mbar_init(&sm->v_empty[s], 1);
+            mbar_init(&sm->k_full[s], 1); mbar_init(&sm->v_full[s], 1);
             mbar_init(&sm->s_full[s], 1); mbar_init(&sm->p_full[s], 4);
         }
         mbar_init(&sm->pv_done[0], 1); mbar_init(&sm->pv_done[1], 1);
@@ -568,7 +567,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
                 const int slot = t & 1;
                 const uint32_t round = (uint32_t)(t >> 1);
                 for (int kv = 0; kv < 2 && ok; ++kv) {
-                    uint64_t* empty = kv == 0 ? &sm->k_empty[slot] : &sm->v_empty[slot];
+                    // a K slot is free once the logits read from it are complete, a V slot once its product is:
+                    // the barriers the softmax warps wait on say exactly that, so the issuer commits nothing extra
+                    uint64_t* empty = kv == 0 ? &sm->s_full[slot] : &sm->pv_done[slot];
                     ok = mbar_wait(empty, (round - 1) & 1u, abort_flag, status, 10 + 2 * kv + slot);
                     ok = __all_sync(0xFFFFFFFFu, ok);
                     if (ok && elect_one()) issue_kv(t, kv);
@@ -628,7 +629,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
                 if (elect_one()) {
                     issue_qk(t);
                     tc_commit(&sm->s_full[t]);
-                    tc_commit(&sm->k_empty[t]);
                 }
                 __syncwarp();
             }
@@ -642,7 +642,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
                 tc_fence_after();
                 if (elect_one()) {
                     issue_pv(b, t == 0);
-                    tc_commit(&sm->v_empty[b]);
                     tc_commit(&sm->pv_done[b]);
                 }
                 __syncwarp();
@@ -654,7 +653,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
                     if (elect_one()) {
                         issue_qk(b);
                         tc_commit(&sm->s_full[b]);
-                        tc_commit(&sm->k_empty[b]);
                     }
                     __syncwarp();
                 }
