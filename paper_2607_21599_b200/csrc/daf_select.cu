@@ -439,7 +439,7 @@ struct GatherArgs {
 __global__ void __launch_bounds__(kRowThreads)
 gather_update_kernel(const GatherArgs a) {
     DAF_KT_BEGIN(1);
-    pdl_wait();                // idx comes from the selection kernel launched just before
+    pdl_wait();                // idx may come from the selection kernel launched just before; the packed buffers may still be read by the previous layer
     DAF_KT_BEGIN(2);
     pdl_launch_dependents();   // the attention kernel may start launching; it waits for this grid
     const int row = blockIdx.x;
@@ -650,8 +650,12 @@ int launch_select(const ResolvedParams& rp, const float* scores, int n_sig, cons
         a.cq = rp.Hq * 16; a.ckv = rp.Hkv * 16;
         a.overwrite = rp.overwrite;
         a.status = status;
+        // Always a programmatic dependent of whatever kernel precedes it on the stream: the kernel waits for that
+        // kernel to complete before it touches anything (so the result is that of a plain launch), but its CTAs are
+        // already in place then -- after this library's selection kernel, and equally after the previous layer's
+        // merge when layers are issued back to back.
         cudaError_t e = launch_kernel(gather_update_kernel, dim3((unsigned)rows), dim3(kRowThreads), 0, stream,
-                                      /*after_kernel=*/idx_src == idx_out && scores != nullptr, a);
+                                      /*after_kernel=*/true, a);
         count_launch();
         if (e != cudaSuccess) { set_cuda_error(e); return DAF_ERR_CUDA; }
         if (int rc = check_launch()) return rc;
