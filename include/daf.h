@@ -284,13 +284,27 @@ int daf_layer_fp8(const daf_params* p, const float* scores, int32_t n_sig, const
  *                   (copied back only if copy_back_kv != 0)
  *   h_hidden        host output, layout by fuse_mode (compact mode recommended)
  *   h_idx_out       host int32 [k] (optional)
- * The call synchronises `stream` before returning. */
+ * The call synchronises `stream` before returning.
+ *
+ * daf_layer_host_begin / daf_layer_host_end are the two halves of that call: `begin` (same arguments) enqueues the
+ * copies in, the layer and the copies out on `stream` and returns without waiting; `end` waits for `stream` and
+ * returns the layer's status.  A caller with two arenas and two streams begins layer i + 1 before it ends layer
+ * i, so that the copies in of one layer run beside the kernels and the copies out of the other (the link to the
+ * host carries both directions at once).  Between `begin` and `end` the host buffers and the arena belong to the
+ * call; the host buffers must be pinned for the copies to overlap anything.  `end` without a `begin` on that
+ * arena returns whatever status word the arena holds. */
 size_t daf_layer_host_arena_bytes(const daf_params* p);
 int daf_layer_host(const daf_params* p, const float* h_scores, int32_t n_sig, const int32_t* h_idx_in,
                    const void* h_q_fresh, const void* h_k_fresh, const void* h_v_fresh,
                    void* h_kv_k, void* h_kv_v, int32_t copy_back_kv,
                    void* h_hidden, int32_t* h_idx_out,
                    void* arena, size_t arena_bytes, void* stream);
+int daf_layer_host_begin(const daf_params* p, const float* h_scores, int32_t n_sig, const int32_t* h_idx_in,
+                         const void* h_q_fresh, const void* h_k_fresh, const void* h_v_fresh,
+                         void* h_kv_k, void* h_kv_v, int32_t copy_back_kv,
+                         void* h_hidden, int32_t* h_idx_out,
+                         void* arena, size_t arena_bytes, void* stream);
+int daf_layer_host_end(const daf_params* p, void* arena, size_t arena_bytes, void* stream);
 
 /* Validation of caller-given positions (no counterpart in the paper).  daf_select and daf_layer trust idx_in to be
  * strictly increasing positions in [0, L_d): only then is "causal in packed order" the same as "causal by position"

@@ -29,7 +29,7 @@ DAF_ERR_BOUNDS = -7
 EXPORTS = [
     "daf_num_important", "daf_workspace_bytes", "daf_workspace_init", "daf_select", "daf_important_attn",
     "daf_qd_attn", "daf_fuse", "daf_full_causal_attn", "daf_layer", "daf_layer_host_arena_bytes",
-    "daf_layer_host", "daf_poll_status", "daf_strerror", "daf_last_cuda_error", "daf_launch_count",
+    "daf_layer_host", "daf_layer_host_begin", "daf_layer_host_end", "daf_poll_status", "daf_strerror", "daf_last_cuda_error", "daf_launch_count",
     "daf_qd_attn_static", "daf_qd_attn_static_max_bytes", "daf_deviation_scores", "daf_blend_attn",
     "daf_imp_qd_attn", "daf_selftest_bounded_wait", "daf_qd_attn_static_poll_status",
     "daf_imp_qd_attn_launches", "daf_select_from_kv", "daf_expand_fp8_cache", "daf_layer_fp8", "daf_check_indices", "daf_select_topk",
@@ -117,6 +117,10 @@ def lib() -> ctypes.CDLL:
         L.daf_layer_host_arena_bytes.argtypes = [pp]
         L.daf_layer_host.restype = ctypes.c_int
         L.daf_layer_host.argtypes = [pp, vp, i32, vp] + [vp] * 3 + [vp, vp, i32] + [vp, vp] + [vp, sz, vp]
+        L.daf_layer_host_begin.restype = ctypes.c_int
+        L.daf_layer_host_begin.argtypes = [pp, vp, i32, vp] + [vp] * 3 + [vp, vp, i32] + [vp, vp] + [vp, sz, vp]
+        L.daf_layer_host_end.restype = ctypes.c_int
+        L.daf_layer_host_end.argtypes = [pp, vp, sz, vp]
         L.daf_select_topk.restype = ctypes.c_int
         L.daf_select_topk.argtypes = [pp, vp, i32, vp, vp, sz, vp]
         L.daf_check_indices.restype = ctypes.c_int
@@ -314,6 +318,21 @@ def daf_layer_host(p, h_scores, n_sig, h_idx_in, h_q_fresh, h_k_fresh, h_v_fresh
     return lib().daf_layer_host(ctypes.byref(p), _ptr(h_scores), int(n_sig), _ptr(h_idx_in), _ptr(h_q_fresh),
                                 _ptr(h_k_fresh), _ptr(h_v_fresh), _ptr(h_kv_k), _ptr(h_kv_v), int(copy_back_kv),
                                 _ptr(h_hidden), _ptr(h_idx_out), _ptr(arena), _nbytes(arena), _stream(stream))
+
+
+def daf_layer_host_begin(p, h_scores, n_sig, h_idx_in, h_q_fresh, h_k_fresh, h_v_fresh, h_kv_k, h_kv_v, copy_back_kv,
+                         h_hidden, h_idx_out, arena, stream=None) -> int:
+    """daf_layer_host without the wait at its end (pinned host tensors); finish with daf_layer_host_end."""
+    for t in (h_scores, h_idx_in, h_q_fresh, h_k_fresh, h_v_fresh, h_kv_k, h_kv_v, h_hidden, h_idx_out):
+        if t is not None and t.is_cuda:
+            raise ValueError("daf_layer_host_begin takes host tensors")
+    return lib().daf_layer_host_begin(ctypes.byref(p), _ptr(h_scores), int(n_sig), _ptr(h_idx_in), _ptr(h_q_fresh),
+                                      _ptr(h_k_fresh), _ptr(h_v_fresh), _ptr(h_kv_k), _ptr(h_kv_v), int(copy_back_kv),
+                                      _ptr(h_hidden), _ptr(h_idx_out), _ptr(arena), _nbytes(arena), _stream(stream))
+
+
+def daf_layer_host_end(p, arena, stream=None) -> int:
+    return lib().daf_layer_host_end(ctypes.byref(p), _ptr(arena), _nbytes(arena), _stream(stream))
 
 
 def daf_select_topk(p, scores, n_sig, idx_out, workspace, stream=None) -> int:

@@ -467,11 +467,11 @@ size_t daf_layer_host_arena_bytes(const daf_params* p) {
 }
 
 
-int daf_layer_host(const daf_params* p, const float* h_scores, int32_t n_sig, const int32_t* h_idx_in,
-                   const void* h_q_fresh, const void* h_k_fresh, const void* h_v_fresh,
-                   void* h_kv_k, void* h_kv_v, int32_t copy_back_kv,
-                   void* h_hidden, int32_t* h_idx_out,
-                   void* arena, size_t arena_bytes, void* stream) {
+int daf_layer_host_begin(const daf_params* p, const float* h_scores, int32_t n_sig, const int32_t* h_idx_in,
+                         const void* h_q_fresh, const void* h_k_fresh, const void* h_v_fresh,
+                         void* h_kv_k, void* h_kv_v, int32_t copy_back_kv,
+                         void* h_hidden, int32_t* h_idx_out,
+                         void* arena, size_t arena_bytes, void* stream) {
     ResolvedParams rp;
     if (int rc = resolve_params(p, &rp)) return rc;
     if (h_scores != nullptr && (n_sig < 1 || n_sig > kArenaSignalRows)) return DAF_ERR_INVALID_ARG;
@@ -504,10 +504,31 @@ int daf_layer_host(const daf_params* p, const float* h_scores, int32_t n_sig, co
         DAF_CUDA_TRY(cudaMemcpyAsync(h_kv_k, a.kv_k, kvrow * rp.N, cudaMemcpyDeviceToHost, st));
         DAF_CUDA_TRY(cudaMemcpyAsync(h_kv_v, a.kv_v, kvrow * rp.N, cudaMemcpyDeviceToHost, st));
     }
-    DAF_CUDA_TRY(cudaStreamSynchronize(st));
+    return DAF_OK;
+}
+
+int daf_layer_host_end(const daf_params* p, void* arena, size_t arena_bytes, void* stream) {
+    ResolvedParams rp;
+    if (int rc = resolve_params(p, &rp)) return rc;
+    if (arena == nullptr || !aligned16(arena)) return DAF_ERR_WORKSPACE;
+    Arena a;
+    carve_arena(rp, kArenaSignalRows, reinterpret_cast<char*>(arena), &a);
+    if (arena_bytes < a.total) return DAF_ERR_WORKSPACE;
+    DAF_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+    if (rp.k + rp.L_q == 0) return DAF_OK;
     DeviceStatus hs;
     DAF_CUDA_TRY(cudaMemcpy(&hs, a.ws, sizeof(hs), cudaMemcpyDeviceToHost));
     return hs.code;
+}
+
+int daf_layer_host(const daf_params* p, const float* h_scores, int32_t n_sig, const int32_t* h_idx_in,
+                   const void* h_q_fresh, const void* h_k_fresh, const void* h_v_fresh,
+                   void* h_kv_k, void* h_kv_v, int32_t copy_back_kv,
+                   void* h_hidden, int32_t* h_idx_out,
+                   void* arena, size_t arena_bytes, void* stream) {
+    if (int rc = daf_layer_host_begin(p, h_scores, n_sig, h_idx_in, h_q_fresh, h_k_fresh, h_v_fresh, h_kv_k, h_kv_v,
+                                      copy_back_kv, h_hidden, h_idx_out, arena, arena_bytes, stream)) return rc;
+    return daf_layer_host_end(p, arena, arena_bytes, stream);
 }
 
 int daf_workspace_init(void* workspace, size_t workspace_bytes_, void* stream) {

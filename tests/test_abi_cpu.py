@@ -127,6 +127,8 @@ def test_host_side_argument_validation(lib):
     assert api.daf_launch_count() == 0
     assert "workspace" in api.daf_strerror(api.DAF_ERR_WORKSPACE)
     assert api.daf_layer_host(ok, None, 1, None, None, None, None, None, None, 0, None, None, None) == api.DAF_ERR_WORKSPACE
+    assert api.daf_layer_host_begin(ok, None, 1, None, None, None, None, None, None, 0, None, None, None) == api.DAF_ERR_WORKSPACE
+    assert api.daf_layer_host_end(ok, None) == api.DAF_ERR_WORKSPACE
 
 
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):

@@ -442,6 +442,49 @@ def _oracle_layer(w, L, fuse_mode):
                             hidden=base)
 
 
+def test_host_layers_pipelined_on_two_arenas_match_the_plain_host_call():
+    """daf_layer_host_begin / _end with two arenas and two streams (layer i + 1 begun before layer i is ended) give,
+    layer by layer, exactly what daf_layer_host gives."""
+    w = W.Workload("t", 31, 8, 2, 128, 5, 1200, 500, 40, 0.25, "lognormal", 2)
+    dev = "cuda"
+    p = api.make_params(w.L_d, w.L_q, w.r, w.n_q_heads, w.n_kv_heads)
+    k = api.daf_num_important(w.L_d, w.r)
+    pin = lambda t: None if t is None else t.pin_memory()  # noqa: E731
+
+    def host_layer(i):
+        L = W.make_layer(w, i)
+        h = {n: pin(t) for n, t in L.items()}
+        for n, src in (("kv_k", "k_cached"), ("kv_v", "v_cached")):
+            h[n] = torch.zeros(w.N, w.n_kv_heads, 128, dtype=torch.bfloat16).pin_memory()
+            h[n][: w.L_d] = L[src]
+        h["hidden"] = torch.full((k + w.L_q, w.n_q_heads, 128), -9.0, dtype=torch.bfloat16).pin_memory()
+        h["idx_out"] = torch.full((k,), -1, dtype=torch.int32).pin_memory()
+        return h
+
+    def args(h, arena):
+        return (p, h["scores"], 2, h["idx_in"], h["q_fresh"], h["k_fresh"], h["v_fresh"], h["kv_k"], h["kv_v"], 1,
+                h["hidden"], h["idx_out"], arena)
+
+    plain = [host_layer(i) for i in range(w.layers)]
+    arena = torch.zeros(api.daf_layer_host_arena_bytes(p), dtype=torch.uint8, device=dev)
+    for h in plain:
+        api.check(api.daf_layer_host(*args(h, arena)), "daf_layer_host")
+    piped = [host_layer(i) for i in range(w.layers)]
+    arenas = [torch.zeros_like(arena) for _ in range(2)]
+    lanes = [torch.cuda.Stream(), torch.cuda.Stream()]
+    pending = None
+    for i, h in enumerate(piped):
+        api.check(api.daf_layer_host_begin(*args(h, arenas[i & 1]), stream=lanes[i & 1]), "begin")
+        if pending is not None:
+            api.check(api.daf_layer_host_end(p, arenas[pending], stream=lanes[pending]), "end")
+        pending = i & 1
+    api.check(api.daf_layer_host_end(p, arenas[pending], stream=lanes[pending]), "end")
+    for a, b in zip(plain, piped):
+        for n in ("hidden", "idx_out", "kv_k", "kv_v"):
+            assert torch.equal(a[n], b[n]), n
+    assert not torch.equal(plain[0]["hidden"], plain[1]["hidden"])   # the layers do differ
+
+
 @pytest.mark.parametrize("fuse_mode", [0, 1])
 def test_layer_smallest_configuration(fuse_mode):
     w = W.CONFIGS["c0"]
