@@ -42,7 +42,7 @@ UNIT = "us/layer"
 Q_IN_PLACE_MIN_K = 16384    # from this many important tokens on, the layer is called without a packed-Q buffer
 # DRAM bytes per launch of the dominant kernel (the joint attention launch), dram__bytes_read.sum +
 # dram__bytes_write.sum of the committed ncu capture of that workload; no entry where none was captured.
-NCU_TRAFFIC_BYTES = {"c1": 21747456, "c2": 94365184, "c3": 148989696}
+NCU_TRAFFIC_BYTES = {"c1": 21746944, "c2": 93970176, "c3": 148794368}
 DEFAULT_PRIMARY, DEFAULT_OTHERS = "c3", ("c1", "c2")
 
 
