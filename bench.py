@@ -287,11 +287,15 @@ def measure_config(env: Env, w: W.Workload, primary: bool):
     # long condensed sequences are run that way.
     both = w.k > 0 and w.L_q > 0
     q_in_place = both and w.k >= Q_IN_PLACE_MIN_K
+    # Likewise the K/V rows of step 2 (--kv-in-place; slower, for comparison): the attention kernel fetches them
+    # through the positions and the kernel in front of it only updates the hybrid cache.
+    kv_in_place = both and args.kv_in_place
 
     def layer_call(b: LayerBuffers):
         L = b.L
         api.check(api.daf_layer(p, L["scores"], b.n_sig, L["idx_in"], L["q_fresh"], L["k_fresh"], L["v_fresh"], b.kv_k,
-                                b.kv_v, b.idx_out, None if q_in_place else b.q_pack, b.k_pack, b.v_pack, b.hidden, None, ws),
+                                b.kv_v, b.idx_out, None if q_in_place else b.q_pack, None if kv_in_place else b.k_pack,
+                                None if kv_in_place else b.v_pack, b.hidden, None, ws),
                   "daf_layer")
 
     def st_select(b, pack_q=False):
@@ -370,7 +374,8 @@ def measure_config(env: Env, w: W.Workload, primary: bool):
             main.wait_event(e)
             L = b.L
             api.check(api.daf_layer(p, None, 0, b.idx_sel, L["q_fresh"], L["k_fresh"], L["v_fresh"], b.kv_k, b.kv_v, b.idx_out,
-                                    None if q_in_place else b.q_pack, b.k_pack, b.v_pack, b.hidden, None, ws, stream=main),
+                                    None if q_in_place else b.q_pack, None if kv_in_place else b.k_pack,
+                                    None if kv_in_place else b.v_pack, b.hidden, None, ws, stream=main),
                       "daf_layer")
         main.wait_stream(side)
 
@@ -709,6 +714,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying a CUDA graph")
     ap.add_argument("--no-overlap", action="store_true", help="keep the selection kernels on the layer's own stream")
+    ap.add_argument("--kv-in-place", action="store_true",
+                    help="step 2 reads its K/V rows in place (no packed copies are written); slower, for comparison")
     ap.add_argument("--layers", type=int, default=0, help="use only the first LAYERS layers (profiling captures)")
     args = ap.parse_args()
     import dataclasses

@@ -111,7 +111,9 @@ int daf_deviation_scores(const daf_params* p, const void* k_fresh, const void* v
  *   idx_out  int32 [k] selected positions, ascending (also written when idx_in is given)
  *   q_pack   [k, n_q_heads, 128]; k_pack, v_pack [k, n_kv_heads, 128]: rows idx of the fresh tensors.
  *            q_pack may be NULL when no packed copy of the Q rows is wanted (daf_layer and
- *            daf_imp_qd_attn can read them in place).
+ *            daf_imp_qd_attn can read them in place).  k_pack and v_pack may be NULL, both or
+ *            neither, when no packed copies of the K/V rows are wanted (daf_layer can read them
+ *            in place); the cache update is done all the same.
  */
 int daf_select(const daf_params* p, const float* scores, int32_t n_sig, const int32_t* idx_in,
                const void* q_fresh, const void* k_fresh, const void* v_fresh,
@@ -247,6 +249,12 @@ int daf_full_causal_attn(const daf_params* p, int32_t n_tokens, const void* q, c
  *   hidden       compact: [k+L_q, n_q_heads*128]; scatter: [N, n_q_heads*128]
  *   row_pos_out  optional int32 [k+L_q]
  *   q_pack       may be NULL when L_q > 0: step 2 then reads its Q rows in place (see daf_imp_qd_attn)
+ *   k_pack, v_pack  may be NULL (both or neither) when k > 0 and L_q > 0: step 2 then reads its K/V rows in
+ *                place too -- rows idx of k_fresh / v_fresh, fetched by the attention kernel itself -- and
+ *                the kernel in front of it only updates the hybrid cache.  Same results, bit for bit, and no
+ *                packed buffers to provide; measured slower than the packed form at every size tried (the
+ *                rows are re-read by every query tile of their KV group), so pass the buffers where time matters.
+ *                DAF_ERR_INVALID_ARG if only one of the two is NULL, or if they are NULL while L_q == 0.
  */
 int daf_layer(const daf_params* p, const float* scores, int32_t n_sig, const int32_t* idx_in,
               const void* q_fresh, const void* k_fresh, const void* v_fresh, void* kv_k, void* kv_v,

@@ -99,7 +99,8 @@ static int do_select(const ResolvedParams& rp, const float* scores, int32_t n_si
     if (rp.k > 0) {
         if (scores == nullptr && idx_in == nullptr) return DAF_ERR_INVALID_ARG;
         if (scores != nullptr && idx_out == nullptr) return DAF_ERR_INVALID_ARG;
-        if (!q_fresh || !k_fresh || !v_fresh || !k_pack || !v_pack) return DAF_ERR_INVALID_ARG;   // q_pack is optional
+        if (!q_fresh || !k_fresh || !v_fresh) return DAF_ERR_INVALID_ARG;   // q_pack is optional
+        if ((k_pack == nullptr) != (v_pack == nullptr)) return DAF_ERR_INVALID_ARG;   // k_pack / v_pack: both or neither
         if (rp.overwrite && (!kv_k || !kv_v)) return DAF_ERR_INVALID_ARG;
     }
     if (rp.L_q > 0 && (!k_fresh || !v_fresh || !kv_k || !kv_v)) return DAF_ERR_INVALID_ARG;
@@ -238,7 +239,7 @@ int daf_imp_qd_attn_launches(const daf_params* p, const void* q_pack, const void
     if (int rc = check_out(hidden, row_bytes, rp.Hq)) return rc;
     char* h = reinterpret_cast<char*>(hidden);
     const int64_t first_row = rp.fuse_mode == 1 ? rp.L_d : rp.k;
-    return launch_attention_joint(q_pack, q_fresh, idx, k_pack, v_pack, rp.k, h, rp.fuse_mode == 1 ? idx : nullptr, q_question, kv_k, kv_v,
+    return launch_attention_joint(q_pack, q_fresh, idx, k_pack, v_pack, nullptr, nullptr, rp.k, h, rp.fuse_mode == 1 ? idx : nullptr, q_question, kv_k, kv_v,
                                   rp.L_q, rp.L_d, h + first_row * row_bytes, row_bytes, rp.Hq, rp.Hkv, rp.scale, ws.status,
                                   ws.attn_scratch, ws.attn_bytes, (cudaStream_t)stream, /*after_kernel=*/false, launches);
 }
@@ -323,10 +324,11 @@ int layer_impl(const daf_params* p, const Fp8Cache* fp8, const float* scores, in
         if (!aligned16(fp8->k8) || !aligned16(fp8->v8) || !aligned16(kv_k) || !aligned16(kv_v)) return DAF_ERR_ALIGNMENT;
     }
     if (rp.k > 0 && idx_out == nullptr) return DAF_ERR_INVALID_ARG;
-    if (rp.k > 0 && rp.L_q == 0 && q_pack == nullptr) return DAF_ERR_INVALID_ARG;   // only the joint launch reads Q in place
+    // only the joint launch reads the important rows in place
+    if (rp.k > 0 && rp.L_q == 0 && (q_pack == nullptr || k_pack == nullptr || v_pack == nullptr)) return DAF_ERR_INVALID_ARG;
     // the question rows are read from q_fresh even when nothing is selected (r = 0)
     if (rp.L_q > 0 && (q_fresh == nullptr || kv_k == nullptr || kv_v == nullptr)) return DAF_ERR_INVALID_ARG;
-    if (rp.k > 0 && (q_fresh == nullptr || k_pack == nullptr || v_pack == nullptr)) return DAF_ERR_INVALID_ARG;
+    if (rp.k > 0 && (q_fresh == nullptr || (k_pack == nullptr) != (v_pack == nullptr))) return DAF_ERR_INVALID_ARG;
     if (q_fresh != nullptr && !aligned16(q_fresh)) return DAF_ERR_ALIGNMENT;
     const int64_t row_bytes = (int64_t)rp.Hq * 256;
     if (int rc = check_out(hidden, row_bytes, rp.Hq)) return rc;
@@ -345,7 +347,7 @@ int layer_impl(const daf_params* p, const Fp8Cache* fp8, const float* scores, in
     const char* qq = reinterpret_cast<const char*>(q_fresh) + (int64_t)rp.L_d * row_bytes;
     const int32_t* dst = rp.fuse_mode == 1 ? idx_out : nullptr;
     if (rp.k > 0 && rp.L_q > 0) {
-        if (int rc = launch_attention_joint(q_pack, q_fresh, idx_out, k_pack, v_pack, rp.k, h, dst, qq, kv_k, kv_v, rp.L_q, rp.L_d,
+        if (int rc = launch_attention_joint(q_pack, q_fresh, idx_out, k_pack, v_pack, k_fresh, v_fresh, rp.k, h, dst, qq, kv_k, kv_v, rp.L_q, rp.L_d,
                                             h + first_row * row_bytes, row_bytes, rp.Hq, rp.Hkv, rp.scale, ws.status,
                                             ws.attn_scratch, ws.attn_bytes, st, /*after_kernel=*/true)) return rc;
     } else if (rp.L_q > 0) {

@@ -45,6 +45,12 @@ struct SegArgs {
     const __nv_bfloat16* q_src;
     const int32_t* q_idx;
     int q_src_rows;
+    // Likewise the keys: key j is row kv_idx[j] of k_src / v_src, [kv_src_rows, kv_heads, 128] tensors.
+    // k_src == nullptr: the K and V tensor maps cover packed rows.
+    const __nv_bfloat16* k_src;
+    const __nv_bfloat16* v_src;
+    const int32_t* kv_idx;
+    int kv_src_rows, kv_heads;
     // Work items.  A CTA owns one token block (a unit).  Either every unit is cut into the same n_splits
     // KV ranges of tiles_per_split tiles (chunk == 0), or -- packed causal attention only, where unit u
     // sees min(u + 1, n_tb) tiles -- units [g chunk, (g + 1) chunk) are cut into g + 1 balanced ranges
@@ -429,6 +435,7 @@ struct AttnSmem {
 };
 constexpr size_t kAttnSmemBytes = 1024 + 3 * (size_t)kTileBytes + sizeof(AttnSmem);
 
+template <bool kGatherKV>
 __global__ void __launch_bounds__(kAttnThreads, 2)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_constant__ CUtensorMap tmap_k0,
                   const __grid_constant__ CUtensorMap tmap_v0, const __grid_constant__ CUtensorMap tmap_q1,
@@ -457,6 +464,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
     const int g_kv = h0 / a.G;
     const int t0 = a.unit * a.Tt;
     const int key_begin = a.j_begin * kBlockN;
+    // kGatherKV: the launch has a problem whose K/V rows the producer warp fetches in place through an index (k_src
+    // non-null); a form of its own, so that the plain form carries none of that code
+    const __nv_bfloat16* const k_src = kGatherKV ? DAF_SEG(k_src) : nullptr;
+    const bool kv_gather = kGatherKV && k_src != nullptr;
 
     // Loads K (kv = 0) or V (kv = 1) of sub-step t into its ring slot (the slot must be free).
     auto issue_kv = [&](int t, int kv) {
@@ -468,6 +479,44 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
         mbar_arrive_expect_tx(full, (uint32_t)kSubBytes);
         tma_load_3d(dst, tm, full, 0, g_kv, key0);
         tma_load_3d(dst + kSubHalfBytes, tm, full, 64, g_kv, key0);
+    };
+    // The same for K/V rows fetched in place (the whole producer warp): row j of the sub-step is row idx[key0 + j] of
+    // the source tensor, copied by cp.async in 16-byte chunks into the layout the tiled load would have produced;
+    // rows past the end are zero-filled.  pos_lo / pos_hi: this lane's source rows for sub-tile rows `lane` and
+    // `32 + lane` (-1: none).  A copy group is handed to the tensor cores by kv_gather_arrive once it has landed.
+    uint64_t* gather_pending = nullptr;          // full-barrier of the copy group committed last
+    auto kv_gather_arrive = [&](bool all) {
+        if (gather_pending != nullptr) {
+            if (all) cp_async_wait_group<0>(); else cp_async_wait_group<1>();
+            fence_proxy_async();                 // this lane's landed copies, before the tensor cores read them
+            mbar_arrive(gather_pending);
+        }
+    };
+    auto gather_kv = [&](int t, int kv, int pos_lo, int pos_hi) {
+        const int slot = t & 1;
+        uint64_t* full = kv == 0 ? &sm->k_full[slot] : &sm->v_full[slot];
+        const uint32_t dst = smem_u32((kv == 0 ? k_smem : v_smem) + (size_t)slot * kSubBytes);
+        const __nv_bfloat16* src = (kv == 0 ? k_src : DAF_SEG(v_src)) + (size_t)g_kv * kD;
+        const size_t row_elems = (size_t)DAF_SEG(kv_heads) * kD;
+        const int sub = lane >> 4, ch = lane & 15;
+#pragma unroll 8
+        for (int i = 0; i < 32; ++i) {
+            const int j = 2 * i + sub;
+            const int pos = __shfl_sync(0xFFFFFFFFu, i < 16 ? pos_lo : pos_hi, j & 31);
+            cp_async16(dst + (uint32_t)((ch >> 3) * kSubHalfBytes + j * 128 + (((ch & 7) ^ (j & 7)) << 4)),
+                       src + (size_t)(pos < 0 ? 0 : pos) * row_elems + ch * 8, pos < 0 ? 0u : 16u);
+        }
+        cp_async_commit();
+        kv_gather_arrive(false);                 // the group before this one has landed (or is waited for here)
+        gather_pending = full;
+    };
+    auto gather_positions = [&](int t, int& pos_lo, int& pos_hi) {
+        const int key0 = key_begin + t * kSubN;
+        const int rows = DAF_SEG(kv_src_rows);
+        const int32_t* kv_idx = DAF_SEG(kv_idx);
+        pos_lo = pos_hi = -1;
+        if (key0 + lane < a.n_kv) { const int v = __ldg(kv_idx + key0 + lane); if ((unsigned)v < (unsigned)rows) pos_lo = v; }
+        if (key0 + 32 + lane < a.n_kv) { const int v = __ldg(kv_idx + key0 + 32 + lane); if ((unsigned)v < (unsigned)rows) pos_hi = v; }
     };
     // Set-up.  The producer thread prepares the barriers and at once starts the loads that need no free
     // slot (Q and the first two sub-steps), so that their latency overlaps the rest of the set-up: the
@@ -483,7 +532,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
     if (warp == 4 && lane == 0) {
         mbar_init(&sm->q_full, q_idx != nullptr ? 4 : 1);
         for (int s = 0; s < 2; ++s) {
-            mbar_init(&sm->k_full[s], 1); mbar_init(&sm->v_full[s], 1);
+            mbar_init(&sm->k_full[s], kv_gather ? 32 : 1); mbar_init(&sm->v_full[s], kv_gather ? 32 : 1);
             mbar_init(&sm->s_full[s], 1); mbar_init(&sm->p_full[s], 4);
         }
         mbar_init(&sm->pv_done[0], 1); mbar_init(&sm->pv_done[1], 1);
@@ -511,7 +560,17 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
                 tma_load_3d(q_smem, tmap_q, &sm->q_full, 0, h0, t0);
                 tma_load_3d(q_smem + kHalfBytes, tmap_q, &sm->q_full, 64, h0, t0);
             }
-            for (int t = 0; t < 2 && t < n_t; ++t) { issue_kv(t, 0); issue_kv(t, 1); }
+            if (!kv_gather)
+                for (int t = 0; t < 2 && t < n_t; ++t) { issue_kv(t, 0); issue_kv(t, 1); }
+        }
+    }
+    if (warp == 4 && kv_gather) {
+        __syncwarp();              // the barriers that lane 0 prepared above, before the other lanes arrive on them
+        for (int t = 0; t < 2 && t < n_t; ++t) {
+            int pos_lo, pos_hi;
+            gather_positions(t, pos_lo, pos_hi);
+            gather_kv(t, 0, pos_lo, pos_hi);
+            gather_kv(t, 1, pos_lo, pos_hi);
         }
     }
     if (q_idx != nullptr && n_t > 0 && warp < 4) {
@@ -552,7 +611,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
 
     if (skip) {
         // nothing is computed; the loads already under way get a bounded chance to land before the CTA retires
-        if (warp == 4 && lane == 0 && n_t > 0) {
+        if (warp == 4 && kv_gather) kv_gather_arrive(true);
+        if (warp == 4 && lane == 0 && n_t > 0 && !kv_gather) {
             for (int i = 0; i < 4096 && !mbar_try_wait(&sm->q_full, 0); ++i) {}
             for (int s = 0; s < 2 && s < n_t; ++s) {
                 for (int i = 0; i < 4096 && !mbar_try_wait(&sm->k_full[s], 0); ++i) {}
@@ -566,17 +626,20 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
             for (int t = 2; t < n_t && ok; ++t) {
                 const int slot = t & 1;
                 const uint32_t round = (uint32_t)(t >> 1);
+                int pos_lo = -1, pos_hi = -1;
+                if (kv_gather) gather_positions(t, pos_lo, pos_hi);
                 for (int kv = 0; kv < 2 && ok; ++kv) {
                     // a K slot is free once the logits read from it are complete, a V slot once its product is:
                     // the barriers the softmax warps wait on say exactly that, so the issuer commits nothing extra
                     uint64_t* empty = kv == 0 ? &sm->s_full[slot] : &sm->pv_done[slot];
                     ok = mbar_wait(empty, (round - 1) & 1u, abort_flag, status, 10 + 2 * kv + slot);
                     ok = __all_sync(0xFFFFFFFFu, ok);
-                    if (ok && elect_one()) issue_kv(t, kv);
+                    if (ok && kv_gather) gather_kv(t, kv, pos_lo, pos_hi);
+                    else if (ok && elect_one()) issue_kv(t, kv);
                     __syncwarp();
                 }
             }
-            if (!ok && lane == 0) {
+            if (!ok && lane == 0 && !kv_gather) {
                 // give loads already in flight a bounded chance to land before the CTA retires
                 for (int s = 0; s < 2; ++s) {
                     for (int i = 0; i < 4096 && !mbar_try_wait(&sm->k_full[s], 0) && !mbar_try_wait(&sm->k_full[s], 1); ++i) {}
@@ -584,6 +647,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
                 }
             }
         }
+        if (kv_gather) kv_gather_arrive(true);   // the last copy group (also on the way out after a give-up: copies always land)
     } else if (warp == 5) {
         // ------------------------------------------------------------ MMA issuer
         // The whole warp walks the loop and waits on the barriers, one elected lane issues: control flow
@@ -911,7 +975,9 @@ static int set_kernel_attributes() {
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !attr_done[dev].load(std::memory_order_acquire)) {
-        cudaError_t e = cudaFuncSetAttribute(attn_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttnSmemBytes);
+        cudaError_t e = cudaFuncSetAttribute(attn_fwd_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttnSmemBytes);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(attn_fwd_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttnSmemBytes);
         if (e != cudaSuccess) { set_cuda_error(e); return DAF_ERR_CUDA; }
         attr_done[dev].store(true, std::memory_order_release);
     }
@@ -1200,7 +1266,7 @@ int launch_attention(const void* q, const void* k, const void* v, int n_q, int n
     a.joint = 0;
     a.status = status;
     dim3 grid((unsigned)pl.head_blocks, (unsigned)pl.n_tb, (unsigned)pl.n_splits);
-    cudaError_t e = launch_kernel(attn_fwd_kernel, grid, dim3(kAttnThreads), kAttnSmemBytes, stream, after_kernel, tq, tk, tv, tq, tk, tv,
+    cudaError_t e = launch_kernel(attn_fwd_kernel<false>, grid, dim3(kAttnThreads), kAttnSmemBytes, stream, after_kernel, tq, tk, tv, tq, tk, tv,
                                   to, to, a);
     count_launch();
     if (e != cudaSuccess) { set_cuda_error(e); return DAF_ERR_CUDA; }
@@ -1238,6 +1304,7 @@ int launch_bounded_wait_selftest(DeviceStatus* status, int limit_ms, cudaStream_
 size_t joint_partial_bytes(const JointPlan& jp) { return jp.part_bytes_q + jp.part_bytes_i; }
 
 int launch_attention_joint(const void* q_imp, const void* q_fresh, const int32_t* idx, const void* k_imp, const void* v_imp,
+                           const void* k_fresh, const void* v_fresh,
                            int k, void* out_imp, const int32_t* dst_rows_imp, const void* q_question, const void* kv_k,
                            const void* kv_v,
                            int L_q, int L_d, void* out_question, long long out_row_stride_bytes, int Hq, int Hkv,
@@ -1252,11 +1319,18 @@ int launch_attention_joint(const void* q_imp, const void* q_fresh, const int32_t
     const bool gather_q = q_imp == nullptr;
     if (gather_q && (q_fresh == nullptr || idx == nullptr)) return DAF_ERR_INVALID_ARG;
     if (int rc = make_tmap(&tq0, gather_q ? q_question : q_imp, gather_q ? L_q : k, Hq, 1, kBlockM)) return rc;
-    if (int rc = make_tmap(&tk0, k_imp, k, Hkv, 1, kSubN)) return rc;
-    if (int rc = make_tmap(&tv0, v_imp, k, Hkv, 1, kSubN)) return rc;
+    // without packed K/V rows the producer warp reads them in place through idx as well
+    const bool gather_kv = k_imp == nullptr;
+    if (gather_kv && (v_imp != nullptr || k_fresh == nullptr || v_fresh == nullptr || idx == nullptr)) return DAF_ERR_INVALID_ARG;
+    if (!gather_kv && v_imp == nullptr) return DAF_ERR_INVALID_ARG;
     if (int rc = make_tmap(&tq1, q_question, L_q, Hq, jp.Gp_q, jp.Tt_q)) return rc;
     if (int rc = make_tmap(&tk1, kv_k, N, Hkv, 1, kSubN)) return rc;
     if (int rc = make_tmap(&tv1, kv_v, N, Hkv, 1, kSubN)) return rc;
+    tk0 = tk1; tv0 = tv1;      // placeholders when the important rows' K/V are read in place
+    if (!gather_kv) {
+        if (int rc = make_tmap(&tk0, k_imp, k, Hkv, 1, kSubN)) return rc;
+        if (int rc = make_tmap(&tv0, v_imp, k, Hkv, 1, kSubN)) return rc;
+    }
     // final rows in token order (the compact layout) leave by tiled stores
     CUtensorMap to0 = tq1, to1 = tq1;
     const bool imp_tiled = dst_rows_imp == nullptr;
@@ -1286,6 +1360,13 @@ int launch_attention_joint(const void* q_imp, const void* q_fresh, const int32_t
         si.q_idx = idx;
         si.q_src_rows = L_d;
     }
+    if (gather_kv) {
+        si.k_src = reinterpret_cast<const __nv_bfloat16*>(k_fresh);
+        si.v_src = reinterpret_cast<const __nv_bfloat16*>(v_fresh);
+        si.kv_idx = idx;
+        si.kv_src_rows = L_d;
+        si.kv_heads = Hkv;
+    }
     si.out_tiled = imp_tiled ? 1 : 0;
     si.n_units = jp.n_tb_i;
     si.n_splits = 1; si.tiles_per_split = jp.n_tb_i;
@@ -1299,8 +1380,11 @@ int launch_attention_joint(const void* q_imp, const void* q_fresh, const int32_t
 
     const int items = jp.items_q + jp.items_i;
     if (launches & 1) {
-        const cudaError_t e = launch_kernel(attn_fwd_kernel, dim3((unsigned)items), dim3(kAttnThreads), kAttnSmemBytes, stream,
-                                            after_kernel, tq0, tk0, tv0, tq1, tk1, tv1, to0, to1, a);
+        const cudaError_t e = gather_kv
+            ? launch_kernel(attn_fwd_kernel<true>, dim3((unsigned)items), dim3(kAttnThreads), kAttnSmemBytes, stream,
+                            after_kernel, tq0, tk0, tv0, tq1, tk1, tv1, to0, to1, a)
+            : launch_kernel(attn_fwd_kernel<false>, dim3((unsigned)items), dim3(kAttnThreads), kAttnSmemBytes, stream,
+                            after_kernel, tq0, tk0, tv0, tq1, tk1, tv1, to0, to1, a);
         count_launch();
         if (e != cudaSuccess) { set_cuda_error(e); return DAF_ERR_CUDA; }
         if (int rc = check_launch()) return rc;

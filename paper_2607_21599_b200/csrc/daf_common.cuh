@@ -68,8 +68,10 @@ struct JointPlan {
 JointPlan plan_joint(int k, int L_q, int L_d, int Hq, int G);
 size_t joint_partial_bytes(const JointPlan& jp);
 int launch_bounded_wait_selftest(DeviceStatus* status, int limit_ms, cudaStream_t stream);
-// q_imp == nullptr: the important rows' Q is read in place, row idx[j] of q_fresh
+// q_imp == nullptr: the important rows' Q is read in place, row idx[j] of q_fresh;
+// k_imp == nullptr (then v_imp too): their K and V are read in place, rows idx[j] of k_fresh / v_fresh
 int launch_attention_joint(const void* q_imp, const void* q_fresh, const int32_t* idx, const void* k_imp, const void* v_imp,
+                           const void* k_fresh, const void* v_fresh,
                            int k, void* out_imp, const int32_t* dst_rows_imp, const void* q_question, const void* kv_k,
                            const void* kv_v,
                            int L_q, int L_d, void* out_question, long long out_row_stride_bytes, int Hq, int Hkv,
@@ -213,6 +215,15 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap* m, const void* s
 __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 // waits until the bulk stores committed so far have finished reading shared memory
 __device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+
+// ---- cp.async (16-byte copies global -> shared by ordinary threads; used where rows are fetched through an index)
+// copies 16 bytes, or writes 16 zero bytes when src_bytes == 0 (src must still be a valid address)
+__device__ __forceinline__ void cp_async16(uint32_t dst_smem, const void* src, uint32_t src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst_smem), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait_group() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 // makes this thread's earlier shared-memory writes visible to the asynchronous proxy (TMA, tensor cores)
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }

@@ -424,7 +424,6 @@ select_topk_cta_kernel(const float* __restrict__ scores, int n_sig, int L_d, int
 // go to the packed buffers and (K/V) into the cache rows at their positions.
 // Rows k..k+L_q-1 are the question tokens: fresh K/V rows are appended to the cache.
 constexpr int kRowThreads = 192;
-constexpr int kRowMaxChunks = 4;      // chunks a thread requests before it stores any (4 x 192 x 16 B = 12 KB: a row of 32 + 2 x 8 heads)
 
 struct GatherArgs {
     const int4* q_fresh; const int4* k_fresh; const int4* v_fresh;
@@ -454,33 +453,21 @@ gather_update_kernel(const GatherArgs a) {
         }
         const size_t qsrc = (size_t)p * a.cq, qdst = (size_t)row * a.cq;
         const size_t ksrc = (size_t)p * a.ckv, kdst = (size_t)row * a.ckv;
-        // Every thread first requests all its 16-byte chunks of the row (at most kRowMaxChunks), then stores them: the
-        // kernel is a chain of two dependent round trips per row (position, then row), and a third or fourth one per
-        // thread -- loads held back behind the stores of the chunk before -- is what can be avoided.
-        const int c0 = (a.q_pack != nullptr ? 0 : a.cq) + threadIdx.x;       // no packed Q wanted: K, V only
-        for (int base = c0; base < per_row; base += kRowThreads * kRowMaxChunks) {
-            int4 v[kRowMaxChunks];
-#pragma unroll
-            for (int u = 0; u < kRowMaxChunks; ++u) {
-                const int c = base + u * kRowThreads;
-                if (c < a.cq) v[u] = __ldg(a.q_fresh + qsrc + c);
-                else if (c < a.cq + a.ckv) v[u] = __ldg(a.k_fresh + ksrc + (c - a.cq));
-                else if (c < per_row) v[u] = __ldg(a.v_fresh + ksrc + (c - a.cq - a.ckv));
-            }
-#pragma unroll
-            for (int u = 0; u < kRowMaxChunks; ++u) {
-                const int c = base + u * kRowThreads;
-                if (c < a.cq) {
-                    a.q_pack[qdst + c] = v[u];
-                } else if (c < a.cq + a.ckv) {
-                    const int cc = c - a.cq;
-                    a.k_pack[kdst + cc] = v[u];
-                    if (a.overwrite) a.kv_k[ksrc + cc] = v[u];
-                } else if (c < per_row) {
-                    const int cc = c - a.cq - a.ckv;
-                    a.v_pack[kdst + cc] = v[u];
-                    if (a.overwrite) a.kv_v[ksrc + cc] = v[u];
-                }
+        // no packed Q wanted: K, V only; no packed K/V wanted and nothing to overwrite in the cache: nothing at all
+        const int c_end = (a.k_pack != nullptr || a.overwrite) ? per_row : a.cq;
+        for (int c = (a.q_pack != nullptr ? 0 : a.cq) + threadIdx.x; c < c_end; c += kRowThreads) {
+            if (c < a.cq) {
+                a.q_pack[qdst + c] = __ldg(a.q_fresh + qsrc + c);
+            } else if (c < a.cq + a.ckv) {
+                const int cc = c - a.cq;
+                const int4 v = __ldg(a.k_fresh + ksrc + cc);
+                if (a.k_pack != nullptr) a.k_pack[kdst + cc] = v;
+                if (a.overwrite) a.kv_k[ksrc + cc] = v;
+            } else {
+                const int cc = c - a.cq - a.ckv;
+                const int4 v = __ldg(a.v_fresh + ksrc + cc);
+                if (a.v_pack != nullptr) a.v_pack[kdst + cc] = v;
+                if (a.overwrite) a.kv_v[ksrc + cc] = v;
             }
         }
     } else {

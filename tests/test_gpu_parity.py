@@ -433,13 +433,13 @@ def _run_layer(w, layer, fuse_mode, host=False):
     return L, hidden.cpu(), idx_out[:k].cpu().numpy(), row_pos[: k + w.L_q].cpu().numpy(), kv_k.cpu(), kv_v.cpu()
 
 
-def _oracle_layer(w, L, fuse_mode):
+def _oracle_layer(w, L, fuse_mode, overwrite=1):
     base = np.full((w.N, w.n_q_heads, 128), -9.0) if fuse_mode == 1 else None
     return oracle.daf_layer(_f(L["q_fresh"]), _f(L["k_fresh"]), _f(L["v_fresh"]), _f(L["k_cached"]), _f(L["v_cached"]),
                             w.L_d, w.L_q, w.softmax_scale,
                             scores=None if L["scores"] is None else L["scores"].numpy(),
                             idx=None if L["idx_in"] is None else L["idx_in"].numpy(), r=w.r, fuse_mode=fuse_mode,
-                            hidden=base)
+                            overwrite=bool(overwrite), hidden=base)
 
 
 def test_host_layers_pipelined_on_two_arenas_match_the_plain_host_call():
@@ -784,6 +784,68 @@ def test_layer_without_packed_q_buffer(fuse_mode):
                        ws), ws, "daf_select")
     assert torch.equal(idx_out.cpu(), outs[0][1]) and torch.equal(kp.cpu(), outs[0][2]) and torch.equal(vp.cpu(), outs[0][3])
     assert torch.equal(kv_k.cpu(), outs[0][4]) and torch.equal(kv_v.cpu(), outs[0][5])
+
+
+@pytest.mark.parametrize("fuse_mode,overwrite,with_q", [(0, 1, True), (1, 1, False), (0, 0, False), (1, 0, True)])
+@pytest.mark.parametrize("shape", [(1500, 70, 0.3, 8, 2), (3000, 64, 0.31, 28, 4), (700, 140, 0.9, 4, 4), (260, 3, 0.5, 8, 1)])
+def test_layer_without_packed_kv_buffers(shape, fuse_mode, overwrite, with_q):
+    """daf_layer with k_pack = v_pack = NULL: the attention kernel fetches the important rows' K/V in place (rows idx
+    of the fresh tensors, ragged last sub-step zero-filled) and the kernel before it only updates the cache.  Same
+    bits as with the packed copies, in both fusion modes, with and without the cache overwrite, with and without
+    a packed Q; and against the oracle."""
+    L_d, L_q, r, Hq, Hkv = shape
+    w = W.Workload("t", 23, Hq, Hkv, 128, 1, L_d, 500, L_q, r, "lognormal", 2)
+    L = W.make_layer(w, 0)
+    dev = "cuda"
+    p = api.make_params(w.L_d, w.L_q, w.r, Hq, Hkv, fuse_mode=fuse_mode, overwrite_doc_kv=overwrite)
+    k = api.daf_num_important(w.L_d, w.r)
+    g = {n: (None if t is None else t.to(dev)) for n, t in L.items()}
+    rows = k + w.L_q if fuse_mode == 0 else w.N
+    outs = []
+    for with_kv in (True, False):
+        ws = api.alloc_workspace(p)
+        kv_k = torch.zeros(w.N, Hkv, 128, dtype=torch.bfloat16, device=dev)
+        kv_v = torch.zeros_like(kv_k)
+        kv_k[: w.L_d], kv_v[: w.L_d] = g["k_cached"], g["v_cached"]
+        idx_out = torch.full((k,), -1, dtype=torch.int32, device=dev)
+        qp = torch.zeros(k, Hq, 128, dtype=torch.bfloat16, device=dev) if with_q else None
+        kp = torch.zeros(k, Hkv, 128, dtype=torch.bfloat16, device=dev) if with_kv else None
+        vp = torch.zeros(k, Hkv, 128, dtype=torch.bfloat16, device=dev) if with_kv else None
+        hidden = torch.full((rows, Hq, 128), -9.0, dtype=torch.bfloat16, device=dev)
+        _ok(api.daf_layer(p, g["scores"], 2, None, g["q_fresh"], g["k_fresh"], g["v_fresh"], kv_k, kv_v, idx_out,
+                          qp, kp, vp, hidden, None, ws), ws, "daf_layer")
+        outs.append((hidden.cpu(), idx_out.cpu(), kv_k.cpu(), kv_v.cpu()))
+    for a, b in zip(outs[0], outs[1]):
+        assert torch.equal(a, b), "reading K/V in place must give the same bits as reading the packed copies"
+    ref = _oracle_layer(w, L, fuse_mode, overwrite=overwrite)
+    hid = outs[1][0]
+    assert np.array_equal(outs[1][1].numpy(), ref["idx"])
+    assert np.array_equal(_f(outs[1][2]), ref["kv_k"]) and np.array_equal(_f(outs[1][3]), ref["kv_v"])
+    sel = np.arange(len(ref["row_pos"])) if fuse_mode == 0 else ref["row_pos"]
+    _assert_close(hid[sel], ref["hidden"][sel], "hidden rows, K/V read in place")
+
+
+def test_layer_rejects_half_a_pair_of_packed_kv_buffers():
+    """k_pack and v_pack go together; without a question there is no joint launch to read rows in place."""
+    dev = "cuda"
+    w = W.Workload("t", 3, 4, 2, 128, 1, 300, 100, 20, 0.3, "lognormal", 1)
+    L = {n: (None if t is None else t.to(dev)) for n, t in W.make_layer(w, 0).items()}
+    p = api.make_params(w.L_d, w.L_q, w.r, 4, 2)
+    k = api.daf_num_important(w.L_d, w.r)
+    ws = api.alloc_workspace(p)
+    kv = torch.zeros(w.N, 2, 128, dtype=torch.bfloat16, device=dev)
+    kv2 = torch.zeros_like(kv)
+    idx_out = torch.zeros(k, dtype=torch.int32, device=dev)
+    kp = torch.zeros(k, 2, 128, dtype=torch.bfloat16, device=dev)
+    hidden = torch.zeros(k + w.L_q, 4, 128, dtype=torch.bfloat16, device=dev)
+    for a, b in ((kp, None), (None, kp)):
+        assert api.daf_layer(p, L["scores"], 1, None, L["q_fresh"], L["k_fresh"], L["v_fresh"], kv, kv2, idx_out, None, a, b,
+                             hidden, None, ws) == api.DAF_ERR_INVALID_ARG
+    p0 = api.make_params(w.L_d, 0, w.r, 4, 2)
+    ws0 = api.alloc_workspace(p0)
+    qp = torch.zeros(k, 4, 128, dtype=torch.bfloat16, device=dev)
+    assert api.daf_layer(p0, L["scores"], 1, None, L["q_fresh"][: w.L_d], L["k_fresh"][: w.L_d], L["v_fresh"][: w.L_d],
+                         kv[: w.L_d], kv2[: w.L_d], idx_out, qp, None, None, hidden, None, ws0) == api.DAF_ERR_INVALID_ARG
 
 
 def test_work_list_shapes_drawn_at_random():
