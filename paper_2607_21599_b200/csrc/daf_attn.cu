@@ -422,6 +422,8 @@ constexpr int kSubN = 64;                               // keys per sub-step
 constexpr int kSubBytes = kSubN * kD * 2;               // 16 KB: K or V of one sub-step, two 64-column halves
 constexpr int kSubHalfBytes = kSubBytes / 2;
 constexpr int kAttnThreads = 192;                      // warps 0-3 softmax, warp 4 TMA, warp 5 MMA
+constexpr int kGatherWarps = 3;                        // form that fetches K/V rows in place: warps 4, 6 and 7 copy them
+constexpr int kAttnThreadsGather = 256;
 constexpr int kAttnTmemCols = 256;                     // S (two halves of 64) and O (128)
 
 struct AttnSmem {
@@ -436,7 +438,7 @@ struct AttnSmem {
 constexpr size_t kAttnSmemBytes = 1024 + 3 * (size_t)kTileBytes + sizeof(AttnSmem);
 
 template <bool kGatherKV>
-__global__ void __launch_bounds__(kAttnThreads, 2)
+__global__ void __launch_bounds__(kGatherKV ? kAttnThreadsGather : kAttnThreads, 2)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_constant__ CUtensorMap tmap_k0,
                   const __grid_constant__ CUtensorMap tmap_v0, const __grid_constant__ CUtensorMap tmap_q1,
                   const __grid_constant__ CUtensorMap tmap_k1, const __grid_constant__ CUtensorMap tmap_v1,
@@ -468,6 +470,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
     // non-null); a form of its own, so that the plain form carries none of that code
     const __nv_bfloat16* const k_src = kGatherKV ? DAF_SEG(k_src) : nullptr;
     const bool kv_gather = kGatherKV && k_src != nullptr;
+    const int gather_warp = warp == 4 ? 0 : warp - 5;    // 0, 1, 2 for warps 4, 6, 7 (meaningful only for those)
 
     // Loads K (kv = 0) or V (kv = 1) of sub-step t into its ring slot (the slot must be free).
     auto issue_kv = [&](int t, int kv) {
@@ -480,7 +483,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
         tma_load_3d(dst, tm, full, 0, g_kv, key0);
         tma_load_3d(dst + kSubHalfBytes, tm, full, 64, g_kv, key0);
     };
-    // The same for K/V rows fetched in place (the whole producer warp): row j of the sub-step is row idx[key0 + j] of
+    // The same for K/V rows fetched in place (three warps share the rows of a sub-step, every lane arrives on the
+    // slot's barrier): row j of the sub-step is row idx[key0 + j] of
     // the source tensor, copied by cp.async in 16-byte chunks into the layout the tiled load would have produced;
     // rows past the end are zero-filled.  pos_lo / pos_hi: this lane's source rows for sub-tile rows `lane` and
     // `32 + lane` (-1: none).  A copy group is handed to the tensor cores by kv_gather_arrive once it has landed.
@@ -499,8 +503,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
         const __nv_bfloat16* src = (kv == 0 ? k_src : DAF_SEG(v_src)) + (size_t)g_kv * kD;
         const size_t row_elems = (size_t)DAF_SEG(kv_heads) * kD;
         const int sub = lane >> 4, ch = lane & 15;
-#pragma unroll 8
-        for (int i = 0; i < 32; ++i) {
+#pragma unroll 4
+        for (int i = gather_warp; i < 32; i += kGatherWarps) {     // this warp's pairs of rows
             const int j = 2 * i + sub;
             const int pos = __shfl_sync(0xFFFFFFFFu, i < 16 ? pos_lo : pos_hi, j & 31);
             cp_async16(dst + (uint32_t)((ch >> 3) * kSubHalfBytes + j * 128 + (((ch & 7) ^ (j & 7)) << 4)),
@@ -532,7 +536,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
     if (warp == 4 && lane == 0) {
         mbar_init(&sm->q_full, q_idx != nullptr ? 4 : 1);
         for (int s = 0; s < 2; ++s) {
-            mbar_init(&sm->k_full[s], kv_gather ? 32 : 1); mbar_init(&sm->v_full[s], kv_gather ? 32 : 1);
+            mbar_init(&sm->k_full[s], kv_gather ? 32 * kGatherWarps : 1); mbar_init(&sm->v_full[s], kv_gather ? 32 * kGatherWarps : 1);
             mbar_init(&sm->s_full[s], 1); mbar_init(&sm->p_full[s], 4);
         }
         mbar_init(&sm->pv_done[0], 1); mbar_init(&sm->pv_done[1], 1);
@@ -562,15 +566,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
             }
             if (!kv_gather)
                 for (int t = 0; t < 2 && t < n_t; ++t) { issue_kv(t, 0); issue_kv(t, 1); }
-        }
-    }
-    if (warp == 4 && kv_gather) {
-        __syncwarp();              // the barriers that lane 0 prepared above, before the other lanes arrive on them
-        for (int t = 0; t < 2 && t < n_t; ++t) {
-            int pos_lo, pos_hi;
-            gather_positions(t, pos_lo, pos_hi);
-            gather_kv(t, 0, pos_lo, pos_hi);
-            gather_kv(t, 1, pos_lo, pos_hi);
         }
     }
     if (q_idx != nullptr && n_t > 0 && warp < 4) {
@@ -611,7 +606,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
 
     if (skip) {
         // nothing is computed; the loads already under way get a bounded chance to land before the CTA retires
-        if (warp == 4 && kv_gather) kv_gather_arrive(true);
         if (warp == 4 && lane == 0 && n_t > 0 && !kv_gather) {
             for (int i = 0; i < 4096 && !mbar_try_wait(&sm->q_full, 0); ++i) {}
             for (int s = 0; s < 2 && s < n_t; ++s) {
@@ -619,6 +613,26 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
                 for (int i = 0; i < 4096 && !mbar_try_wait(&sm->v_full[s], 0); ++i) {}
             }
         }
+    } else if (kv_gather && (warp == 4 || warp >= 6)) {
+        // ------------------------------------------------------------ producers of the form that fetches K/V rows in place
+        // (all sub-steps, after the set-up barrier: the barriers must be ready before three warps arrive on them)
+        bool ok = true;
+        for (int t = 0; t < n_t && ok; ++t) {
+            const int slot = t & 1;
+            const uint32_t round = (uint32_t)(t >> 1);
+            int pos_lo, pos_hi;
+            gather_positions(t, pos_lo, pos_hi);
+            for (int kv = 0; kv < 2 && ok; ++kv) {
+                if (t >= 2) {
+                    uint64_t* empty = kv == 0 ? &sm->s_full[slot] : &sm->pv_done[slot];
+                    ok = mbar_wait(empty, (round - 1) & 1u, abort_flag, status, 14 + 2 * kv + slot);
+                    ok = __all_sync(0xFFFFFFFFu, ok);
+                }
+                if (ok) gather_kv(t, kv, pos_lo, pos_hi);
+                __syncwarp();
+            }
+        }
+        kv_gather_arrive(true);   // the last copy group (also on the way out after a give-up: copies always land)
     } else if (warp == 4) {
         // ------------------------------------------------------------ TMA producer (the rest of the sub-steps)
         if (n_t > 2) {   // the whole warp walks the loop, one elected lane issues (uniform control flow)
@@ -626,20 +640,17 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
             for (int t = 2; t < n_t && ok; ++t) {
                 const int slot = t & 1;
                 const uint32_t round = (uint32_t)(t >> 1);
-                int pos_lo = -1, pos_hi = -1;
-                if (kv_gather) gather_positions(t, pos_lo, pos_hi);
                 for (int kv = 0; kv < 2 && ok; ++kv) {
                     // a K slot is free once the logits read from it are complete, a V slot once its product is:
                     // the barriers the softmax warps wait on say exactly that, so the issuer commits nothing extra
                     uint64_t* empty = kv == 0 ? &sm->s_full[slot] : &sm->pv_done[slot];
                     ok = mbar_wait(empty, (round - 1) & 1u, abort_flag, status, 10 + 2 * kv + slot);
                     ok = __all_sync(0xFFFFFFFFu, ok);
-                    if (ok && kv_gather) gather_kv(t, kv, pos_lo, pos_hi);
-                    else if (ok && elect_one()) issue_kv(t, kv);
+                    if (ok && elect_one()) issue_kv(t, kv);
                     __syncwarp();
                 }
             }
-            if (!ok && lane == 0 && !kv_gather) {
+            if (!ok && lane == 0) {
                 // give loads already in flight a bounded chance to land before the CTA retires
                 for (int s = 0; s < 2; ++s) {
                     for (int i = 0; i < 4096 && !mbar_try_wait(&sm->k_full[s], 0) && !mbar_try_wait(&sm->k_full[s], 1); ++i) {}
@@ -647,7 +658,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
                 }
             }
         }
-        if (kv_gather) kv_gather_arrive(true);   // the last copy group (also on the way out after a give-up: copies always land)
     } else if (warp == 5) {
         // ------------------------------------------------------------ MMA issuer
         // The whole warp walks the loop and waits on the barriers, one elected lane issues: control flow
@@ -722,7 +732,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
                 }
             }
         }
-    } else {
+    } else if (warp < 4) {
         // ------------------------------------------------------------ softmax + epilogue, one row per thread
         const int quad = warp;
         const int r = quad * 32 + lane;
@@ -1381,7 +1391,7 @@ int launch_attention_joint(const void* q_imp, const void* q_fresh, const int32_t
     const int items = jp.items_q + jp.items_i;
     if (launches & 1) {
         const cudaError_t e = gather_kv
-            ? launch_kernel(attn_fwd_kernel<true>, dim3((unsigned)items), dim3(kAttnThreads), kAttnSmemBytes, stream,
+            ? launch_kernel(attn_fwd_kernel<true>, dim3((unsigned)items), dim3(kAttnThreadsGather), kAttnSmemBytes, stream,
                             after_kernel, tq0, tk0, tv0, tq1, tk1, tv1, to0, to1, a)
             : launch_kernel(attn_fwd_kernel<false>, dim3((unsigned)items), dim3(kAttnThreads), kAttnSmemBytes, stream,
                             after_kernel, tq0, tk0, tv0, tq1, tk1, tv1, to0, to1, a);
