@@ -496,31 +496,45 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
             mbar_arrive(gather_pending);
         }
     };
-    auto gather_kv = [&](int t, int kv, int pos_lo, int pos_hi) {
-        const int slot = t & 1;
-        uint64_t* full = kv == 0 ? &sm->k_full[slot] : &sm->v_full[slot];
-        const uint32_t dst = smem_u32((kv == 0 ? k_smem : v_smem) + (size_t)slot * kSubBytes);
-        const __nv_bfloat16* src = (kv == 0 ? k_src : DAF_SEG(v_src)) + (size_t)g_kv * kD;
-        const size_t row_elems = (size_t)DAF_SEG(kv_heads) * kD;
+    // Byte offsets (within the K or V tensor) of the 16-byte chunks this lane copies for its warp's pairs of rows of
+    // sub-step t: computed once, used for K and for V.  -1: the row lies past the end (zero fill).
+    constexpr int kGatherPairs = (32 + kGatherWarps - 1) / kGatherWarps;
+    auto gather_offsets = [&](int t, long long (&off)[kGatherPairs]) {
+        const int key0 = key_begin + t * kSubN;
+        const int rows = DAF_SEG(kv_src_rows);
+        const int32_t* kv_idx = DAF_SEG(kv_idx);
+        int pos_lo = -1, pos_hi = -1;
+        if (key0 + lane < a.n_kv) { const int v = __ldg(kv_idx + key0 + lane); if ((unsigned)v < (unsigned)rows) pos_lo = v; }
+        if (key0 + 32 + lane < a.n_kv) { const int v = __ldg(kv_idx + key0 + 32 + lane); if ((unsigned)v < (unsigned)rows) pos_hi = v; }
+        const long long row_bytes = (long long)DAF_SEG(kv_heads) * kD * 2;
         const int sub = lane >> 4, ch = lane & 15;
-#pragma unroll 4
-        for (int i = gather_warp; i < 32; i += kGatherWarps) {     // this warp's pairs of rows
+#pragma unroll
+        for (int u = 0; u < kGatherPairs; ++u) {
+            const int i = gather_warp + u * kGatherWarps;          // pair of rows (2i, 2i + 1)
             const int j = 2 * i + sub;
             const int pos = __shfl_sync(0xFFFFFFFFu, i < 16 ? pos_lo : pos_hi, j & 31);
-            cp_async16(dst + (uint32_t)((ch >> 3) * kSubHalfBytes + j * 128 + (((ch & 7) ^ (j & 7)) << 4)),
-                       src + (size_t)(pos < 0 ? 0 : pos) * row_elems + ch * 8, pos < 0 ? 0u : 16u);
+            off[u] = (i < 32 && pos >= 0) ? (long long)pos * row_bytes + (long long)(g_kv * kD * 2 + ch * 16) : -1;
+        }
+    };
+    auto gather_kv = [&](int t, int kv, const long long (&off)[kGatherPairs]) {
+        const int slot = t & 1;
+        uint64_t* full = kv == 0 ? &sm->k_full[slot] : &sm->v_full[slot];
+        const char* src = reinterpret_cast<const char*>(kv == 0 ? k_src : DAF_SEG(v_src));
+        const int sub = lane >> 4, ch = lane & 15;
+        // this lane's chunk of row j lands at half (ch >> 3), row j, chunk ((ch & 7) ^ (j & 7)); j & 7 = ((2 i) & 7) | sub
+        const uint32_t dst = smem_u32((kv == 0 ? k_smem : v_smem) + (size_t)slot * kSubBytes) +
+                             (uint32_t)((ch >> 3) * kSubHalfBytes + sub * 128);
+        const uint32_t x = (uint32_t)((ch & 7) ^ sub);
+#pragma unroll
+        for (int u = 0; u < kGatherPairs; ++u) {
+            const int i = gather_warp + u * kGatherWarps;
+            if (i < 32)
+                cp_async16(dst + (uint32_t)(i * 256) + ((x ^ (uint32_t)((2 * i) & 7)) << 4),
+                           src + (off[u] < 0 ? 0 : off[u]), off[u] < 0 ? 0u : 16u);
         }
         cp_async_commit();
         kv_gather_arrive(false);                 // the group before this one has landed (or is waited for here)
         gather_pending = full;
-    };
-    auto gather_positions = [&](int t, int& pos_lo, int& pos_hi) {
-        const int key0 = key_begin + t * kSubN;
-        const int rows = DAF_SEG(kv_src_rows);
-        const int32_t* kv_idx = DAF_SEG(kv_idx);
-        pos_lo = pos_hi = -1;
-        if (key0 + lane < a.n_kv) { const int v = __ldg(kv_idx + key0 + lane); if ((unsigned)v < (unsigned)rows) pos_lo = v; }
-        if (key0 + 32 + lane < a.n_kv) { const int v = __ldg(kv_idx + key0 + 32 + lane); if ((unsigned)v < (unsigned)rows) pos_hi = v; }
     };
     // Set-up.  The producer thread prepares the barriers and at once starts the loads that need no free
     // slot (Q and the first two sub-steps), so that their latency overlaps the rest of the set-up: the
@@ -620,15 +634,15 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q0, const __grid_consta
         for (int t = 0; t < n_t && ok; ++t) {
             const int slot = t & 1;
             const uint32_t round = (uint32_t)(t >> 1);
-            int pos_lo, pos_hi;
-            gather_positions(t, pos_lo, pos_hi);
+            long long off[kGatherPairs];
+            gather_offsets(t, off);
             for (int kv = 0; kv < 2 && ok; ++kv) {
                 if (t >= 2) {
                     uint64_t* empty = kv == 0 ? &sm->s_full[slot] : &sm->pv_done[slot];
                     ok = mbar_wait(empty, (round - 1) & 1u, abort_flag, status, 14 + 2 * kv + slot);
                     ok = __all_sync(0xFFFFFFFFu, ok);
                 }
-                if (ok) gather_kv(t, kv, pos_lo, pos_hi);
+                if (ok) gather_kv(t, kv, off);
                 __syncwarp();
             }
         }
