@@ -53,11 +53,12 @@ def _workload(name):
     return {w.name: w for w in W.sweep_points(api.daf_num_important)}[name]
 
 
-def _layer_parity(name, layer, rows_imp, rows_q, n_full_rows, hoisted=False):
+def _layer_parity(name, layer, rows_imp, rows_q, n_full_rows, hoisted=False, kv_in_place=False):
     """Runs one layer the way the benchmark does and compares it with the oracle.  rows_imp / rows_q:
     None = every row, an int = that many sampled rows, "edges:<n>" = every tile edge and n rows in all.
     hoisted: the benchmark's schedule -- the selection alone on a second stream (daf_select_topk), then the layer
-    from those positions (idx_in) on the main stream; otherwise daf_layer from the scores on one stream."""
+    from those positions (idx_in) on the main stream; otherwise daf_layer from the scores on one stream.
+    kv_in_place: no packed K/V buffers are given, the attention kernel fetches those rows through the positions."""
     assert torch.cuda.is_available()
     build.build()
     w = _workload(name)
@@ -85,9 +86,10 @@ def _layer_parity(name, layer, rows_imp, rows_q, n_full_rows, hoisted=False):
     def run():
         # as the benchmark calls it: from 16384 important tokens on without a packed copy of the Q rows
         qp = None if k >= 16384 else q_pack
+        kp, vp = (None, None) if kv_in_place else (k_pack, v_pack)
         if not hoisted:
             api.check(api.daf_layer(p, L["scores"], n_sig, None, L["q_fresh"], L["k_fresh"], L["v_fresh"], kv_k, kv_v,
-                                    idx_out, qp, k_pack, v_pack, hidden, None, ws), "daf_layer")
+                                    idx_out, qp, kp, vp, hidden, None, ws), "daf_layer")
             return
         main = torch.cuda.current_stream()
         side.wait_stream(main)
@@ -96,7 +98,7 @@ def _layer_parity(name, layer, rows_imp, rows_q, n_full_rows, hoisted=False):
         done.record(side)
         main.wait_event(done)
         api.check(api.daf_layer(p, None, 0, idx_sel, L["q_fresh"], L["k_fresh"], L["v_fresh"], kv_k, kv_v,
-                                idx_out, qp, k_pack, v_pack, hidden, None, ws, stream=main), "daf_layer")
+                                idx_out, qp, kp, vp, hidden, None, ws, stream=main), "daf_layer")
         main.wait_stream(side)
 
     run()  # eager once (sets kernel attributes), then the timed configuration: a graph replay
@@ -116,6 +118,8 @@ def _layer_parity(name, layer, rows_imp, rows_q, n_full_rows, hoisted=False):
     assert np.array_equal(idx_out.cpu().numpy(), idx), "selected positions differ"
     idx_t = torch.from_numpy(idx).long().to(dev)
     q_pack = L["q_fresh"][idx_t]          # what a packed copy would hold (the layer may not have written one)
+    if kv_in_place:
+        k_pack, v_pack = L["k_fresh"][idx_t], L["v_fresh"][idx_t]
     assert torch.equal(k_pack, L["k_fresh"][idx_t])
     assert torch.equal(v_pack, L["v_fresh"][idx_t])
     exp_k = torch.cat([L["k_cached"], L["k_fresh"][w.L_d:]], 0)
@@ -178,6 +182,11 @@ def test_c4_every_sweep_point(name):
     w = _workload(name)
     big = w.N > 8320
     _layer_parity(name, 0, 96 if big else None, 32 if big else None, 0 if big else 64)
+
+
+@pytest.mark.parametrize("name,layer,rows_imp", [("c1", 5, None), ("c2", 7, None), ("c3", 9, "edges:544")])
+def test_step_2_fed_from_the_unpacked_key_value_rows(name, layer, rows_imp):
+    _layer_parity(name, layer, rows_imp, None, 0, hoisted=True, kv_in_place=True)
 
 
 def test_x136k_sampled_rows():
