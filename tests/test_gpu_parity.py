@@ -848,6 +848,44 @@ def test_layer_rejects_half_a_pair_of_packed_kv_buffers():
                          kv[: w.L_d], kv2[: w.L_d], idx_out, qp, None, None, hidden, None, ws0) == api.DAF_ERR_INVALID_ARG
 
 
+def test_layers_drawn_at_random():
+    """Seeded random layers through daf_layer against the oracle: group sizes 1-8, document lengths that leave ragged
+    tiles, one to a few hundred question tokens, r from 0.05 to 1, both fusion modes, with and without the cache
+    overwrite, with and without packed Q and packed K/V buffers."""
+    rng = np.random.default_rng(20261125)
+    dev = "cuda"
+    for case in range(24):
+        Hkv = int(rng.choice([1, 2, 4, 8]))
+        Hq = min(Hkv * int(rng.choice([1, 2, 4, 7, 8])), 32 // Hkv * Hkv)
+        L_d, L_q = int(rng.integers(130, 2600)), int(rng.integers(1, 200))
+        r = float(rng.choice([0.05, 0.1, 0.2, 0.3, 0.5, 0.9, 1.0]))
+        fuse, ow = int(rng.integers(0, 2)), int(rng.integers(0, 2))
+        with_q, with_kv = bool(rng.integers(0, 2)), bool(rng.integers(0, 2))
+        w = W.Workload("f", int(rng.integers(1, 1000)), Hq, Hkv, 128, 1, L_d, 500, L_q, r, "lognormal", int(rng.integers(1, 4)))
+        L = W.make_layer(w, 0)
+        p = api.make_params(L_d, L_q, r, Hq, Hkv, fuse_mode=fuse, overwrite_doc_kv=ow)
+        k = api.daf_num_important(L_d, r)
+        g = {n: (None if t is None else t.to(dev)) for n, t in L.items()}
+        ws = api.alloc_workspace(p)
+        kv_k = torch.zeros(w.N, Hkv, 128, dtype=torch.bfloat16, device=dev)
+        kv_v = torch.zeros_like(kv_k)
+        kv_k[:L_d], kv_v[:L_d] = g["k_cached"], g["v_cached"]
+        idx_out = torch.full((k,), -1, dtype=torch.int32, device=dev)
+        qp = torch.zeros(k, Hq, 128, dtype=torch.bfloat16, device=dev) if with_q else None
+        kp = torch.zeros(k, Hkv, 128, dtype=torch.bfloat16, device=dev) if with_kv else None
+        vp = torch.zeros(k, Hkv, 128, dtype=torch.bfloat16, device=dev) if with_kv else None
+        rows = k + L_q if fuse == 0 else w.N
+        hidden = torch.full((rows, Hq, 128), -9.0, dtype=torch.bfloat16, device=dev)
+        what = f"case {case}: L_d={L_d} L_q={L_q} r={r} Hq={Hq} Hkv={Hkv} fuse={fuse} overwrite={ow} q_pack={with_q} kv_pack={with_kv}"
+        _ok(api.daf_layer(p, g["scores"], L["scores"].shape[0], None, g["q_fresh"], g["k_fresh"], g["v_fresh"], kv_k, kv_v,
+                          idx_out, qp, kp, vp, hidden, None, ws), ws, what)
+        ref = _oracle_layer(w, L, fuse, overwrite=ow)
+        assert np.array_equal(idx_out.cpu().numpy(), ref["idx"]), what
+        assert np.array_equal(_f(kv_k), ref["kv_k"]) and np.array_equal(_f(kv_v), ref["kv_v"]), what
+        sel = np.arange(len(ref["row_pos"])) if fuse == 0 else ref["row_pos"]
+        _assert_close(hidden.cpu()[sel], ref["hidden"][sel], what)
+
+
 def test_work_list_shapes_drawn_at_random():
     """Seeded random shapes through daf_imp_qd_attn: group sizes 1-8, condensed sequences around multiples of
     the 128-row tile and of the 64-key sub-step, question blocks that see different numbers of key tiles."""
