@@ -397,14 +397,19 @@ def measure_config(env: Env, w: W.Workload, primary: bool):
     with ClockSampler(env.local_rank) as clocks:
         barrier()
         e0.record(stream)
+        marks = []                      # one event after every step (on the same stream: they cost nothing measurable)
         for _ in range(args.steps):
             if use_graph:
                 g_step.replay()
             else:
                 step()
+            m = torch.cuda.Event(enable_timing=True)
+            m.record(stream)
+            marks.append(m)
         e1.record(stream)
         barrier()
     ms_total = e0.elapsed_time(e1)
+    step_ms = [a.elapsed_time(b) for a, b in zip([e0] + marks[:-1], marks)]
     launches = launches_per_step * args.steps if use_graph else api.daf_launch_count() - launches0
     api.check(api.daf_poll_status(ws), "timed region (device status)")
     ms_total = max_over_ranks(dist, ms_total, dev)
@@ -661,6 +666,7 @@ def measure_config(env: Env, w: W.Workload, primary: bool):
     flop_ratio = flops["full"] / daf_flops
     res = {
         "value": us_per_layer, "unit": UNIT, "ms_per_step": ms_per_step, "config": _config_dict(w, world),
+        "ms_per_step_median": float(statistics.median(step_ms)), "ms_per_step_min": float(min(step_ms)),
         "tflops": tflops, "frac_of_bf16_peak": tflops / (peaks["bf16_tflops"] * world),
         "roofline": roofline,
         "schedule": ("selection of every layer on a second stream (daf_select_topk), layers from idx_in on the main one"
