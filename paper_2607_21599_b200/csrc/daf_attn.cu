@@ -1207,7 +1207,7 @@ JointPlan plan_joint(int k, int L_q, int L_d, int Hq, int G) {
     return best;
 }
 
-#ifdef DAF_TRACE
+#if defined(DAF_TRACE) || defined(DAF_TUNE)     // tuning builds: pin the planner's choice, read its prediction
 extern "C" void daf_dbg_joint_force(int chunk, int n_splits_q) { g_force_chunk = chunk; g_force_splits_q = n_splits_q; }
 extern "C" float daf_dbg_joint_predicted_us(void) { return g_last_predicted_us; }
 extern "C" void daf_dbg_joint_plan(int k, int L_q, int L_d, int Hq, int G, int* out) {
