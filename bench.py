@@ -643,11 +643,21 @@ def measure_config(env: Env, w: W.Workload, primary: bool):
         torch.cuda.synchronize()
         dt = time.perf_counter() - t0
         dt = max_over_ranks(dist, dt, dev)
+        # what crosses the link per layer: the scores, the document rows of the offline cache, the question's Q rows
+        # (copies) and the fresh Q/K/V rows of the important tokens and K/V rows of the question, which the gather /
+        # cache-update kernel reads straight from the pinned host tensors; the rest of the fresh tensors stays on the host
+        kv_row = 2 * w.n_kv_heads * 256
+        crossing = (w.L_d * 4 * max(bufs[0].n_sig, 1) + w.L_d * kv_row + w.L_q * row_bytes +
+                    w.k * (row_bytes + kv_row) + w.L_q * kv_row)
         e2e = {"value": dt / e2e_steps / (n_e2e * world) * 1e6, "unit": UNIT,
-               "h2d_bytes_per_step": int(per_layer_in * n_e2e), "d2h_bytes_per_step": int((w.k + w.L_q) * row_bytes * n_e2e),
+               "h2d_bytes_per_step": int(crossing * n_e2e), "d2h_bytes_per_step": int((w.k + w.L_q) * row_bytes * n_e2e),
+               "host_input_bytes_per_step": int(per_layer_in * n_e2e),
                "layers_per_step": n_e2e, "steps": e2e_steps,
                "api": "daf_layer_host_begin / daf_layer_host_end on two arenas and two streams (pinned host tensors in, "
-                      "hidden rows out; every layer's result is waited for inside the timed region)"}
+                      "hidden rows out; every layer's result is waited for inside the timed region); of the fresh "
+                      "tensors only the rows of the important tokens and of the question cross the link "
+                      "(h2d_bytes_per_step), read in place by the gather kernel; host_input_bytes_per_step is the size "
+                      "of all host input tensors"}
         del arenas, host
 
     # ---- CPU oracle on this machine's cores, bounded sample (rank 0, N = 1 only)

@@ -293,6 +293,10 @@ int daf_layer_fp8(const daf_params* p, const float* scores, int32_t n_sig, const
  *   h_hidden        host output, layout by fuse_mode (compact mode recommended)
  *   h_idx_out       host int32 [k] (optional)
  * The call synchronises `stream` before returning.
+ * Of the fresh tensors a layer touches only the rows of the important tokens and of the question: when h_q_fresh,
+ * h_k_fresh and h_v_fresh are all pinned memory that the device can address, those rows are read straight from the
+ * host by the gather / cache-update kernel (k + L_q rows cross the link instead of N) and only the question's Q rows
+ * are copied; otherwise the three tensors are copied whole.  Same results either way.
  *
  * daf_layer_host_begin / daf_layer_host_end are the two halves of that call: `begin` (same arguments) enqueues the
  * copies in, the layer and the copies out on `stream` and returns without waiting; `end` waits for `stream` and

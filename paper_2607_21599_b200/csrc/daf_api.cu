@@ -307,18 +307,22 @@ int daf_full_causal_attn(const daf_params* p, int32_t n_tokens, const void* q, c
 namespace {
 // Offline cache of one layer kept in fp8 (daf_layer_fp8): expanded into kv_k / kv_v ahead of everything else.
 struct Fp8Cache { const void* k8; const void* v8; const float* k_scale; const float* v_scale; };
+// Where the gather / cache-update kernel reads the fresh rows when that is not the tensors the attention reads the
+// question rows from: device-accessible pointers to [N, heads, 128] tensors (mapped pinned host memory).
+struct RowSource { const void* q; const void* k; const void* v; };
 
 int layer_impl(const daf_params* p, const Fp8Cache* fp8, const float* scores, int32_t n_sig, const int32_t* idx_in,
                const void* q_fresh, const void* k_fresh, const void* v_fresh, void* kv_k, void* kv_v,
                int32_t* idx_out, void* q_pack, void* k_pack, void* v_pack,
                void* hidden, int32_t* row_pos_out,
-               void* workspace, size_t workspace_bytes_, void* stream) {
+               void* workspace, size_t workspace_bytes_, void* stream, const RowSource* rows = nullptr) {
     ResolvedParams rp;
     if (int rc = resolve_params(p, &rp)) return rc;
     Workspace ws;
     if (int rc = carve_workspace(rp, workspace, workspace_bytes_, &ws)) return rc;
     cudaStream_t st = (cudaStream_t)stream;
     if (rp.k + rp.L_q == 0) return DAF_OK;
+    if (rows != nullptr && (q_pack == nullptr || k_pack == nullptr)) return DAF_ERR_INVALID_ARG;   // only the gather kernel reads them
     if (fp8 != nullptr) {
         if (rp.L_d > 0 && (!fp8->k8 || !fp8->v8 || !kv_k || !kv_v)) return DAF_ERR_INVALID_ARG;
         if (!aligned16(fp8->k8) || !aligned16(fp8->v8) || !aligned16(kv_k) || !aligned16(kv_v)) return DAF_ERR_ALIGNMENT;
@@ -337,7 +341,8 @@ int layer_impl(const daf_params* p, const Fp8Cache* fp8, const float* scores, in
     // the expanded cache) runs behind both.
     if (fp8 != nullptr)
         if (int rc = launch_expand_fp8(rp, fp8->k8, fp8->v8, fp8->k_scale, fp8->v_scale, kv_k, kv_v, st)) return rc;
-    if (int rc = do_select(rp, scores, n_sig, idx_in, q_fresh, k_fresh, v_fresh, kv_k, kv_v, idx_out, q_pack, k_pack,
+    if (int rc = do_select(rp, scores, n_sig, idx_in, rows ? rows->q : q_fresh, rows ? rows->k : k_fresh,
+                           rows ? rows->v : v_fresh, kv_k, kv_v, idx_out, q_pack, k_pack,
                            v_pack, ws, st, false, /*beside_previous_kernel=*/fp8 != nullptr && rp.L_d > 0)) return rc;
     char* h = reinterpret_cast<char*>(hidden);
     // State fusion is done by the attention epilogues: each stage writes its final rows.  When both
@@ -458,6 +463,15 @@ constexpr int kArenaSignalRows = 8;   // arena is sized for up to this many sign
 // From this many important tokens on the host-buffer layer skips the packed copy of the Q rows (step 2 reads
 // them in place): measured -2 % layer time at k = 41780, +-1 % at k = 6554, +10 % at k = 922.
 constexpr int kQInPlaceMinK = 16384;
+
+// True (and *dev set) when `h` is pinned host memory that kernels on the current device can address.
+bool mapped_host_pointer(const void* h, const void** dev) {
+    cudaPointerAttributes attr;
+    if (cudaPointerGetAttributes(&attr, h) != cudaSuccess) { (void)cudaGetLastError(); return false; }
+    if (attr.type != cudaMemoryTypeHost || attr.devicePointer == nullptr) return false;
+    *dev = attr.devicePointer;
+    return true;
+}
 }  // namespace
 
 size_t daf_layer_host_arena_bytes(const daf_params* p) {
@@ -489,16 +503,31 @@ int daf_layer_host_begin(const daf_params* p, const float* h_scores, int32_t n_s
     DAF_CUDA_TRY(cudaMemsetAsync(a.ws, 0, kStatusBytes, st));
     if (h_scores) DAF_CUDA_TRY(cudaMemcpyAsync(a.scores, h_scores, (size_t)n_sig * rp.L_d * 4, cudaMemcpyHostToDevice, st));
     else if (rp.k > 0) DAF_CUDA_TRY(cudaMemcpyAsync(a.idx_in, h_idx_in, (size_t)rp.k * 4, cudaMemcpyHostToDevice, st));
-    DAF_CUDA_TRY(cudaMemcpyAsync(a.q_fresh, h_q_fresh, qrow * rp.N, cudaMemcpyHostToDevice, st));
-    DAF_CUDA_TRY(cudaMemcpyAsync(a.k_fresh, h_k_fresh, kvrow * rp.N, cudaMemcpyHostToDevice, st));
-    DAF_CUDA_TRY(cudaMemcpyAsync(a.v_fresh, h_v_fresh, kvrow * rp.N, cudaMemcpyHostToDevice, st));
+    // Of the fresh tensors the layer touches only the rows of the important tokens and of the question.  When the
+    // three host tensors are pinned memory that the device can address, the gather / cache-update kernel reads those
+    // rows straight from the host (k + L_q rows instead of N cross the link) and only the question's Q rows, which
+    // the attention kernel reads through a tensor map, are copied; otherwise the tensors are copied whole.
+    RowSource rows = {nullptr, nullptr, nullptr};
+    const bool in_place_rows = rp.k > 0 && mapped_host_pointer(h_q_fresh, &rows.q) && mapped_host_pointer(h_k_fresh, &rows.k) &&
+                               mapped_host_pointer(h_v_fresh, &rows.v);
+    if (in_place_rows) {
+        if (rp.L_q > 0)
+            DAF_CUDA_TRY(cudaMemcpyAsync(reinterpret_cast<char*>(a.q_fresh) + qrow * rp.L_d,
+                                         reinterpret_cast<const char*>(h_q_fresh) + qrow * rp.L_d, qrow * rp.L_q,
+                                         cudaMemcpyHostToDevice, st));
+    } else {
+        DAF_CUDA_TRY(cudaMemcpyAsync(a.q_fresh, h_q_fresh, qrow * rp.N, cudaMemcpyHostToDevice, st));
+        DAF_CUDA_TRY(cudaMemcpyAsync(a.k_fresh, h_k_fresh, kvrow * rp.N, cudaMemcpyHostToDevice, st));
+        DAF_CUDA_TRY(cudaMemcpyAsync(a.v_fresh, h_v_fresh, kvrow * rp.N, cudaMemcpyHostToDevice, st));
+    }
     // only the document rows of the cache carry information on entry
     DAF_CUDA_TRY(cudaMemcpyAsync(a.kv_k, h_kv_k, kvrow * rp.L_d, cudaMemcpyHostToDevice, st));
     DAF_CUDA_TRY(cudaMemcpyAsync(a.kv_v, h_kv_v, kvrow * rp.L_d, cudaMemcpyHostToDevice, st));
-    if (int rc = daf_layer(p, h_scores ? a.scores : nullptr, n_sig, h_scores ? nullptr : a.idx_in, a.q_fresh, a.k_fresh,
-                           a.v_fresh, a.kv_k, a.kv_v, a.idx_out, (rp.k >= kQInPlaceMinK && rp.L_q > 0) ? nullptr : a.q_pack, a.k_pack,
-                           a.v_pack, a.hidden, nullptr, a.ws,
-                           a.ws_bytes, stream)) return rc;
+    // (rows read from the host: always with packed copies on the device, the attention kernel must not go to the host)
+    void* qp = (!in_place_rows && rp.k >= kQInPlaceMinK && rp.L_q > 0) ? nullptr : a.q_pack;
+    if (int rc = layer_impl(p, nullptr, h_scores ? a.scores : nullptr, n_sig, h_scores ? nullptr : a.idx_in, a.q_fresh, a.k_fresh,
+                            a.v_fresh, a.kv_k, a.kv_v, a.idx_out, qp, a.k_pack, a.v_pack, a.hidden, nullptr, a.ws, a.ws_bytes, stream,
+                            in_place_rows ? &rows : nullptr)) return rc;
     const size_t hidden_rows = rp.fuse_mode == 1 ? rp.N : rp.k + rp.L_q;
     DAF_CUDA_TRY(cudaMemcpyAsync(h_hidden, a.hidden, qrow * hidden_rows, cudaMemcpyDeviceToHost, st));
     if (h_idx_out && rp.k > 0) DAF_CUDA_TRY(cudaMemcpyAsync(h_idx_out, a.idx_out, (size_t)rp.k * 4, cudaMemcpyDeviceToHost, st));

@@ -442,6 +442,35 @@ def _oracle_layer(w, L, fuse_mode, overwrite=1):
                             overwrite=bool(overwrite), hidden=base)
 
 
+def test_host_layer_from_pageable_and_from_pinned_fresh_tensors_agree():
+    """daf_layer_host reads the needed fresh rows straight from pinned host tensors and copies pageable ones whole:
+    the same bits either way."""
+    w = W.Workload("t", 37, 8, 2, 128, 1, 1100, 500, 33, 0.3, "lognormal", 1)
+    dev = "cuda"
+    p = api.make_params(w.L_d, w.L_q, w.r, w.n_q_heads, w.n_kv_heads)
+    k = api.daf_num_important(w.L_d, w.r)
+    L = W.make_layer(w, 0)
+    arena = torch.zeros(api.daf_layer_host_arena_bytes(p), dtype=torch.uint8, device=dev)
+    outs = []
+    for pinned in (True, False):
+        fresh = {n: (L[n].pin_memory() if pinned else L[n].clone()) for n in ("q_fresh", "k_fresh", "v_fresh")}
+        assert all(t.is_pinned() == pinned for t in fresh.values())
+        kv_k = torch.zeros(w.N, w.n_kv_heads, 128, dtype=torch.bfloat16)
+        kv_v = torch.zeros_like(kv_k)
+        kv_k[: w.L_d], kv_v[: w.L_d] = L["k_cached"], L["v_cached"]
+        hidden = torch.full((k + w.L_q, w.n_q_heads, 128), -9.0, dtype=torch.bfloat16).pin_memory()
+        idx_out = torch.full((k,), -1, dtype=torch.int32)
+        api.check(api.daf_layer_host(p, L["scores"], 1, None, fresh["q_fresh"], fresh["k_fresh"], fresh["v_fresh"], kv_k, kv_v, 1,
+                                     hidden, idx_out, arena), "daf_layer_host")
+        outs.append((hidden.clone(), idx_out, kv_k, kv_v))
+    for a, b in zip(outs[0], outs[1]):
+        assert torch.equal(a, b)
+    ref = _oracle_layer(w, L, 0)
+    assert np.array_equal(outs[0][1].numpy(), ref["idx"])
+    assert np.array_equal(_f(outs[0][2]), ref["kv_k"]) and np.array_equal(_f(outs[0][3]), ref["kv_v"])
+    _assert_close(outs[0][0], ref["hidden"], "hidden rows from pinned host tensors")
+
+
 def test_host_layers_pipelined_on_two_arenas_match_the_plain_host_call():
     """daf_layer_host_begin / _end with two arenas and two streams (layer i + 1 begun before layer i is ended) give,
     layer by layer, exactly what daf_layer_host gives."""
