@@ -94,7 +94,7 @@ static int carve_workspace(const ResolvedParams& rp, void* workspace, size_t byt
 static int do_select(const ResolvedParams& rp, const float* scores, int32_t n_sig, const int32_t* idx_in,
                      const void* q_fresh, const void* k_fresh, const void* v_fresh, void* kv_k, void* kv_v,
                      int32_t* idx_out, void* q_pack, void* k_pack, void* v_pack, const Workspace& ws, cudaStream_t st,
-                     bool scores_from_previous_kernel = false, bool beside_previous_kernel = false) {
+                     bool scores_from_previous_kernel = false, bool beside_previous_kernel = false, bool rows_far = false) {
     if (scores != nullptr && n_sig < 1) return DAF_ERR_INVALID_ARG;
     if (rp.k > 0) {
         if (scores == nullptr && idx_in == nullptr) return DAF_ERR_INVALID_ARG;
@@ -109,7 +109,8 @@ static int do_select(const ResolvedParams& rp, const float* scores, int32_t n_si
     for (const void* ptr : ptrs)
         if (ptr != nullptr && !aligned16(ptr)) return DAF_ERR_ALIGNMENT;
     return launch_select(rp, scores, n_sig, idx_in, q_fresh, k_fresh, v_fresh, kv_k, kv_v, idx_out, q_pack, k_pack,
-                         v_pack, ws.status, ws.select_scratch, st, scores_from_previous_kernel, beside_previous_kernel);
+                         v_pack, ws.status, ws.select_scratch, st, scores_from_previous_kernel, beside_previous_kernel,
+                         /*select_only=*/false, rows_far);
 }
 
 static int check_out(const void* out, int64_t stride_bytes, int Hq) {
@@ -343,7 +344,8 @@ int layer_impl(const daf_params* p, const Fp8Cache* fp8, const float* scores, in
         if (int rc = launch_expand_fp8(rp, fp8->k8, fp8->v8, fp8->k_scale, fp8->v_scale, kv_k, kv_v, st)) return rc;
     if (int rc = do_select(rp, scores, n_sig, idx_in, rows ? rows->q : q_fresh, rows ? rows->k : k_fresh,
                            rows ? rows->v : v_fresh, kv_k, kv_v, idx_out, q_pack, k_pack,
-                           v_pack, ws, st, false, /*beside_previous_kernel=*/fp8 != nullptr && rp.L_d > 0)) return rc;
+                           v_pack, ws, st, false, /*beside_previous_kernel=*/fp8 != nullptr && rp.L_d > 0,
+                           /*rows_far=*/rows != nullptr)) return rc;
     char* h = reinterpret_cast<char*>(hidden);
     // State fusion is done by the attention epilogues: each stage writes its final rows.  When both
     // stages have rows they run as one list of work items in one launch, right behind the gather

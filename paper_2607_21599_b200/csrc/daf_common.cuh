@@ -41,7 +41,7 @@ int launch_select(const ResolvedParams& rp, const float* scores, int n_sig, cons
                   const void* q_fresh, const void* k_fresh, const void* v_fresh, void* kv_k, void* kv_v,
                   int32_t* idx_out, void* q_pack, void* k_pack, void* v_pack,
                   DeviceStatus* status, void* scratch, cudaStream_t stream, bool scores_from_previous_kernel = false,
-                  bool beside_previous_kernel = false, bool select_only = false);
+                  bool beside_previous_kernel = false, bool select_only = false, bool rows_far = false);
 int launch_check_indices(const int32_t* idx, int k, int L_d, DeviceStatus* status, cudaStream_t stream);
 int launch_expand_fp8(const ResolvedParams& rp, const void* k8, const void* v8, const float* k_scale, const float* v_scale,
                       void* kv_k, void* kv_v, cudaStream_t stream);
