@@ -1078,7 +1078,8 @@ namespace {
 constexpr float kCostItemUs = 7.0f;        // set-up, first logits and row epilogue of an item (5-6 us alone; fitted)
 constexpr float kCostSubStepUs = 1.05f;    // 64 keys through one tile with two CTAs per SM (measured 0.95-1.1 us)
 constexpr float kCostMergeUs = 2.0f;       // merge launch
-constexpr float kCostMergeUsPerMB = 0.15f; // plus re-reading the partial rows (fitted together with the item cost)
+constexpr float kCostMergeUsPerMB = 0.15f; // plus re-reading the partial rows of the question ranges (fitted together with the item cost)
+constexpr float kCostMergeUsPerMBCut = 0.45f;  // partial rows of cut causal chains (measured: 7.0 us for 14.8 MB, 13.3 for 25, 42.6 for 96)
 
 int g_force_chunk = 0, g_force_splits_q = 0;   // tuning builds can pin the choice
 float g_last_predicted_us = 0.f;
@@ -1149,9 +1150,10 @@ float predict_us(const JointPlan& jp, int k, int L_q, int L_d, int Hq) {
         if (g >= 1) part_rows_i += (size_t)kBlockM * Hq;
     }
     (void)k;
-    const float merge_mb = (float)(jp.part_bytes_q + part_rows_i * 516) / 1e6f;
+    const float merge_us = kCostMergeUs + kCostMergeUsPerMB * (float)jp.part_bytes_q / 1e6f +
+                           kCostMergeUsPerMBCut * (float)(part_rows_i * 516) / 1e6f;
     const bool merges = jp.n_splits_q > 1 || jp.chunk < jp.n_tb_i;
-    return makespan + (merges ? kCostMergeUs + kCostMergeUsPerMB * merge_mb : 0.f);
+    return makespan + (merges ? merge_us : 0.f);
 }
 }  // namespace
 
